@@ -1,0 +1,704 @@
+/*
+ * CPU oracle for the Fed-CVLC per-round compression path (test infrastructure
+ * only; see cvlc_oracle.h).  One thread, plain loops, the paper's steps in the
+ * paper's order.  Build: gcc -O2 -ffp-contract=off -shared -fPIC.
+ *
+ * Notation follows the paper: d coordinates, k transmitted, R packets, P_r
+ * records in packet r, y_r bits per value, s bits per position ID, b packet
+ * bits, H header bits, B the scale-down constant, beta = 2*alpha + 1.
+ */
+#include "cvlc_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ======================================================================== */
+/* Spec math: log2 / exp2 built from IEEE + - * / only, so that any machine   */
+/* that evaluates the same operations in the same order gets the same bits.  */
+/* ======================================================================== */
+
+static double bits_to_double(uint64_t u) {
+  double v;
+  memcpy(&v, &u, 8);
+  return v;
+}
+static uint64_t double_to_bits(double v) {
+  uint64_t u;
+  memcpy(&u, &v, 8);
+  return u;
+}
+
+/* log2 of a positive, finite, normal double.
+ * v = m * 2^e with m in [1,2); fold m into (sqrt(1/2), sqrt(2)];
+ * ln m = 2 atanh(t), t = (m-1)/(m+1), as the odd series up to t^25. */
+double cvlc_log2_oracle(double v) {
+  uint64_t bits = double_to_bits(v);
+  int e = (int)((bits >> 52) & 0x7FF) - 1023;
+  double m = bits_to_double((bits & 0x000FFFFFFFFFFFFFull) | 0x3FF0000000000000ull);
+  if (m > 1.4142135623730951) {
+    m = m / 2.0;
+    e = e + 1;
+  }
+  double t = (m - 1.0) / (m + 1.0);
+  double q = t * t;
+  double p = 1.0 / 25.0;
+  for (int j = 11; j >= 0; --j) p = p * q + 1.0 / (double)(2 * j + 1);
+  double ln_m = (2.0 * t) * p;
+  return (double)e + ln_m * 1.4426950408889634;
+}
+
+/* 2^v for |v| <= 1000: v = n + r, |r| <= 1/2, e^(r ln 2) as a degree-20 Taylor
+ * polynomial in Horner form, then n added to the exponent field. */
+double cvlc_exp2_oracle(double v) {
+  double n = floor(v + 0.5);
+  double r = v - n;
+  double u = r * 0.6931471805599453;
+  double p = 1.0;
+  for (int j = 20; j >= 1; --j) p = 1.0 + (u / (double)j) * p;
+  int64_t ni = (int64_t)n;
+  uint64_t pb = double_to_bits(p);
+  pb = (uint64_t)((int64_t)pb + ni * ((int64_t)1 << 52));
+  return bits_to_double(pb);
+}
+
+/* a^beta for a >= 1 */
+double cvlc_powr_oracle(double a, double beta) { return cvlc_exp2_oracle(beta * cvlc_log2_oracle(a)); }
+
+/* ======================================================================== */
+/* Philox4x32-10, written from the published definition (Salmon, Moraes,     */
+/* Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11).        */
+/* ======================================================================== */
+
+void cvlc_philox4x32_10_oracle(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+    uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+    uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    uint32_t n0 = hi1 ^ c1 ^ k0;
+    uint32_t n1 = lo1;
+    uint32_t n2 = hi0 ^ c3 ^ k1;
+    uint32_t n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The random word of coordinate `coord`: counter (coord lo, coord hi, client, round),
+ * key (seed lo, seed hi), output word 0. */
+uint32_t cvlc_philox_coord_oracle(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t coord) {
+  uint32_t ctr[4] = {(uint32_t)coord, (uint32_t)(coord >> 32), client_id, round};
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  cvlc_philox4x32_10_oracle(ctr, key, out);
+  return out[0];
+}
+
+/* ======================================================================== */
+/* Keys, histogram, power-law exponent (Definition 1; Algorithm 1, step 1)   */
+/* ======================================================================== */
+
+static uint32_t key_of(float x) {
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  return u & 0x7FFFFFFFu;
+}
+
+/* h[j] = number of coordinates whose magnitude key has top bits j
+ * (8 exponent bits and the 4 leading mantissa bits). */
+int cvlc_histogram_oracle(const float* x, uint64_t d, uint64_t h[ORC_HIST_BINS]) {
+  memset(h, 0, sizeof(uint64_t) * ORC_HIST_BINS);
+  int nonfinite = 0;
+  for (uint64_t i = 0; i < d; ++i) {
+    uint32_t key = key_of(x[i]);
+    if (key >= 0x7F800000u) nonfinite = 1;
+    h[key >> 19] += 1;
+  }
+  return nonfinite ? ORC_ERR_NONFINITE_INPUT : ORC_OK;
+}
+
+/* Least squares of log2|U{l}| on log2 l (Definition 1: |U{l}| <= phi * l^alpha)
+ * over the histogram's survival counts: the point of bin j is
+ * (log2 N_j, log2 of the bin's lower edge), N_j = #{key >> 19 >= j}, for the
+ * non-empty normal bins in the upper half of the ranks. */
+void cvlc_alpha_fit_oracle(const uint64_t h[ORC_HIST_BINS], uint64_t d, double* alpha, double* alpha_q) {
+  static uint64_t N[ORC_HIST_BINS + 1];
+  N[ORC_HIST_BINS] = 0;
+  for (int j = ORC_HIST_BINS - 1; j >= 0; --j) N[j] = N[j + 1] + h[j];
+  double n = 0.0, Sx = 0.0, Sy = 0.0, Sxx = 0.0, Sxy = 0.0;
+  for (int j = 16; j <= 4079; ++j) {
+    if (h[j] == 0) continue;
+    if (N[j] < 1 || N[j] > d / 2) continue;
+    double X = cvlc_log2_oracle((double)N[j]);
+    double Y = (double)((j >> 4) - 127) + cvlc_log2_oracle(1.0 + (double)(j & 15) / 16.0);
+    n = n + 1.0;
+    Sx = Sx + X;
+    Sy = Sy + Y;
+    Sxx = Sxx + X * X;
+    Sxy = Sxy + X * Y;
+  }
+  double den = n * Sxx - Sx * Sx;
+  double a;
+  if (n < 2.0 || !(den > 0.0))
+    a = -1.0;
+  else
+    a = (n * Sxy - Sx * Sy) / den;
+  double aq = floor(a * 256.0 + 0.5) / 256.0;
+  if (aq < -4.0) aq = -4.0;
+  if (aq > -1.0 / 256.0) aq = -1.0 / 256.0;
+  if (aq == -0.5) aq = -0.5 - 1.0 / 256.0; /* beta = 0 would make d^beta - 1 vanish */
+  *alpha = a;
+  *alpha_q = aq;
+}
+
+/* ======================================================================== */
+/* Packet constraint (Eq. (3)) and per-length coefficients (Eq. (5))         */
+/* ======================================================================== */
+
+static int params_ok(const orc_params* p) {
+  if (!p) return 0;
+  if (p->d < 2 || p->d > ((uint64_t)1 << 31)) return 0;
+  if (p->packet_bits == 0 || (p->packet_bits % 32) != 0) return 0;
+  if (p->header_bits < 80 || p->header_bits >= p->packet_bits) return 0;
+  if (p->quantizer != 0) return 0;
+  if (p->max_code_bits < 1 || p->max_code_bits > ORC_MAX_Y) return 0;
+  if (!(p->scale_B >= 1.0) || !(p->scale_B < 1e300)) return 0;
+  return 1;
+}
+
+/* s = ceil(log2 d) (Section IV-C); R = floor(budget / b); cap(y) = the most
+ * records P that satisfy P*(s+y) + H <= b. */
+int cvlc_derive_oracle(const orc_params* p, uint32_t* s_out, uint32_t* R_out, uint32_t cap[ORC_MAX_Y + 1]) {
+  if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
+  uint32_t s = 1;
+  while (((uint64_t)1 << s) < p->d) ++s;
+  uint64_t R = p->budget_bits / p->packet_bits;
+  if (R == 0) return ORC_ERR_BUDGET_TOO_SMALL;
+  if (R > 0xFFFFFFFFull) return ORC_ERR_BUDGET_TOO_LARGE;
+  for (uint32_t y = 0; y <= ORC_MAX_Y; ++y) cap[y] = 0;
+  for (uint32_t y = 1; y <= p->max_code_bits; ++y) cap[y] = (p->packet_bits - p->header_bits) / (s + y);
+  if (cap[p->max_code_bits] < 1) return ORC_ERR_PACKET_TOO_SMALL;
+  *s_out = s;
+  *R_out = (uint32_t)R;
+  return ORC_OK;
+}
+
+size_t cvlc_stream_bytes_oracle(const orc_params* p) {
+  uint64_t R = p->budget_bits / p->packet_bits;
+  return (size_t)(64 + R * (p->packet_bits / 8));
+}
+
+/* Quantization error factor of PQ with P = cap(y) values at y bits:
+ * Q = P / (2^y - 1)^2 (Appendix, case study). */
+static double Q_of(uint32_t cap_y, uint32_t y) {
+  double L = (double)(((uint64_t)1 << y) - 1);
+  return (double)cap_y / (L * L);
+}
+
+double cvlc_quant_error_Q_oracle(const orc_params* p, uint32_t y) {
+  uint32_t s, R, cap[ORC_MAX_Y + 1];
+  if (cvlc_derive_oracle(p, &s, &R, cap) != ORC_OK || y < 1 || y > p->max_code_bits) return NAN;
+  return Q_of(cap[y], y);
+}
+
+/* The bracket of Eq. (5) is c = Q/B^2 + 1/B_c^2 with 1/B_c = 1 - 1/B; g = 1 - c is
+ * what a packet gains over sparsifying its coordinates. */
+static double g_of(double Q, double B) {
+  double c = Q / (B * B) + (1.0 - 1.0 / B) * (1.0 - 1.0 / B);
+  return 1.0 - c;
+}
+
+double cvlc_coeff_g_oracle(const orc_params* p, uint32_t y) {
+  double Q = cvlc_quant_error_Q_oracle(p, y);
+  return g_of(Q, p->scale_B);
+}
+
+double cvlc_default_scale_oracle(const orc_params* p) {
+  orc_params q = *p;
+  q.scale_B = 1.0;
+  q.max_code_bits = ORC_MAX_Y;
+  uint32_t s, R, cap[ORC_MAX_Y + 1];
+  int rc = cvlc_derive_oracle(&q, &s, &R, cap);
+  if (rc != ORC_OK && rc != ORC_ERR_BUDGET_TOO_SMALL) return NAN;
+  if (rc == ORC_ERR_BUDGET_TOO_SMALL) {
+    s = 1;
+    while (((uint64_t)1 << s) < p->d) ++s;
+    cap[8] = (p->packet_bits - p->header_bits) / (s + 8);
+  }
+  return 1.0 + Q_of(cap[8], 8);
+}
+
+/* Planner context: candidate lengths and their coefficients */
+typedef struct {
+  uint64_t d;
+  uint32_t R;
+  int nY;
+  uint32_t Y[ORC_MAX_Y + 1];   /* ascending */
+  double g[ORC_MAX_Y + 1];     /* by length */
+  double Q[ORC_MAX_Y + 1];     /* by length */
+  uint32_t cap[ORC_MAX_Y + 1]; /* by length */
+  uint32_t y_min;
+  double beta, D;
+  uint64_t n_evals;
+} plan_ctx;
+
+static int ctx_init(plan_ctx* c, const orc_params* p, uint32_t* s_out) {
+  uint32_t s, R;
+  int rc = cvlc_derive_oracle(p, &s, &R, c->cap);
+  if (rc != ORC_OK) return rc;
+  *s_out = s;
+  c->d = p->d;
+  c->R = R;
+  c->n_evals = 0;
+  c->y_min = 0;
+  c->nY = 0;
+  for (uint32_t y = 1; y <= p->max_code_bits; ++y) {
+    c->Q[y] = Q_of(c->cap[y], y);
+    c->g[y] = g_of(c->Q[y], p->scale_B);
+    if (c->y_min == 0 && c->g[y] > 0.0) c->y_min = y;
+  }
+  if (c->y_min == 0) return ORC_ERR_SCALE_TOO_SMALL;
+  c->nY = 0;
+  for (uint32_t y = c->y_min; y <= p->max_code_bits; ++y) {
+    /* a length that fits no more records than the next longer one is dominated */
+    if (y == p->max_code_bits || c->cap[y] > c->cap[y + 1]) c->Y[c->nY++] = y;
+  }
+  return ORC_OK;
+}
+
+int cvlc_candidates_oracle(const orc_params* p, uint32_t Y[ORC_MAX_Y + 1]) {
+  plan_ctx c;
+  uint32_t s;
+  if (ctx_init(&c, p, &s) != ORC_OK) return 0;
+  for (int i = 0; i < c.nY; ++i) Y[i] = c.Y[i];
+  return c.nY;
+}
+
+static void ctx_set_beta(plan_ctx* c, double beta) {
+  c->beta = beta;
+  c->D = cvlc_powr_oracle((double)c->d, beta) - 1.0;
+}
+
+/* Share of ||U||^2 carried by the top Z ranks under Definition 1:
+ * sum_{l<=Z} l^(2 alpha) ~ ((Z+1)^beta - 1) / (d^beta - 1), the boundary the first
+ * term of Eq. (5) uses (d^beta - (k+1)^beta), applied to every packet boundary. */
+static double energy_E(const plan_ctx* c, uint64_t Z) {
+  return (cvlc_powr_oracle((double)(Z + 1), c->beta) - 1.0) / c->D;
+}
+
+/* F(n) = 1 - gamma, gamma of Eq. (5) with the packets grouped by code length as in
+ * Eq. (1): packets are laid out longest code first, so the group of length y covers
+ * ranks (W_prev, W]. */
+static double objective_F(plan_ctx* c, const uint32_t n[ORC_MAX_Y + 1]) {
+  uint64_t W = 0;
+  double Eprev = 0.0, F = 0.0;
+  c->n_evals += 1;
+  for (int i = c->nY - 1; i >= 0; --i) {
+    uint32_t y = c->Y[i];
+    if (n[y] == 0) continue;
+    W += (uint64_t)n[y] * (uint64_t)c->cap[y];
+    double Ecur = energy_E(c, W);
+    F = F + c->g[y] * (Ecur - Eprev);
+    Eprev = Ecur;
+  }
+  if (W > c->d) return -INFINITY;
+  return F;
+}
+
+double cvlc_objective_oracle(const orc_params* p, double beta, const uint32_t n_y[ORC_MAX_Y + 1]) {
+  plan_ctx c;
+  uint32_t s;
+  if (ctx_init(&c, p, &s) != ORC_OK) return NAN;
+  ctx_set_beta(&c, beta);
+  uint32_t n[ORC_MAX_Y + 1];
+  memset(n, 0, sizeof n);
+  for (int i = 0; i < c.nY; ++i) n[c.Y[i]] = n_y[c.Y[i]];
+  return objective_F(&c, n);
+}
+
+/* Atomic operation (Section IV-C): two lengths a > c share X = n_a + n_c packets;
+ * choose the split that maximises F (minimises gamma).  F is discretely concave in
+ * the split (Lemma 2), so the first t with F(t+1) <= F(t) is found by bisection. */
+static int atomic_op(plan_ctx* c, uint32_t n[ORC_MAX_Y + 1], uint32_t a, uint32_t cc) {
+  uint32_t X = n[a] + n[cc];
+  if (X == 0) return 0;
+  uint32_t na0 = n[a], nc0 = n[cc];
+  uint32_t lo = 0, hi = X;
+  while (lo < hi) {
+    uint32_t mid = lo + (hi - lo) / 2;
+    n[a] = mid + 1; n[cc] = X - (mid + 1);
+    double F1 = objective_F(c, n);
+    n[a] = mid; n[cc] = X - mid;
+    double F0 = objective_F(c, n);
+    if (F1 > F0) lo = mid + 1; else hi = mid;
+  }
+  int moved = 0;
+  if (lo != na0) {
+    n[a] = lo; n[cc] = X - lo;
+    double Fnew = objective_F(c, n);
+    n[a] = na0; n[cc] = nc0;
+    double Fold = objective_F(c, n);
+    if (Fnew > Fold) { n[a] = lo; n[cc] = X - lo; moved = 1; }
+  } else {
+    n[a] = na0; n[cc] = nc0;
+  }
+  return moved;
+}
+
+static void plan_fill(orc_plan* plan, plan_ctx* c, uint32_t s, const uint32_t n[ORC_MAX_Y + 1],
+                      double alpha, double alpha_q) {
+  memset(plan, 0, sizeof *plan);
+  plan->s = s;
+  plan->R = c->R;
+  plan->y_min = c->y_min;
+  plan->n_lengths = (uint32_t)c->nY;
+  plan->alpha = alpha;
+  plan->alpha_q = alpha_q;
+  plan->beta = c->beta;
+  uint64_t k = 0;
+  double Qmax = 0.0;
+  for (uint32_t y = 1; y <= ORC_MAX_Y; ++y) {
+    plan->cap[y] = c->cap[y];
+    plan->n_y[y] = n[y];
+    k += (uint64_t)n[y] * c->cap[y];
+    if (n[y] > 0 && c->Q[y] > Qmax) Qmax = c->Q[y];
+  }
+  plan->k = k;
+  double F = objective_F(c, n);
+  plan->gamma = 1.0 - F;
+  plan->B_next = 1.0 + Qmax;
+  plan->n_evals = c->n_evals;
+}
+
+/* Algorithm 1, steps 2-14, on integer code lengths: start from equal packets, then
+ * repeat atomic operations on pairs of lengths until no pair can be improved. */
+int cvlc_plan_from_alpha_oracle(const orc_params* p, double alpha_q, orc_plan* plan) {
+  plan_ctx c;
+  uint32_t s;
+  int rc = ctx_init(&c, p, &s);
+  if (rc != ORC_OK) return rc;
+  ctx_set_beta(&c, 2.0 * alpha_q + 1.0);
+
+  uint32_t n[ORC_MAX_Y + 1];
+  /* equal packets: the best admissible single-length plan, ties to the longer code */
+  int best = -1;
+  double bestF = -INFINITY;
+  for (int i = 0; i < c.nY; ++i) {
+    memset(n, 0, sizeof n);
+    n[c.Y[i]] = c.R;
+    double F = objective_F(&c, n);
+    if (F == -INFINITY) continue;
+    if (best < 0 || F >= bestF) { best = i; bestF = F; }
+  }
+  if (best < 0) return ORC_ERR_BUDGET_TOO_LARGE;
+  memset(n, 0, sizeof n);
+  n[c.Y[best]] = c.R;
+
+  for (int round = 0; round < 64; ++round) {
+    /* phase A: neighbouring lengths, until a sweep moves nothing */
+    for (int sweep = 0; sweep < 256; ++sweep) {
+      int moved = 0;
+      for (int i = c.nY - 1; i >= 1; --i) moved |= atomic_op(&c, n, c.Y[i], c.Y[i - 1]);
+      if (!moved) break;
+    }
+    /* phase B: every pair once */
+    int movedB = 0;
+    for (int i = c.nY - 1; i >= 1; --i)
+      for (int j = i - 1; j >= 0; --j) movedB |= atomic_op(&c, n, c.Y[i], c.Y[j]);
+    if (!movedB) break;
+  }
+  plan_fill(plan, &c, s, n, alpha_q, alpha_q);
+  return ORC_OK;
+}
+
+int cvlc_plan_oracle(const float* x, const orc_params* p, orc_plan* plan) {
+  if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
+  static uint64_t h[ORC_HIST_BINS];
+  int rc = cvlc_histogram_oracle(x, p->d, h);
+  if (rc != ORC_OK) return rc;
+  double alpha, alpha_q;
+  cvlc_alpha_fit_oracle(h, p->d, &alpha, &alpha_q);
+  rc = cvlc_plan_from_alpha_oracle(p, alpha_q, plan);
+  if (rc == ORC_OK) plan->alpha = alpha;
+  return rc;
+}
+
+/* Degenerate plan: every packet at one length y ("Top_k plus y-bit quantization",
+ * the baselines of Section V). */
+int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan) {
+  if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
+  if (y < 1 || y > p->max_code_bits) return ORC_ERR_INVALID_ARG;
+  plan_ctx c;
+  uint32_t s;
+  int rc = ctx_init(&c, p, &s);
+  if (rc != ORC_OK && rc != ORC_ERR_SCALE_TOO_SMALL) return rc;
+  if ((uint64_t)c.R * c.cap[y] > p->d) return ORC_ERR_BUDGET_TOO_LARGE;
+  /* evaluate gamma with the single length y as the only candidate */
+  c.nY = 1;
+  c.Y[0] = y;
+  c.Q[y] = Q_of(c.cap[y], y);
+  c.g[y] = g_of(c.Q[y], p->scale_B);
+  c.y_min = y;
+  ctx_set_beta(&c, 2.0 * (-1.0) + 1.0);
+  uint32_t n[ORC_MAX_Y + 1];
+  memset(n, 0, sizeof n);
+  n[y] = c.R;
+  plan_fill(plan, &c, s, n, -1.0, -1.0);
+  return ORC_OK;
+}
+
+/* ======================================================================== */
+/* Ranking ("ranked in a descending order of their absolute values")          */
+/* ======================================================================== */
+
+static int cmp_desc_u64(const void* a, const void* b) {
+  uint64_t x = *(const uint64_t*)a, y = *(const uint64_t*)b;
+  return (x < y) - (x > y);
+}
+
+/* Order: magnitude key descending, ties by ascending index.  The pair is packed
+ * as key * 2^32 + (2^32 - 1 - index) so one descending sort gives that order. */
+int cvlc_rank_oracle(const float* x, uint64_t d, uint64_t k, uint32_t* idx_out) {
+  if (k > d) return ORC_ERR_INVALID_ARG;
+  uint64_t* comp = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)d);
+  if (!comp) return ORC_ERR_INVALID_ARG;
+  for (uint64_t i = 0; i < d; ++i) comp[i] = ((uint64_t)key_of(x[i]) << 32) | (uint64_t)(0xFFFFFFFFu - (uint32_t)i);
+  qsort(comp, (size_t)d, sizeof(uint64_t), cmp_desc_u64);
+  for (uint64_t r = 0; r < k; ++r) idx_out[r] = 0xFFFFFFFFu - (uint32_t)(comp[r] & 0xFFFFFFFFu);
+  free(comp);
+  return ORC_OK;
+}
+
+/* ======================================================================== */
+/* PQ stochastic quantization (uniform centroids on [min,max], each value     */
+/* mapped to its upper or lower centroid, unbiased)                           */
+/* ======================================================================== */
+
+uint32_t cvlc_pq_quantize_oracle(float x, float lo, float hi, uint32_t y, uint32_t rnd) {
+  if (hi == lo) return 0;
+  double L = (double)(((uint64_t)1 << y) - 1);
+  double num = (double)x - (double)lo;
+  double den = (double)hi - (double)lo;
+  double t = (num / den) * L;
+  double j0 = floor(t);
+  if (j0 > L) j0 = L;
+  double frac = t - j0;
+  double u = (double)rnd * (1.0 / 4294967296.0);
+  uint32_t code = (uint32_t)j0;
+  if (u < frac) code += 1;
+  return code;
+}
+
+float cvlc_pq_dequantize_oracle(uint32_t code, float lo, float hi, uint32_t y) {
+  if (hi == lo) return lo;
+  double L = (double)(((uint64_t)1 << y) - 1);
+  double den = (double)hi - (double)lo;
+  return (float)((double)lo + (double)code * (den / L));
+}
+
+/* ======================================================================== */
+/* Bit stream (packet layout of Fig. 2: header with s, y_r and the centroid   */
+/* distribution, then (PID, CID) pairs)                                       */
+/* ======================================================================== */
+
+/* bit i of a packet is bit (i mod 32) of its (i / 32)-th little-endian 32-bit word */
+static void put_bits(uint8_t* pkt, uint64_t bitpos, uint64_t value, uint32_t width) {
+  for (uint32_t i = 0; i < width; ++i) {
+    uint64_t bp = bitpos + i;
+    if ((value >> i) & 1) pkt[bp >> 3] |= (uint8_t)(1u << (bp & 7));
+  }
+}
+static uint64_t get_bits(const uint8_t* pkt, uint64_t bitpos, uint32_t width) {
+  uint64_t v = 0;
+  for (uint32_t i = 0; i < width; ++i) {
+    uint64_t bp = bitpos + i;
+    if ((pkt[bp >> 3] >> (bp & 7)) & 1) v |= ((uint64_t)1 << i);
+  }
+  return v;
+}
+
+static void put_le(uint8_t* p, uint64_t v, int nbytes) {
+  for (int i = 0; i < nbytes; ++i) p[i] = (uint8_t)(v >> (8 * i));
+}
+static uint64_t get_le(const uint8_t* p, int nbytes) {
+  uint64_t v = 0;
+  for (int i = 0; i < nbytes; ++i) v |= (uint64_t)p[i] << (8 * i);
+  return v;
+}
+
+static float canon(float x) { return (key_of(x) == 0) ? 0.0f : x; }
+static uint32_t float_bits(float x) {
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  return u;
+}
+static float bits_float(uint32_t u) {
+  float x;
+  memcpy(&x, &u, 4);
+  return x;
+}
+
+/* Algorithm 1, steps 15-17: packet r takes the next P_r ranked coordinates and
+ * quantizes them with y_r bits; everything not sent is zero at the receiver. */
+int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan, uint8_t* stream,
+                       size_t capacity, uint32_t* ranked_idx_out) {
+  if (!params_ok(p) || !plan) return ORC_ERR_INVALID_ARG;
+  uint32_t s, R, cap[ORC_MAX_Y + 1];
+  int rc = cvlc_derive_oracle(p, &s, &R, cap);
+  if (rc != ORC_OK) return rc;
+  if (plan->R != R || plan->s != s) return ORC_ERR_INVALID_ARG;
+  size_t total = cvlc_stream_bytes_oracle(p);
+  if (capacity < total) return ORC_ERR_OUTPUT_TOO_SMALL;
+  uint64_t k = 0, nsum = 0;
+  for (uint32_t y = 1; y <= ORC_MAX_Y; ++y) {
+    if (plan->n_y[y] && cap[y] == 0) return ORC_ERR_INVALID_ARG;
+    k += (uint64_t)plan->n_y[y] * cap[y];
+    nsum += plan->n_y[y];
+  }
+  if (nsum != R || k != plan->k || k > p->d) return ORC_ERR_INVALID_ARG;
+  for (uint64_t i = 0; i < p->d; ++i)
+    if (key_of(x[i]) >= 0x7F800000u) return ORC_ERR_NONFINITE_INPUT;
+
+  uint32_t* rank = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)(k ? k : 1));
+  if (!rank) return ORC_ERR_INVALID_ARG;
+  rc = cvlc_rank_oracle(x, p->d, k, rank);
+  if (rc != ORC_OK) { free(rank); return rc; }
+  if (ranked_idx_out) memcpy(ranked_idx_out, rank, sizeof(uint32_t) * (size_t)k);
+
+  memset(stream, 0, total);
+  /* global header, 64 bytes, little-endian */
+  put_le(stream + 0, 0x434C5643u, 4);
+  put_le(stream + 4, 1, 2);
+  put_le(stream + 6, p->quantizer, 1);
+  put_le(stream + 7, s, 1);
+  put_le(stream + 8, p->d, 8);
+  put_le(stream + 16, R, 4);
+  put_le(stream + 20, p->packet_bits, 4);
+  put_le(stream + 24, p->header_bits, 4);
+  put_le(stream + 28, p->client_id, 4);
+  put_le(stream + 32, p->seed, 8);
+  put_le(stream + 40, p->round, 4);
+  put_le(stream + 44, 0, 4);
+  put_le(stream + 48, double_to_bits(p->scale_B), 8);
+  put_le(stream + 56, k, 8);
+
+  const uint32_t pkt_bytes = p->packet_bits / 8;
+  uint64_t Z = 0; /* ranks already packed */
+  uint32_t r = 0;
+  for (int y = ORC_MAX_Y; y >= 1; --y) {      /* longest codes first: P_1 <= ... <= P_R */
+    for (uint32_t q = 0; q < plan->n_y[y]; ++q, ++r) {
+      uint8_t* pkt = stream + 64 + (size_t)r * pkt_bytes;
+      uint32_t P = cap[y];
+      /* centroid distribution of PQ: minimum and maximum of the packet's values */
+      float lo = canon(x[rank[Z]]), hi = lo;
+      for (uint32_t j = 1; j < P; ++j) {
+        float v = canon(x[rank[Z + j]]);
+        if (v < lo) lo = v;
+        if (v > hi) hi = v;
+      }
+      put_bits(pkt, 0, s, 8);
+      put_bits(pkt, 8, (uint64_t)y, 8);
+      put_bits(pkt, 16, float_bits(lo), 32);
+      put_bits(pkt, 48, float_bits(hi), 32);
+      for (uint32_t j = 0; j < P; ++j) {
+        uint32_t pid = rank[Z + j];
+        uint32_t rnd = cvlc_philox_coord_oracle(p->seed, p->client_id, p->round, pid);
+        uint32_t code = cvlc_pq_quantize_oracle(canon(x[pid]), lo, hi, (uint32_t)y, rnd);
+        uint64_t bitpos = (uint64_t)p->header_bits + (uint64_t)j * (s + (uint32_t)y);
+        put_bits(pkt, bitpos, pid, s);
+        put_bits(pkt, bitpos + s, code, (uint32_t)y);
+      }
+      Z += P;
+    }
+  }
+  free(rank);
+  return ORC_OK;
+}
+
+/* ======================================================================== */
+/* Parameter-server side: w_{t+1} = w_t - (1/|S_t|) sum_i U_i (Section III,   */
+/* step 3), with U_i rebuilt from the packets and divided by B_i               */
+/* ======================================================================== */
+
+typedef struct {
+  uint32_t s, R, packet_bits, header_bits;
+  uint64_t d;
+  double B;
+} stream_head;
+
+static int parse_head(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_head* h) {
+  if (nbytes < 64) return ORC_ERR_BAD_STREAM;
+  if (get_le(st, 4) != 0x434C5643u) return ORC_ERR_BAD_STREAM;
+  if (get_le(st + 4, 2) != 1) return ORC_ERR_BAD_STREAM;
+  if (get_le(st + 6, 1) != 0) return ORC_ERR_BAD_STREAM;
+  h->s = (uint32_t)get_le(st + 7, 1);
+  h->d = get_le(st + 8, 8);
+  h->R = (uint32_t)get_le(st + 16, 4);
+  h->packet_bits = (uint32_t)get_le(st + 20, 4);
+  h->header_bits = (uint32_t)get_le(st + 24, 4);
+  h->B = bits_to_double(get_le(st + 48, 8));
+  if (h->d != d) return ORC_ERR_BAD_STREAM;
+  uint32_t s = 1;
+  while (((uint64_t)1 << s) < d) ++s;
+  if (h->s != s) return ORC_ERR_BAD_STREAM;
+  if (h->packet_bits == 0 || h->packet_bits % 32) return ORC_ERR_BAD_STREAM;
+  if (h->header_bits < 80 || h->header_bits >= h->packet_bits) return ORC_ERR_BAD_STREAM;
+  if (64 + (uint64_t)h->R * (h->packet_bits / 8) != nbytes) return ORC_ERR_BAD_STREAM;
+  if (!(h->B >= 1.0) || !(h->B < 1e300)) return ORC_ERR_BAD_STREAM;
+  return ORC_OK;
+}
+
+int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
+                                 const float* weights, uint32_t n_clients, double weight_total,
+                                 uint64_t d, float* out, int accumulate) {
+  if (d < 2 || d > ((uint64_t)1 << 31) || n_clients == 0) return ORC_ERR_INVALID_ARG;
+  double W = weight_total;
+  if (W == 0.0) {
+    for (uint32_t i = 0; i < n_clients; ++i) W = W + (double)weights[i];
+  }
+  if (!(W > 0.0)) return ORC_ERR_INVALID_ARG;
+  double* acc = (double*)calloc((size_t)d, sizeof(double));
+  if (!acc) return ORC_ERR_INVALID_ARG;
+  int rc = ORC_OK;
+  for (uint32_t i = 0; i < n_clients && rc == ORC_OK; ++i) {
+    stream_head h;
+    rc = parse_head(streams[i], stream_bytes[i], d, &h);
+    if (rc != ORC_OK) break;
+    float coef = (float)((double)weights[i] / (W * h.B));
+    uint32_t y_prev = ORC_MAX_Y;
+    for (uint32_t r = 0; r < h.R; ++r) {
+      const uint8_t* pkt = streams[i] + 64 + (size_t)r * (h.packet_bits / 8);
+      uint32_t s = (uint32_t)get_bits(pkt, 0, 8);
+      uint32_t y = (uint32_t)get_bits(pkt, 8, 8);
+      if (s != h.s || y < 1 || y > ORC_MAX_Y || y > y_prev) { rc = ORC_ERR_BAD_STREAM; break; }
+      y_prev = y;
+      float lo = bits_float((uint32_t)get_bits(pkt, 16, 32));
+      float hi = bits_float((uint32_t)get_bits(pkt, 48, 32));
+      uint32_t P = (h.packet_bits - h.header_bits) / (s + y);
+      for (uint32_t j = 0; j < P; ++j) {
+        uint64_t bitpos = (uint64_t)h.header_bits + (uint64_t)j * (s + y);
+        uint64_t pid = get_bits(pkt, bitpos, s);
+        uint32_t code = (uint32_t)get_bits(pkt, bitpos + s, y);
+        if (pid >= d) { rc = ORC_ERR_BAD_STREAM; break; }
+        float v = cvlc_pq_dequantize_oracle(code, lo, hi, y);
+        acc[pid] = acc[pid] + (double)coef * (double)v;
+      }
+      if (rc != ORC_OK) break;
+    }
+  }
+  if (rc == ORC_OK) {
+    for (uint64_t i = 0; i < d; ++i) {
+      if (accumulate)
+        out[i] = (float)((double)out[i] + acc[i]);
+      else
+        out[i] = (float)acc[i];
+    }
+  }
+  free(acc);
+  return rc;
+}

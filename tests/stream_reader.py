@@ -1,0 +1,90 @@
+"""An independent reader of the packet stream, written from the format definition
+(global header + fixed-size packets; packet = header {s, y_r, min, max} + (PID, CID)
+pairs, Fig. 2 of the paper), used by the tests to check both encoders.  It shares
+no code with the oracle or with the CUDA library."""
+from __future__ import annotations
+
+import struct
+from dataclasses import dataclass
+from typing import List
+
+import numpy as np
+
+
+@dataclass
+class Packet:
+    s: int
+    y: int
+    lo: float
+    hi: float
+    pid: np.ndarray   # uint64
+    cid: np.ndarray   # uint64
+    pad_bits_zero: bool
+
+
+@dataclass
+class Stream:
+    magic: int
+    version: int
+    quantizer: int
+    s: int
+    d: int
+    R: int
+    packet_bits: int
+    header_bits: int
+    client_id: int
+    seed: int
+    round: int
+    scale_B: float
+    k: int
+    packets: List[Packet]
+
+
+def _bits_of(packet: np.ndarray) -> np.ndarray:
+    """bit i of the packet = bit (i mod 8) of byte i // 8 (little-endian words)."""
+    return np.unpackbits(packet, bitorder="little")
+
+
+def _field(bits: np.ndarray, start: int, width: int) -> int:
+    v = 0
+    for i in range(width):
+        v |= int(bits[start + i]) << i
+    return v
+
+
+def parse(stream: np.ndarray) -> Stream:
+    raw = np.ascontiguousarray(stream, dtype=np.uint8).tobytes()
+    (magic, version, quantizer, s, d, R, packet_bits, header_bits, client_id, seed, rnd, zero, scale_B,
+     k) = struct.unpack_from("<IHBBQIIIIQIIdQ", raw, 0)
+    assert zero == 0
+    out = Stream(magic, version, quantizer, s, d, R, packet_bits, header_bits, client_id, seed, rnd,
+                 scale_B, k, [])
+    nbytes = packet_bits // 8
+    assert len(raw) == 64 + R * nbytes
+    for r in range(R):
+        pkt = np.frombuffer(raw, dtype=np.uint8, count=nbytes, offset=64 + r * nbytes)
+        bits = _bits_of(pkt)
+        ps = _field(bits, 0, 8)
+        y = _field(bits, 8, 8)
+        lo = struct.unpack("<f", struct.pack("<I", _field(bits, 16, 32)))[0]
+        hi = struct.unpack("<f", struct.pack("<I", _field(bits, 48, 32)))[0]
+        hdr_zero = not bits[80:header_bits].any()
+        w = ps + y
+        P = (packet_bits - header_bits) // w
+        body = bits[header_bits:header_bits + P * w].reshape(P, w).astype(np.uint64)
+        wp = (np.uint64(1) << np.arange(ps, dtype=np.uint64))
+        wc = (np.uint64(1) << np.arange(y, dtype=np.uint64))
+        pid = (body[:, :ps] * wp).sum(axis=1, dtype=np.uint64)
+        cid = (body[:, ps:] * wc).sum(axis=1, dtype=np.uint64)
+        pad_zero = hdr_zero and not bits[header_bits + P * w:].any()
+        out.packets.append(Packet(ps, y, lo, hi, pid, cid, pad_zero))
+    return out
+
+
+def dequantize(pk: Packet) -> np.ndarray:
+    """centroid value of each record: uniform grid of 2^y points on [lo, hi]."""
+    if pk.hi == pk.lo:
+        return np.full(pk.cid.shape, np.float32(pk.lo), dtype=np.float32)
+    L = float(2 ** pk.y - 1)
+    step = (np.float64(pk.hi) - np.float64(pk.lo)) / L
+    return (np.float64(pk.lo) + pk.cid.astype(np.float64) * step).astype(np.float32)

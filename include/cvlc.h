@@ -1,0 +1,191 @@
+/*
+ * libcvlc: Fed-CVLC per-round compression on one NVIDIA B200 (sm_100a).
+ *
+ * A client compresses its fp32 model update U (d coordinates) into R fixed-size
+ * packets: the k largest |U| are ranked, split into packets, packet r carries P_r
+ * (position ID, centroid ID) pairs at y_r bits per value, and the code lengths y_r
+ * are tuned to minimise the error bound gamma under the packet and budget
+ * constraints (paper: Section IV-B "three operations", Eq. (3), Proposition 2 /
+ * Eq. (5), Algorithm 1, packet format of Fig. 2).  The parameter server decodes
+ * the packets of many clients and forms their weighted average (Section III,
+ * step 3).
+ *
+ * Conventions
+ *  - Every function returns a status (0 = CVLC_OK); nothing throws, prints or aborts.
+ *  - Pointers named *_dev are DEVICE pointers owned by the caller; cvlc_params is
+ *    read from HOST memory at call time.  The library allocates no device memory,
+ *    keeps no state between calls and only enqueues kernels on `cuda_stream`
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *  - Host-detectable errors are returned at once.  Errors only the device can see
+ *    (non-finite input, malformed stream, a wait that ran out) are written to the
+ *    status word at byte 0 of the plan / workspace and read with cvlc_read_status;
+ *    after such an error the outputs are unspecified, but no access is out of
+ *    bounds and no kernel waits without limit.
+ *  - Workspaces: 256-byte aligned, sized by the *_workspace_bytes calls, private to
+ *    one call in flight (two calls that overlap on the GPU need two workspaces).
+ *  - There is no CPU fallback: without a CUDA device every launch call returns
+ *    CVLC_ERR_CUDA.
+ */
+#ifndef CVLC_H
+#define CVLC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  CVLC_OK = 0,
+  CVLC_ERR_INVALID_ARG = 1,
+  CVLC_ERR_BUDGET_TOO_SMALL = 2,    /* budget below one packet */
+  CVLC_ERR_BUDGET_TOO_LARGE = 3,    /* even the longest code would send more than d coordinates */
+  CVLC_ERR_PACKET_TOO_SMALL = 4,    /* a packet cannot hold one record of the longest code */
+  CVLC_ERR_NONFINITE_INPUT = 5,     /* Inf or NaN in the update (device-detected) */
+  CVLC_ERR_WORKSPACE_TOO_SMALL = 6,
+  CVLC_ERR_OUTPUT_TOO_SMALL = 7,
+  CVLC_ERR_BAD_STREAM = 8,          /* malformed stream (device-detected) */
+  CVLC_ERR_DEVICE_TIMEOUT = 9,      /* a bounded device-side wait ran out */
+  CVLC_ERR_CUDA = 10,
+  CVLC_ERR_NOT_IMPLEMENTED = 11,
+  CVLC_ERR_SCALE_TOO_SMALL = 12,    /* scale_B violates B > (Q+1)/2 for every code length */
+  CVLC_ERR_PLAN_MISMATCH = 13       /* plan does not belong to these params / this update */
+};
+
+#define CVLC_MAX_CODE_BITS 32
+#define CVLC_HIST_BINS 4096
+#define CVLC_STREAM_HEADER_BYTES 64
+#define CVLC_STREAM_MAGIC 0x434C5643u
+#define CVLC_MAX_CLIENTS_PER_CALL 4096
+
+/* Problem statement of Section IV-C: the update has d coordinates, the client may
+ * send budget_bits this round in packets of packet_bits (b) with header_bits (H)
+ * of header each; lengths are chosen from 1..max_code_bits (Section IV-B, "Y kinds
+ * of codes"), coordinates outside the top k get 0 bits. */
+typedef struct cvlc_params {
+  uint64_t d;             /* coordinates, 2 <= d <= 2^31 */
+  uint64_t budget_bits;   /* uplink budget of this client this round; R = floor(budget_bits / packet_bits) */
+  uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes) */
+  uint32_t header_bits;   /* H; 80 <= H < b; 80 = s (8) + y_r (8) + min,max (64), Fig. 2 */
+  uint32_t quantizer;     /* 0 = PQ (uniform centroids on [min,max]) */
+  uint32_t max_code_bits; /* 1..32 */
+  double scale_B;         /* B >= 1 of the scaling operation; cvlc_default_scale() in the first round */
+  uint64_t seed;          /* Philox4x32-10 key */
+  uint32_t client_id;     /* Philox counter word 2 */
+  uint32_t round;         /* Philox counter word 3 */
+} cvlc_params;
+
+/* Device-resident plan, 512 bytes, written by cvlc_plan / cvlc_plan_fixed. */
+typedef struct cvlc_plan_t {
+  int32_t status;         /* byte 0: device status word */
+  uint32_t s;             /* bits per position ID, ceil(log2 d) */
+  uint32_t R;             /* packets */
+  uint32_t y_min;         /* shortest length with a positive coefficient in Eq. (5) */
+  uint32_t n_lengths;     /* number of candidate lengths */
+  uint32_t thresh_bin;    /* histogram bin that holds rank k */
+  uint64_t k;             /* transmitted coordinates, sum of n_y * cap */
+  uint64_t n_candidates;  /* coordinates in bins >= thresh_bin (>= k) */
+  double alpha;           /* fitted decay exponent of Definition 1 */
+  double alpha_q;         /* alpha rounded to 1/256 and clamped */
+  double beta;            /* 2 * alpha_q + 1 */
+  double gamma;           /* Eq. (5) at the chosen lengths */
+  double B_next;          /* 1 + max Q over the used lengths: scale_B for the next round */
+  uint32_t n_y[CVLC_MAX_CODE_BITS + 1]; /* packets per code length; packets are laid out longest code first */
+  uint32_t cap[CVLC_MAX_CODE_BITS + 1]; /* records per packet per code length: floor((b - H) / (s + y)) */
+  uint8_t reserved[512 - 80 - 2 * 4 * (CVLC_MAX_CODE_BITS + 1)];
+} cvlc_plan_t;
+
+/* --- host-only helpers (no GPU work) --------------------------------------- */
+
+int cvlc_version(void);
+const char* cvlc_status_string(int status);
+/* Selects the CUDA device the following calls launch on (one process drives one GPU). */
+int cvlc_set_device(int device);
+
+/* 64 + floor(budget_bits / b) * b / 8: global header plus R whole packets (the
+ * budget bR of Section IV-C is met exactly in whole packets).  0 on invalid params. */
+size_t cvlc_stream_bytes(const cvlc_params* p);
+/* 1 + Q(cap(8), 8): the scale of a first round (Proposition 1, footnote: B is taken
+ * from the previous round's max Q + 1).  NaN on invalid params. */
+double cvlc_default_scale(const cvlc_params* p);
+size_t cvlc_plan_workspace_bytes(const cvlc_params* p);
+size_t cvlc_encode_workspace_bytes(const cvlc_params* p);
+size_t cvlc_decode_workspace_bytes(uint32_t n_clients);
+
+/* --- the hot path ----------------------------------------------------------- */
+
+/*
+ * Algorithm 1, steps 1-14.  Reads the update x_dev (d fp32, 16-byte aligned),
+ * builds the 4096-bin magnitude histogram, fits the power-law exponent of
+ * Definition 1 and tunes the per-packet code lengths by repeated atomic
+ * operations (Section IV-C, Lemma 2, Theorem 1) on integer lengths, minimising
+ * gamma of Eq. (5) under Eq. (3).  Writes *plan_dev.  After the call the 4096
+ * uint64 histogram counts sit at byte 256 of the workspace.
+ * Errors: INVALID_ARG, BUDGET_*, PACKET_TOO_SMALL, SCALE_TOO_SMALL,
+ * WORKSPACE_TOO_SMALL (host); NONFINITE_INPUT (device, in plan_dev->status).
+ */
+int cvlc_plan(const float* x_dev, const cvlc_params* p, cvlc_plan_t* plan_dev, void* ws_dev,
+              size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Degenerate plan with every packet at code length y: Top_k sparsification plus
+ * y-bit quantization, the baselines of Section V that the method contains as
+ * special cases (Section I).  Same arguments and errors as cvlc_plan.
+ */
+int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_plan_t* plan_dev,
+                    void* ws_dev, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 1, steps 15-17.  Ranks the coordinates of x_dev by |x| (ties by
+ * ascending index), gives packet r the next cap(y_r) ranks, stores the packet's
+ * minimum and maximum, quantizes each value stochastically onto the 2^y_r uniform
+ * centroids (unbiased; random word = Philox4x32-10 of the coordinate index) and
+ * packs (position ID, centroid ID) pairs behind the packet header (Fig. 2).
+ * stream_dev (16-byte aligned) receives cvlc_stream_bytes(p) bytes.
+ * plan_dev must come from cvlc_plan / cvlc_plan_fixed on the same x_dev and params.
+ * Errors: INVALID_ARG, OUTPUT_TOO_SMALL, WORKSPACE_TOO_SMALL (host); PLAN_MISMATCH,
+ * DEVICE_TIMEOUT (device, at byte 0 of ws_dev).
+ */
+int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev,
+                uint8_t* stream_dev, size_t stream_capacity, void* ws_dev, size_t ws_bytes,
+                void* cuda_stream);
+
+/*
+ * Parameter-server aggregation (Section III, step 3) fused with decoding: for every
+ * record of every client, value = min + CID * (max - min) / (2^y - 1), scaled by
+ * 1/B_i (Section IV-B, scaling) and by weight_i / weight_total, added into
+ * out_dev[PID].  Uniform weights give the paper's 1/|S_t| average.
+ *  streams_dev       device array of n_clients device pointers (each 16-byte aligned)
+ *  stream_bytes_dev  device array of n_clients stream lengths
+ *  weights_dev       device array of n_clients fp32 weights (> 0)
+ *  weight_total      0 = sum of this call's weights; otherwise the total over all
+ *                    batches when the clients are fed in several calls
+ *  out_dev           d fp32; overwritten when accumulate == 0, added to when 1
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL (host); BAD_STREAM (device, at byte 0
+ * of ws_dev).
+ */
+int cvlc_decode_aggregate(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev,
+                          const float* weights_dev, uint32_t n_clients, double weight_total,
+                          uint64_t d, float* out_dev, int accumulate, void* ws_dev, size_t ws_bytes,
+                          void* cuda_stream);
+
+/* Waits for cuda_stream and returns the status word at byte 0 of a plan or workspace. */
+int cvlc_read_status(const void* plan_or_ws_dev, void* cuda_stream);
+
+/* --- diagnostic entry points (used by the parity tests) --------------------- */
+
+/* out_dev[4*i .. 4*i+3] = Philox4x32-10(counter (i_lo, i_hi, client_id, round), key seed)
+ * for i = first .. first + n - 1 (Salmon et al., SC'11). */
+int cvlc_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t first,
+                         uint64_t n, uint32_t* out_dev, void* cuda_stream);
+/* The planner's series arithmetic: log2_out[i] = log2(in[i]) (in > 0), exp2_out[i] =
+ * 2^in[i] (|in| <= 1000), div_out[i*20 + j-1] = in[i] / j for j = 1..20 (the constant
+ * divisions of the exp2 series), div_ref the same by IEEE division. */
+int cvlc_selftest_math(const double* in_dev, uint64_t n, double* log2_out_dev, double* exp2_out_dev,
+                       double* div_out_dev, double* div_ref_dev, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -218,19 +218,17 @@ double cvlc_coeff_g_oracle(const orc_params* p, uint32_t y) {
   return g_of(Q, p->scale_B);
 }
 
+/* Scale of a first round: 1 + Q of an 8-bit packet (the paper takes B from the previous
+ * round's max Q + 1; there is no previous round yet). */
 double cvlc_default_scale_oracle(const orc_params* p) {
   orc_params q = *p;
   q.scale_B = 1.0;
   q.max_code_bits = ORC_MAX_Y;
-  uint32_t s, R, cap[ORC_MAX_Y + 1];
-  int rc = cvlc_derive_oracle(&q, &s, &R, cap);
-  if (rc != ORC_OK && rc != ORC_ERR_BUDGET_TOO_SMALL) return NAN;
-  if (rc == ORC_ERR_BUDGET_TOO_SMALL) {
-    s = 1;
-    while (((uint64_t)1 << s) < p->d) ++s;
-    cap[8] = (p->packet_bits - p->header_bits) / (s + 8);
-  }
-  return 1.0 + Q_of(cap[8], 8);
+  if (!params_ok(&q)) return NAN;
+  uint32_t s = 1;
+  while (((uint64_t)1 << s) < p->d) ++s;
+  uint32_t cap8 = (p->packet_bits - p->header_bits) / (s + 8);
+  return 1.0 + Q_of(cap8, 8);
 }
 
 /* Planner context: candidate lengths and their coefficients */

@@ -1,0 +1,304 @@
+"""Thin ctypes binding of libcvlc (same names as include/cvlc.h).
+
+Argument marshalling only: every step of the compression path runs in the CUDA
+kernels of libcvlc.so.  torch provides device memory and the stream handle.
+There is no CPU fallback: if the library is missing, importing the entry points
+raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcvlc.so")
+
+CVLC_OK = 0
+CVLC_ERR_INVALID_ARG = 1
+CVLC_ERR_BUDGET_TOO_SMALL = 2
+CVLC_ERR_BUDGET_TOO_LARGE = 3
+CVLC_ERR_PACKET_TOO_SMALL = 4
+CVLC_ERR_NONFINITE_INPUT = 5
+CVLC_ERR_WORKSPACE_TOO_SMALL = 6
+CVLC_ERR_OUTPUT_TOO_SMALL = 7
+CVLC_ERR_BAD_STREAM = 8
+CVLC_ERR_DEVICE_TIMEOUT = 9
+CVLC_ERR_CUDA = 10
+CVLC_ERR_NOT_IMPLEMENTED = 11
+CVLC_ERR_SCALE_TOO_SMALL = 12
+CVLC_ERR_PLAN_MISMATCH = 13
+
+MAX_CODE_BITS = 32
+HIST_BINS = 4096
+PLAN_BYTES = 512
+PLAN_WS_HIST_OFFSET = 256
+
+EXPORTS = [
+    "cvlc_version", "cvlc_status_string", "cvlc_set_device", "cvlc_stream_bytes", "cvlc_default_scale",
+    "cvlc_plan_workspace_bytes", "cvlc_encode_workspace_bytes", "cvlc_decode_workspace_bytes",
+    "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_decode_aggregate", "cvlc_read_status",
+    "cvlc_selftest_philox", "cvlc_selftest_math",
+]
+
+
+class CvlcParams(C.Structure):
+    _fields_ = [
+        ("d", C.c_uint64), ("budget_bits", C.c_uint64),
+        ("packet_bits", C.c_uint32), ("header_bits", C.c_uint32),
+        ("quantizer", C.c_uint32), ("max_code_bits", C.c_uint32),
+        ("scale_B", C.c_double), ("seed", C.c_uint64),
+        ("client_id", C.c_uint32), ("round", C.c_uint32),
+    ]
+
+
+class CvlcPlan(C.Structure):
+    _fields_ = [
+        ("status", C.c_int32), ("s", C.c_uint32), ("R", C.c_uint32), ("y_min", C.c_uint32),
+        ("n_lengths", C.c_uint32), ("thresh_bin", C.c_uint32),
+        ("k", C.c_uint64), ("n_candidates", C.c_uint64),
+        ("alpha", C.c_double), ("alpha_q", C.c_double), ("beta", C.c_double),
+        ("gamma", C.c_double), ("B_next", C.c_double),
+        ("n_y", C.c_uint32 * (MAX_CODE_BITS + 1)), ("cap", C.c_uint32 * (MAX_CODE_BITS + 1)),
+        ("reserved", C.c_uint8 * (512 - 80 - 2 * 4 * (MAX_CODE_BITS + 1))),
+    ]
+
+
+assert C.sizeof(CvlcPlan) == PLAN_BYTES
+
+
+class CvlcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: status {code} ({status_string(code)})")
+        self.code = code
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Loads libcvlc.so; raises if it has not been built (there is nothing to fall back to)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2402_03770_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, u32, u64, f64, sz = C.c_void_p, C.c_uint32, C.c_uint64, C.c_double, C.c_size_t
+    PP = C.POINTER(CvlcParams)
+    L.cvlc_version.restype = C.c_int
+    L.cvlc_version.argtypes = []
+    L.cvlc_status_string.restype = C.c_char_p
+    L.cvlc_status_string.argtypes = [C.c_int]
+    L.cvlc_set_device.restype = C.c_int
+    L.cvlc_set_device.argtypes = [C.c_int]
+    L.cvlc_stream_bytes.restype = sz
+    L.cvlc_stream_bytes.argtypes = [PP]
+    L.cvlc_default_scale.restype = f64
+    L.cvlc_default_scale.argtypes = [PP]
+    L.cvlc_plan_workspace_bytes.restype = sz
+    L.cvlc_plan_workspace_bytes.argtypes = [PP]
+    L.cvlc_encode_workspace_bytes.restype = sz
+    L.cvlc_encode_workspace_bytes.argtypes = [PP]
+    L.cvlc_decode_workspace_bytes.restype = sz
+    L.cvlc_decode_workspace_bytes.argtypes = [u32]
+    L.cvlc_plan.restype = C.c_int
+    L.cvlc_plan.argtypes = [vp, PP, vp, vp, sz, vp]
+    L.cvlc_plan_fixed.restype = C.c_int
+    L.cvlc_plan_fixed.argtypes = [vp, PP, u32, vp, vp, sz, vp]
+    L.cvlc_encode.restype = C.c_int
+    L.cvlc_encode.argtypes = [vp, PP, vp, vp, sz, vp, sz, vp]
+    L.cvlc_decode_aggregate.restype = C.c_int
+    L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
+    L.cvlc_read_status.restype = C.c_int
+    L.cvlc_read_status.argtypes = [vp, vp]
+    L.cvlc_selftest_philox.restype = C.c_int
+    L.cvlc_selftest_philox.argtypes = [u64, u32, u32, u64, u64, vp, vp]
+    L.cvlc_selftest_math.restype = C.c_int
+    L.cvlc_selftest_math.argtypes = [vp, u64, vp, vp, vp, vp, vp]
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().cvlc_status_string(int(code)).decode()
+
+
+def make_params(d: int, budget_bits: int, *, packet_bits: int = 12000, header_bits: int = 80,
+                quantizer: int = 0, max_code_bits: int = 32, scale_B: Optional[float] = None,
+                seed: int = 0, client_id: int = 0, round: int = 0) -> CvlcParams:
+    p = CvlcParams(d, budget_bits, packet_bits, header_bits, quantizer, max_code_bits, 1.0, seed,
+                   client_id, round)
+    p.scale_B = cvlc_default_scale(p) if scale_B is None else float(scale_B)
+    return p
+
+
+def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
+    st = torch.cuda.current_stream() if stream is None else stream
+    return int(st.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous()
+    return t.data_ptr()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != CVLC_OK:
+        raise CvlcError(rc, where)
+
+
+# ---- host-only helpers -------------------------------------------------------------
+
+def cvlc_set_device(device: int) -> None:
+    _check(lib().cvlc_set_device(int(device)), "cvlc_set_device")
+
+
+def cvlc_stream_bytes(p: CvlcParams) -> int:
+    return int(lib().cvlc_stream_bytes(C.byref(p)))
+
+
+def cvlc_default_scale(p: CvlcParams) -> float:
+    return float(lib().cvlc_default_scale(C.byref(p)))
+
+
+def cvlc_plan_workspace_bytes(p: CvlcParams) -> int:
+    return int(lib().cvlc_plan_workspace_bytes(C.byref(p)))
+
+
+def cvlc_encode_workspace_bytes(p: CvlcParams) -> int:
+    return int(lib().cvlc_encode_workspace_bytes(C.byref(p)))
+
+
+def cvlc_decode_workspace_bytes(n_clients: int) -> int:
+    return int(lib().cvlc_decode_workspace_bytes(int(n_clients)))
+
+
+# ---- the hot path (device tensors in, kernels enqueued on the stream) ----------------
+
+def cvlc_plan(x: torch.Tensor, p: CvlcParams, plan: torch.Tensor, ws: torch.Tensor,
+              stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert x.dtype == torch.float32 and x.numel() == p.d
+    assert plan.dtype == torch.uint8 and plan.numel() >= PLAN_BYTES
+    _check(lib().cvlc_plan(_ptr(x), C.byref(p), _ptr(plan), _ptr(ws), ws.numel() * ws.element_size(),
+                           _stream_handle(stream)), "cvlc_plan")
+
+
+def cvlc_plan_fixed(x: torch.Tensor, p: CvlcParams, y: int, plan: torch.Tensor, ws: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert x.dtype == torch.float32 and x.numel() == p.d
+    _check(lib().cvlc_plan_fixed(_ptr(x), C.byref(p), int(y), _ptr(plan), _ptr(ws),
+                                 ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_plan_fixed")
+
+
+def cvlc_encode(x: torch.Tensor, p: CvlcParams, plan: torch.Tensor, out_stream: torch.Tensor,
+                ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert x.dtype == torch.float32 and x.numel() == p.d
+    assert out_stream.dtype == torch.uint8
+    _check(lib().cvlc_encode(_ptr(x), C.byref(p), _ptr(plan), _ptr(out_stream), out_stream.numel(),
+                             _ptr(ws), ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode")
+
+
+def cvlc_decode_aggregate(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor,
+                          n_clients: int, weight_total: float, d: int, out: torch.Tensor, accumulate: bool,
+                          ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert stream_ptrs.dtype in (torch.int64, torch.uint64) and stream_ptrs.numel() >= n_clients
+    assert stream_bytes.dtype in (torch.int64, torch.uint64) and stream_bytes.numel() >= n_clients
+    assert weights.dtype == torch.float32 and out.dtype == torch.float32 and out.numel() == d
+    _check(lib().cvlc_decode_aggregate(_ptr(stream_ptrs), _ptr(stream_bytes), _ptr(weights), int(n_clients),
+                                       float(weight_total), int(d), _ptr(out), 1 if accumulate else 0,
+                                       _ptr(ws), ws.numel() * ws.element_size(), _stream_handle(stream)),
+           "cvlc_decode_aggregate")
+
+
+def cvlc_read_status(plan_or_ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    return int(lib().cvlc_read_status(_ptr(plan_or_ws), _stream_handle(stream)))
+
+
+def cvlc_selftest_philox(seed: int, client_id: int, round: int, first: int, n: int, out: torch.Tensor,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert out.dtype in (torch.int32, torch.uint32) and out.numel() >= 4 * n
+    _check(lib().cvlc_selftest_philox(seed, client_id, round, first, n, _ptr(out), _stream_handle(stream)),
+           "cvlc_selftest_philox")
+
+
+def cvlc_selftest_math(inp: torch.Tensor, log2_out: Optional[torch.Tensor], exp2_out: Optional[torch.Tensor],
+                       div_out: Optional[torch.Tensor], div_ref: Optional[torch.Tensor],
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert inp.dtype == torch.float64
+    _check(lib().cvlc_selftest_math(_ptr(inp), inp.numel(), _ptr(log2_out), _ptr(exp2_out), _ptr(div_out),
+                                    _ptr(div_ref), _stream_handle(stream)), "cvlc_selftest_math")
+
+
+# ---- buffer helpers (allocation only) ---------------------------------------------------
+
+def alloc_bytes(n: int, device: torch.device) -> torch.Tensor:
+    """Device byte buffer; torch's caching allocator returns 512-byte aligned blocks."""
+    return torch.empty(max(int(n), 1), dtype=torch.uint8, device=device)
+
+
+def read_plan(plan: torch.Tensor) -> CvlcPlan:
+    """Copies a device plan to the host (synchronises the current stream)."""
+    raw = bytes(plan[:PLAN_BYTES].cpu().numpy().tobytes())
+    return CvlcPlan.from_buffer_copy(raw)
+
+
+class ClientEncoder:
+    """Owns the buffers one client's plan + encode needs; all work is enqueued on `stream`."""
+
+    def __init__(self, p: CvlcParams, device: torch.device):
+        self.p = p
+        self.device = device
+        self.plan = alloc_bytes(PLAN_BYTES, device)
+        self.plan_ws = alloc_bytes(cvlc_plan_workspace_bytes(p), device)
+        self.enc_ws = alloc_bytes(cvlc_encode_workspace_bytes(p), device)
+        self.out = alloc_bytes(cvlc_stream_bytes(p), device)
+
+    def run(self, x: torch.Tensor, p: Optional[CvlcParams] = None, out: Optional[torch.Tensor] = None,
+            stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0) -> torch.Tensor:
+        p = self.p if p is None else p
+        out = self.out if out is None else out
+        if fixed_y:
+            cvlc_plan_fixed(x, p, fixed_y, self.plan, self.plan_ws, stream)
+        else:
+            cvlc_plan(x, p, self.plan, self.plan_ws, stream)
+        cvlc_encode(x, p, self.plan, out, self.enc_ws, stream)
+        return out
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        rc = cvlc_read_status(self.plan, stream)
+        return rc if rc != CVLC_OK else cvlc_read_status(self.enc_ws, stream)
+
+
+class Aggregator:
+    """Owns the pointer tables and workspace of cvlc_decode_aggregate for up to n_max clients."""
+
+    def __init__(self, n_max: int, d: int, device: torch.device):
+        self.n_max, self.d, self.device = n_max, d, device
+        self.ptrs = torch.zeros(n_max, dtype=torch.int64, device=device)
+        self.sizes = torch.zeros(n_max, dtype=torch.int64, device=device)
+        self.weights = torch.zeros(n_max, dtype=torch.float32, device=device)
+        self.ws = alloc_bytes(cvlc_decode_workspace_bytes(n_max), device)
+        self._keep: List[torch.Tensor] = []
+
+    def set_clients(self, streams: Sequence[torch.Tensor], weights: torch.Tensor) -> int:
+        n = len(streams)
+        assert n <= self.n_max
+        self._keep = list(streams)
+        self.ptrs[:n] = torch.tensor([s.data_ptr() for s in streams], dtype=torch.int64)
+        self.sizes[:n] = torch.tensor([s.numel() for s in streams], dtype=torch.int64)
+        self.weights[:n] = weights.to(self.device, dtype=torch.float32)
+        return n
+
+    def run(self, n: int, out: torch.Tensor, *, weight_total: float = 0.0, accumulate: bool = False,
+            stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        cvlc_decode_aggregate(self.ptrs, self.sizes, self.weights, n, weight_total, self.d, out, accumulate,
+                              self.ws, stream)
+        return out
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return cvlc_read_status(self.ws, stream)

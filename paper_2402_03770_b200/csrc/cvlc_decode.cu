@@ -1,0 +1,197 @@
+// Parameter-server side (Section III, step 3): decode every client's packets
+// (Fig. 2), dequantize, scale by weight_i / (W * B_i) and accumulate into the dense
+// averaged update.  One warp per packet; scatter-accumulate with fp32 reductions.
+#include "cvlc_common.cuh"
+
+namespace cvlc {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kPrepThreads = 1024;
+constexpr int kDecodeThreads = 256;
+
+struct StreamHead {
+  uint32_t magic, ver_q_s, d_lo, d_hi, R, packet_bits, header_bits, client_id, seed_lo, seed_hi, round, zero, B_lo, B_hi, k_lo, k_hi;
+};
+
+// K7a  validate the global headers, derive per-client coefficients and the packet prefix
+__global__ void __launch_bounds__(kPrepThreads)
+k_decode_prepare(const uint8_t* const* __restrict__ streams, const uint64_t* __restrict__ stream_bytes,
+                 const float* __restrict__ weights, uint32_t n, double weight_total, uint64_t d, uint32_t s,
+                 unsigned char* ws) {
+  __shared__ double s_part[kPrepThreads / 32];
+  __shared__ uint32_t s_cnt[kPrepThreads / 32];
+  __shared__ double s_W;
+  __shared__ uint32_t s_carry;
+  int32_t* status = reinterpret_cast<int32_t*>(ws + kDecWsStatus);
+  uint32_t* total_pkts = reinterpret_cast<uint32_t*>(ws + kDecWsTotalPkts);
+  float* coef = reinterpret_cast<float*>(ws + kDecWsCoef);
+  uint32_t* prefix = reinterpret_cast<uint32_t*>(ws + dec_off_prefix(n));
+  uint32_t* meta = reinterpret_cast<uint32_t*>(ws + dec_off_meta(n));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    *status = 0;
+    s_carry = 0;
+  }
+  // total weight
+  double wsum = 0.0;
+  for (uint32_t i = tid; i < n; i += kPrepThreads) wsum += (double)weights[i];
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) wsum += __shfl_xor_sync(kFull, wsum, off);
+  if (lane == 0) s_part[warp] = wsum;
+  __syncthreads();
+  if (tid == 0) {
+    double W = 0.0;
+    for (int w = 0; w < kPrepThreads / 32; ++w) W += s_part[w];
+    s_W = (weight_total != 0.0) ? weight_total : W;
+  }
+  __syncthreads();
+  const double W = s_W;
+  if (tid == 0 && !(W > 0.0)) set_status(status, CVLC_ERR_INVALID_ARG);
+
+  // headers, in chunks of kPrepThreads clients; prefix of packet counts in client order
+  for (uint32_t base = 0; base < n; base += kPrepThreads) {
+    const uint32_t i = base + tid;
+    uint32_t R = 0;
+    if (i < n) {
+      const uint8_t* st = streams[i];
+      const uint64_t nbytes = stream_bytes[i];
+      bool ok = (st != nullptr) && ((reinterpret_cast<uintptr_t>(st) & 15) == 0) && nbytes >= CVLC_STREAM_HEADER_BYTES;
+      if (ok) {
+        const uint4* hv = reinterpret_cast<const uint4*>(st);
+        const uint4 h0 = __ldg(hv), h1 = __ldg(hv + 1), h3 = __ldg(hv + 3);
+        const uint32_t magic = h0.x, ver_q_s = h0.y;
+        const uint64_t sd = (uint64_t)h0.z | ((uint64_t)h0.w << 32);
+        const uint32_t sR = h1.x, pb = h1.y, hb = h1.z;
+        const double B = __longlong_as_double((long long)((uint64_t)h3.x | ((uint64_t)h3.y << 32)));
+        ok = (magic == CVLC_STREAM_MAGIC) && ((ver_q_s & 0xFFFF) == 1) && (((ver_q_s >> 16) & 0xFF) == 0) &&
+             ((ver_q_s >> 24) == s) && (sd == d) && (pb != 0) && ((pb & 31) == 0) && (hb >= 80) && (hb < pb) &&
+             (B >= 1.0) && (B < 1e300);
+        if (ok) ok = ((uint64_t)CVLC_STREAM_HEADER_BYTES + (uint64_t)sR * (pb / 8) == nbytes);
+        if (ok) {
+          R = sR;
+          coef[i] = (float)((double)weights[i] / (W * B));
+          meta[2 * i] = pb;
+          meta[2 * i + 1] = hb;
+        }
+      }
+      if (!ok) {
+        set_status(status, CVLC_ERR_BAD_STREAM);
+        coef[i] = 0.0f;
+        meta[2 * i] = 32;
+        meta[2 * i + 1] = 0;
+      }
+    }
+    uint32_t incl = R;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t o = __shfl_up_sync(kFull, incl, off);
+      if (lane >= off) incl += o;
+    }
+    if (lane == 31) s_cnt[warp] = incl;
+    __syncthreads();
+    uint32_t below = s_carry;
+    for (int w = 0; w < warp; ++w) below += s_cnt[w];
+    if (i < n) prefix[i] = below + incl - R;
+    __syncthreads();
+    if (tid == kPrepThreads - 1) s_carry = below + incl;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    prefix[n] = s_carry;
+    *total_pkts = s_carry;
+  }
+}
+
+// K7b  out = 0 (when not accumulating): 4 bytes written per coordinate
+__global__ void __launch_bounds__(256)
+k_fill_zero(float* __restrict__ out, uint64_t d) {
+  const uint64_t nvec = d >> 2;
+  float4* ov = reinterpret_cast<float4*>(out);
+  const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (uint64_t v = (uint64_t)blockIdx.x * 256 + threadIdx.x; v < nvec; v += (uint64_t)gridDim.x * 256) ov[v] = z;
+  if (blockIdx.x == 0 && threadIdx.x < (d & 3)) out[(nvec << 2) + threadIdx.x] = 0.f;
+}
+
+// K6  decode + dequantize + weighted scatter-accumulate, one warp per packet
+__global__ void __launch_bounds__(kDecodeThreads)
+k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uint32_t s, float* __restrict__ out,
+         unsigned char* ws) {
+  extern __shared__ uint32_t s_prefix[];  // [n + 1]
+  int32_t* status = reinterpret_cast<int32_t*>(ws + kDecWsStatus);
+  const float* coef = reinterpret_cast<const float*>(ws + kDecWsCoef);
+  const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + dec_off_prefix(n));
+  const uint32_t* meta = reinterpret_cast<const uint32_t*>(ws + dec_off_meta(n));
+  if (*status != 0) return;
+  for (uint32_t i = threadIdx.x; i <= n; i += kDecodeThreads) s_prefix[i] = prefix[i];
+  __syncthreads();
+  const uint32_t total = s_prefix[n];
+  const int lane = threadIdx.x & 31;
+  const uint32_t warps_total = gridDim.x * (kDecodeThreads / 32);
+  const unsigned long long pid_mask = (1ull << s) - 1ull;
+
+  for (uint32_t g = blockIdx.x * (kDecodeThreads / 32) + (threadIdx.x >> 5); g < total; g += warps_total) {
+    // client of packet g: last c with prefix[c] <= g
+    uint32_t lo_c = 0, hi_c = n;
+    while (hi_c - lo_c > 1) {
+      const uint32_t mid = (lo_c + hi_c) >> 1;
+      if (s_prefix[mid] <= g) lo_c = mid; else hi_c = mid;
+    }
+    const uint32_t c = lo_c, r = g - s_prefix[c];
+    const uint32_t pb = meta[2 * c], H = meta[2 * c + 1];
+    const uint32_t n_words = pb >> 5;
+    const uint32_t* pkt = reinterpret_cast<const uint32_t*>(streams[c] + CVLC_STREAM_HEADER_BYTES) + (size_t)r * n_words;
+    const uint32_t w0 = __ldg(pkt), w1 = __ldg(pkt + 1), w2 = __ldg(pkt + 2);
+    const uint32_t ps = w0 & 0xFF, y = (w0 >> 8) & 0xFF;
+    uint32_t y_prev = CVLC_MAX_CODE_BITS;
+    if (r > 0) y_prev = (__ldg(pkt - n_words) >> 8) & 0xFF;
+    if (ps != s || y < 1 || y > CVLC_MAX_CODE_BITS || y > y_prev) {  // lengths never increase along a stream
+      if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
+      continue;
+    }
+    const float lo = __uint_as_float((w0 >> 16) | (w1 << 16));
+    const float hi = __uint_as_float((w1 >> 16) | (w2 << 16));
+    const uint32_t wd = s + y;
+    const uint32_t P = (pb - H) / wd;
+    const double dlo = (double)lo;
+    const double step = (hi == lo) ? 0.0 : __ddiv_rn(__dsub_rn((double)hi, dlo), (double)((1ull << y) - 1ull));
+    const float cf = coef[c];
+    const unsigned long long code_mask = (1ull << y) - 1ull;
+    for (uint32_t j = lane; j < P; j += 32) {
+      const uint32_t bit = H + j * wd;
+      const uint32_t wi = bit >> 5, sh = bit & 31;
+      // a record of up to 63 bits starting at bit sh of word wi spans at most three words
+      const unsigned long long a = __ldg(pkt + wi);
+      const unsigned long long b = (wi + 1 < n_words) ? __ldg(pkt + wi + 1) : 0u;
+      unsigned long long rec = (a | (b << 32)) >> sh;
+      if (sh + wd > 64) {
+        const unsigned long long c2 = (wi + 2 < n_words) ? __ldg(pkt + wi + 2) : 0u;
+        rec |= c2 << (64 - sh);
+      }
+      const unsigned long long pid = rec & pid_mask;
+      const uint32_t code = (uint32_t)((rec >> s) & code_mask);
+      if (pid >= d) {
+        set_status(status, CVLC_ERR_BAD_STREAM);
+        continue;
+      }
+      const float v = (float)__dadd_rn(dlo, __dmul_rn((double)code, step));
+      atomicAdd(out + pid, cf * v);
+    }
+  }
+}
+
+cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
+                          uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
+                          void* ws, cudaStream_t st) {
+  unsigned char* w = static_cast<unsigned char*>(ws);
+  k_decode_prepare<<<1, kPrepThreads, 0, st>>>(streams, stream_bytes, weights, n, weight_total, d, s, w);
+  if (!accumulate) {
+    const uint64_t nvec = d >> 2;
+    uint64_t want = (nvec + 255) / 256;
+    const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? (want ? want : 1) : 8 * kNumSM);
+    k_fill_zero<<<grid, 256, 0, st>>>(out, d);
+  }
+  k_decode<<<8 * kNumSM, kDecodeThreads, ((size_t)n + 1) * 4, st>>>(streams, n, d, s, out, w);
+  return cudaGetLastError();
+}
+
+}  // namespace cvlc

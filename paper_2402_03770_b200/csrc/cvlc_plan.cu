@@ -1,0 +1,516 @@
+// Planning kernels: magnitude histogram (Algorithm 1, step 1) and the single-CTA
+// planner (power-law exponent of Definition 1, code-length tuning by atomic
+// operations on Eq. (5), Algorithm 1 steps 2-14).
+//
+// The planner's floating point is IEEE binary64 with every multiply and add
+// rounded separately (the *_rn intrinsics keep the compiler from contracting
+// them), in a fixed order, so that its decisions do not depend on the machine.
+#include "cvlc_common.cuh"
+
+namespace cvlc {
+
+// ===================================================================================
+// K1  magnitude histogram: h[key >> 19], key = bits(|x|); HBM-bound, 4 bytes / coordinate
+// ===================================================================================
+
+constexpr int kHistThreads = 512;
+constexpr int kHistSub = 4;  // shared sub-histograms per block (64 KB)
+
+__global__ void __launch_bounds__(kHistThreads, 2)
+k_hist(const float* __restrict__ x, uint64_t d, unsigned long long* __restrict__ hist, uint32_t* __restrict__ nonfinite) {
+  extern __shared__ uint32_t sh_hist[];  // [kHistSub][4096]
+  for (int i = threadIdx.x; i < kHistSub * CVLC_HIST_BINS; i += kHistThreads) sh_hist[i] = 0;
+  __syncthreads();
+  uint32_t* my = sh_hist + ((threadIdx.x >> 5) & (kHistSub - 1)) * CVLC_HIST_BINS;
+
+  const uint64_t nvec = d >> 2;
+  const float4* xv = reinterpret_cast<const float4*>(x);
+  const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
+  uint32_t bad = 0;
+  uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x;
+  // four independent 128-bit loads in flight per thread
+  for (; v + 3 * stride < nvec; v += 4 * stride) {
+    float4 a[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * stride);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t k0 = __float_as_uint(a[u].x) & 0x7FFFFFFFu, k1 = __float_as_uint(a[u].y) & 0x7FFFFFFFu;
+      const uint32_t k2 = __float_as_uint(a[u].z) & 0x7FFFFFFFu, k3 = __float_as_uint(a[u].w) & 0x7FFFFFFFu;
+      bad |= (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
+      atomicAdd(my + (k0 >> 19), 1u);
+      atomicAdd(my + (k1 >> 19), 1u);
+      atomicAdd(my + (k2 >> 19), 1u);
+      atomicAdd(my + (k3 >> 19), 1u);
+    }
+  }
+  for (; v < nvec; v += stride) {
+    const float4 a = __ldg(xv + v);
+    const uint32_t k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
+    const uint32_t k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
+    bad |= (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
+    atomicAdd(my + (k0 >> 19), 1u);
+    atomicAdd(my + (k1 >> 19), 1u);
+    atomicAdd(my + (k2 >> 19), 1u);
+    atomicAdd(my + (k3 >> 19), 1u);
+  }
+  // ragged tail (d not a multiple of 4)
+  if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
+    const uint32_t k0 = __float_as_uint(x[(nvec << 2) + threadIdx.x]) & 0x7FFFFFFFu;
+    bad |= (k0 >= 0x7F800000u);
+    atomicAdd(my + (k0 >> 19), 1u);
+  }
+  if (bad) atomicOr(nonfinite, 1u);
+  __syncthreads();
+  for (int b = threadIdx.x; b < CVLC_HIST_BINS; b += kHistThreads) {
+    uint32_t c = 0;
+#pragma unroll
+    for (int s = 0; s < kHistSub; ++s) c += sh_hist[s * CVLC_HIST_BINS + b];
+    if (c) atomicAdd(hist + b, (unsigned long long)c);
+  }
+}
+
+__global__ void k_zero_words(uint32_t* p, size_t n_words) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += (size_t)gridDim.x * blockDim.x) p[i] = 0;
+}
+
+// ===================================================================================
+// Series arithmetic of the planner
+// ===================================================================================
+
+// log2 of a positive normal double: v = m 2^e, m folded into (sqrt(1/2), sqrt(2)],
+// ln m = 2 atanh(t) with t = (m-1)/(m+1), odd series up to t^25.
+__device__ __forceinline__ double series_log2(double v) {
+  const unsigned long long bits = (unsigned long long)__double_as_longlong(v);
+  int e = (int)((bits >> 52) & 0x7FF) - 1023;
+  double m = __longlong_as_double((long long)((bits & 0x000FFFFFFFFFFFFFull) | 0x3FF0000000000000ull));
+  if (m > 1.4142135623730951) {
+    m = __dmul_rn(m, 0.5);
+    e += 1;
+  }
+  const double t = __ddiv_rn(__dsub_rn(m, 1.0), __dadd_rn(m, 1.0));
+  const double q = __dmul_rn(t, t);
+  double p = 1.0 / 25.0;
+#pragma unroll
+  for (int j = 11; j >= 0; --j) p = __dadd_rn(__dmul_rn(p, q), 1.0 / (double)(2 * j + 1));
+  const double ln_m = __dmul_rn(__dmul_rn(2.0, t), p);
+  return __dadd_rn((double)e, __dmul_rn(ln_m, 1.4426950408889634));
+}
+
+// u / j for a small positive integer j, correctly rounded, from the rounded reciprocal:
+// q0 = RN(u * rcp), r = u - j*q0 (exact in one fused operation: it is a small multiple
+// of ulp(q0)), q1 = RN(q0 + r*rcp).  q0 + r*rcp differs from u/j by less than 2^-52 ulp,
+// while u/j, a quotient by an integer below 2^5, is either representable or at least
+// 1/(2j) ulp away from every rounding boundary, so q1 = RN(u/j).
+__device__ __forceinline__ double div_small_int(double u, int j) {
+  const double rcp = 1.0 / (double)j;  // folded at compile time when j is constant
+  const double q0 = __dmul_rn(u, rcp);
+  const double r = __fma_rn(-(double)j, q0, u);
+  return __fma_rn(r, rcp, q0);
+}
+
+// 2^v for |v| <= 1000: v = n + r with |r| <= 1/2, e^(r ln 2) as the degree-20 Taylor
+// polynomial in Horner form p = 1 + (u/j) p, then n added to the exponent field.
+__device__ __forceinline__ double series_exp2(double v) {
+  const double n = floor(__dadd_rn(v, 0.5));
+  const double r = __dsub_rn(v, n);
+  const double u = __dmul_rn(r, 0.6931471805599453);
+  double p = 1.0;
+#pragma unroll
+  for (int j = 20; j >= 1; --j) p = __dadd_rn(1.0, __dmul_rn(div_small_int(u, j), p));
+  const long long ni = (long long)n;
+  return __longlong_as_double(__double_as_longlong(p) + ni * (1ll << 52));
+}
+
+__device__ __forceinline__ double series_powr(double a, double beta) { return series_exp2(__dmul_rn(beta, series_log2(a))); }
+
+// share of ||U||^2 in the top Z ranks under Definition 1: ((Z+1)^beta - 1) / (d^beta - 1)
+__device__ __forceinline__ double energy_E(uint64_t Z, double beta, double D) {
+  return __ddiv_rn(__dsub_rn(series_powr((double)(Z + 1), beta), 1.0), D);
+}
+
+// ===================================================================================
+// K2  planner: one CTA of 1024 threads
+// ===================================================================================
+
+constexpr int kPlanThreads = 1024;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+// F(n) = 1 - gamma of Eq. (5), packets grouped by length, longest first.  One warp:
+// lane l holds candidate length l (count my_n, capacity my_cap, coefficient my_g).
+__device__ __forceinline__ double eval_F_warp(uint32_t my_n, uint32_t my_cap, double my_g, int lane, double beta,
+                                              double D, uint64_t d) {
+  uint64_t W = (uint64_t)my_n * my_cap;  // -> ranks covered down to and including this length
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint64_t o = __shfl_down_sync(kFull, W, off);
+    if (lane + off < 32) W += o;
+  }
+  const unsigned act = __ballot_sync(kFull, my_n > 0);
+  double E = 0.0;
+  if (my_n > 0) E = energy_E(W, beta, D);
+  const unsigned higher = (lane == 31) ? 0u : (act & ~((2u << lane) - 1u));
+  const int src = higher ? (__ffs(higher) - 1) : lane;
+  double Eprev = __shfl_sync(kFull, E, src);
+  if (!higher) Eprev = 0.0;
+  const double term = __dmul_rn(my_g, __dsub_rn(E, Eprev));
+  double F = 0.0;
+  unsigned m = act;
+  while (m) {
+    const int l = 31 - __clz(m);
+    m &= ~(1u << l);
+    F = __dadd_rn(F, __shfl_sync(kFull, term, l));
+  }
+  const uint64_t Wtot = __shfl_sync(kFull, W, 0);
+  if (Wtot > d) F = -CUDART_INF;
+  return F;
+}
+
+struct PlanShared {
+  double Fv[32];
+  uint32_t n[32];
+  double beta, D, alpha, alpha_q;
+  unsigned long long warp_tot[32];
+  unsigned long long carry;
+  uint32_t warp_cnt[32];
+  uint32_t n_points;
+};
+
+__global__ void __launch_bounds__(kPlanThreads, 1)
+k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__ nonfinite,
+       const __grid_constant__ PlanTables T, cvlc_plan_t* __restrict__ plan) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned long long* Nsuf = reinterpret_cast<unsigned long long*>(smem_raw);  // [4096] survival counts
+  double* ptX = reinterpret_cast<double*>(smem_raw + 4096 * 8);                // fit points, ascending bin
+  double* ptY = ptX + 4096;
+  __shared__ PlanShared S;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- survival counts N_j = #{bin >= j} ------------------------------------------
+  unsigned long long h[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = hist[4 * tid + i];
+  {
+    unsigned long long tot = h[0] + h[1] + h[2] + h[3];
+    // inclusive scan from the top bin down: reverse thread order
+    unsigned long long v = tot;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned long long o = __shfl_down_sync(kFull, v, off);
+      if (lane + off < 32) v += o;
+    }
+    if (lane == 0) S.warp_tot[warp] = v;
+    __syncthreads();
+    unsigned long long above = 0;
+    for (int w = warp + 1; w < 32; ++w) above += S.warp_tot[w];
+    const unsigned long long incl = v + above;  // sum over threads >= tid
+    unsigned long long run = incl - tot;        // sum over threads > tid
+#pragma unroll
+    for (int i = 3; i >= 0; --i) {
+      run += h[i];
+      Nsuf[4 * tid + i] = run;
+    }
+  }
+  __syncthreads();
+
+  if (T.fixed_y == 0) {
+    // ---- fit points: non-empty normal bins in the upper half of the ranks ----------
+    uint32_t flags = 0, cnt = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = 4 * tid + i;
+      const unsigned long long N = Nsuf[j];
+      const bool ok = (j >= 16) && (j <= 4079) && (h[i] > 0) && (N >= 1) && (N <= T.d / 2);
+      flags |= (ok ? 1u : 0u) << i;
+      cnt += ok;
+    }
+    uint32_t v = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t o = __shfl_up_sync(kFull, v, off);
+      if (lane >= off) v += o;
+    }
+    if (lane == 31) S.warp_cnt[warp] = v;
+    __syncthreads();
+    uint32_t below = 0;
+    for (int w = 0; w < warp; ++w) below += S.warp_cnt[w];
+    uint32_t pos = below + v - cnt;
+    if (tid == kPlanThreads - 1) S.n_points = below + v;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (flags & (1u << i)) {
+        const int j = 4 * tid + i;
+        ptX[pos] = series_log2((double)Nsuf[j]);
+        ptY[pos] = __dadd_rn((double)((j >> 4) - 127), series_log2(__dadd_rn(1.0, (double)(j & 15) / 16.0)));
+        ++pos;
+      }
+    }
+    __syncthreads();
+    // ---- least squares of log2|U{l}| on log2 l, sums in ascending bin order ----------
+    if (tid == 0) {
+      double n = 0.0, Sx = 0.0, Sy = 0.0, Sxx = 0.0, Sxy = 0.0;
+      const uint32_t np = S.n_points;
+      for (uint32_t i = 0; i < np; ++i) {
+        const double X = ptX[i], Y = ptY[i];
+        n = __dadd_rn(n, 1.0);
+        Sx = __dadd_rn(Sx, X);
+        Sy = __dadd_rn(Sy, Y);
+        Sxx = __dadd_rn(Sxx, __dmul_rn(X, X));
+        Sxy = __dadd_rn(Sxy, __dmul_rn(X, Y));
+      }
+      const double den = __dsub_rn(__dmul_rn(n, Sxx), __dmul_rn(Sx, Sx));
+      double a;
+      if (n < 2.0 || !(den > 0.0))
+        a = -1.0;
+      else
+        a = __ddiv_rn(__dsub_rn(__dmul_rn(n, Sxy), __dmul_rn(Sx, Sy)), den);
+      double aq = __dmul_rn(floor(__dadd_rn(__dmul_rn(a, 256.0), 0.5)), 1.0 / 256.0);
+      if (aq < -4.0) aq = -4.0;
+      if (aq > -1.0 / 256.0) aq = -1.0 / 256.0;
+      if (aq == -0.5) aq = -0.5 - 1.0 / 256.0;  // beta = 0 would make d^beta - 1 vanish
+      S.alpha = a;
+      S.alpha_q = aq;
+    }
+  } else if (tid == 0) {
+    S.alpha = -1.0;
+    S.alpha_q = -1.0;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const double beta = __dadd_rn(__dmul_rn(2.0, S.alpha_q), 1.0);
+    S.beta = beta;
+    S.D = __dsub_rn(series_powr((double)T.d, beta), 1.0);
+  }
+  if (tid < 32) S.n[tid] = 0;
+  __syncthreads();
+  const double beta = S.beta, D = S.D;
+  const int nY = (int)T.nY;
+  const uint32_t my_cap = (lane < nY) ? T.capY[lane] : 0u;
+  const double my_g = (lane < nY) ? T.gY[lane] : 0.0;
+
+  if (T.fixed_y != 0) {
+    if (tid == 0) S.n[0] = T.R;
+    __syncthreads();
+  } else {
+    // ---- equal packets: best admissible single-length plan, ties to the longer code ----
+    if (warp < nY) {
+      const double F = eval_F_warp(lane == warp ? T.R : 0u, my_cap, my_g, lane, beta, D, T.d);
+      if (lane == 0) S.Fv[warp] = F;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int best = -1;
+      double bestF = -CUDART_INF;
+      for (int i = 0; i < nY; ++i) {
+        const double F = S.Fv[i];
+        if (F == -CUDART_INF) continue;
+        if (best < 0 || F >= bestF) {
+          best = i;
+          bestF = F;
+        }
+      }
+      S.n[best < 0 ? 0 : best] = T.R;  // the host has checked that a plan is admissible
+    }
+    __syncthreads();
+
+    // ---- atomic operations (Section IV-C) on pairs of lengths until nothing moves ----
+    // An atomic operation bisects the split of X = n_a + n_c packets between the lengths
+    // a > c for the first t with F(t+1) <= F(t).  Four bisection levels are evaluated at
+    // once: warps 2q, 2q+1 evaluate F(mid+1), F(mid) of node q+1 of the decision tree,
+    // warp 30 evaluates the current split; then every thread walks the tree.
+    for (int round = 0; round < 64; ++round) {
+      int movedB = 0;
+      for (int phase = 0; phase < 2; ++phase) {  // 0: neighbouring lengths until quiet; 1: every pair once
+        const int max_sweeps = (phase == 0) ? 256 : 1;
+        for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+          int moved = 0;
+          for (int i = nY - 1; i >= 1; --i) {
+            const int j_hi = i - 1, j_lo = (phase == 0) ? i - 1 : 0;
+            for (int j = j_hi; j >= j_lo; --j) {
+              const uint32_t na0 = S.n[i], nc0 = S.n[j];
+              const uint32_t X = na0 + nc0;
+              if (X == 0) continue;
+              uint32_t lo = 0, hi = X;
+              double F_final = 0.0, F_cur = 0.0;
+              bool first = true;
+              while (lo < hi) {
+                // which evaluation does this warp own?
+                bool valid = false;
+                uint32_t t = 0;
+                if (warp < 30) {
+                  // node (warp/2 + 1) of the decision tree in heap order: child 2h after
+                  // "F(mid+1) <= F(mid)", child 2h+1 after "F(mid+1) > F(mid)"
+                  const int hnode = (warp >> 1) + 1;
+                  const int depth = 31 - __clz(hnode);
+                  uint32_t l3 = lo, h3 = hi;
+                  bool open = true;
+                  for (int b = depth - 1; b >= 0; --b) {
+                    if (!(l3 < h3)) { open = false; break; }
+                    const uint32_t mid = l3 + (h3 - l3) / 2;
+                    if ((hnode >> b) & 1) l3 = mid + 1; else h3 = mid;
+                  }
+                  if (open && l3 < h3) {
+                    const uint32_t mid = l3 + (h3 - l3) / 2;
+                    t = mid + ((warp & 1) ? 0u : 1u);
+                    valid = true;
+                  }
+                } else if (warp == 30 && first) {
+                  t = na0;
+                  valid = true;
+                }
+                if (valid) {
+                  uint32_t my_n = (lane < nY) ? S.n[lane] : 0u;
+                  if (lane == i) my_n = t;
+                  if (lane == j) my_n = X - t;
+                  const double F = eval_F_warp(my_n, my_cap, my_g, lane, beta, D, T.d);
+                  if (lane == 0) S.Fv[warp] = F;
+                }
+                __syncthreads();
+                if (first) F_cur = S.Fv[30];
+                first = false;
+                int hnode = 1;
+                for (int level = 0; level < 4 && lo < hi; ++level) {
+                  const uint32_t mid = lo + (hi - lo) / 2;
+                  const double F1 = S.Fv[2 * (hnode - 1)], F0 = S.Fv[2 * (hnode - 1) + 1];
+                  if (F1 > F0) {
+                    lo = mid + 1;
+                    F_final = F1;
+                    hnode = 2 * hnode + 1;
+                  } else {
+                    hi = mid;
+                    F_final = F0;
+                    hnode = 2 * hnode;
+                  }
+                }
+                __syncthreads();
+              }
+              if (lo != na0 && F_final > F_cur) {
+                if (tid == 0) {
+                  S.n[i] = lo;
+                  S.n[j] = X - lo;
+                }
+                moved = 1;
+              }
+              __syncthreads();
+            }
+          }
+          if (phase == 1) movedB = moved;
+          if (!moved) break;
+        }
+      }
+      if (!movedB) break;
+    }
+  }
+
+  // ---- outputs ---------------------------------------------------------------------
+  if (warp == 0) {
+    const uint32_t my_n = (lane < nY) ? S.n[lane] : 0u;
+    const double F = eval_F_warp(my_n, my_cap, my_g, lane, beta, D, T.d);
+    if (lane == 0) S.Fv[0] = F;
+  }
+  __syncthreads();
+  unsigned long long k = 0;
+  for (int i = 0; i < nY; ++i) k += (unsigned long long)S.n[i] * T.capY[i];
+  if (tid == 0) {
+    double Qmax = 0.0;
+    for (int i = 0; i < nY; ++i)
+      if (S.n[i] > 0 && T.QY[i] > Qmax) Qmax = T.QY[i];
+    plan->status = (*nonfinite) ? CVLC_ERR_NONFINITE_INPUT : CVLC_OK;
+    plan->s = T.s;
+    plan->R = T.R;
+    plan->y_min = T.y_min;
+    plan->n_lengths = T.nY;
+    plan->k = k;
+    plan->alpha = S.alpha;
+    plan->alpha_q = S.alpha_q;
+    plan->beta = beta;
+    plan->gamma = __dsub_rn(1.0, S.Fv[0]);
+    plan->B_next = __dadd_rn(1.0, Qmax);
+    for (int y = 0; y <= CVLC_MAX_CODE_BITS; ++y) {
+      plan->n_y[y] = 0;
+      plan->cap[y] = T.cap[y];
+    }
+    for (int i = 0; i < nY; ++i) plan->n_y[T.Y[i]] = S.n[i];
+  }
+  // threshold bin: the bin that holds rank k (1-based), and how many coordinates sit in it or above
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int j = 4 * tid + i;
+    const unsigned long long N = Nsuf[j];
+    const unsigned long long Nn = (j == CVLC_HIST_BINS - 1) ? 0ull : Nsuf[j + 1];
+    if (N >= k && Nn < k) {
+      plan->thresh_bin = (uint32_t)j;
+      plan->n_candidates = N;
+    }
+  }
+}
+
+// ===================================================================================
+// launchers
+// ===================================================================================
+
+cudaError_t launch_plan(const float* x, const PlanTables& T, cvlc_plan_t* plan, void* ws, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(k_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  unsigned char* w = static_cast<unsigned char*>(ws);
+  unsigned long long* hist = reinterpret_cast<unsigned long long*>(w + kPlanWsHist);
+  uint32_t* flag = reinterpret_cast<uint32_t*>(w + kPlanWsStatus + 4);
+  k_zero_words<<<8, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsBytes / 4);
+  const uint64_t nvec = T.d >> 2;
+  uint64_t want = (nvec + kHistThreads - 1) / kHistThreads;
+  int grid = (int)(want < (uint64_t)(2 * kNumSM) ? (want ? want : 1) : 2 * kNumSM);
+  k_hist<<<grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(x, T.d, hist, flag);
+  k_plan<<<1, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flag, T, plan);
+  return cudaGetLastError();
+}
+
+// ---- diagnostics ---------------------------------------------------------------------
+
+__global__ void k_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t first, uint64_t n, uint32_t* out) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t c = first + i;
+    const uint4 r = philox4x32_10(make_uint4((uint32_t)c, (uint32_t)(c >> 32), client_id, round),
+                                  make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
+    out[4 * i + 0] = r.x;
+    out[4 * i + 1] = r.y;
+    out[4 * i + 2] = r.z;
+    out[4 * i + 3] = r.w;
+  }
+}
+
+__global__ void k_selftest_math(const double* in, uint64_t n, double* l2, double* e2, double* dv, double* dr) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const double v = in[i];
+    if (l2) l2[i] = (v > 0.0) ? series_log2(v) : 0.0;
+    if (e2) e2[i] = (fabs(v) <= 1000.0) ? series_exp2(v) : 0.0;
+    if (dv && dr) {
+      for (int j = 1; j <= 20; ++j) {
+        dv[i * 20 + j - 1] = div_small_int(v, j);
+        dr[i * 20 + j - 1] = __ddiv_rn(v, (double)j);
+      }
+    }
+  }
+}
+
+cudaError_t launch_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t first, uint64_t n,
+                                   uint32_t* out, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  k_selftest_philox<<<kNumSM, 256, 0, st>>>(seed, client_id, round, first, n, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_selftest_math(const double* in, uint64_t n, double* l2, double* e2, double* dv, double* dr,
+                                 cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  k_selftest_math<<<kNumSM, 256, 0, st>>>(in, n, l2, e2, dv, dr);
+  return cudaGetLastError();
+}
+
+}  // namespace cvlc

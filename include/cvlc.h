@@ -185,6 +185,17 @@ int cvlc_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint
 int cvlc_selftest_math(const double* in_dev, uint64_t n, double* log2_out_dev, double* exp2_out_dev,
                        double* div_out_dev, double* div_ref_dev, void* cuda_stream);
 
+/* Launch accounting: number of kernels this library has launched in this process
+ * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist"). */
+unsigned long long cvlc_launch_count(const char* kernel_name);
+/* Optional timing of one kernel: after cvlc_profile_select(name, n) the next n launches of
+ * that kernel are bracketed by a CUDA event pair on their own stream; cvlc_profile_read
+ * synchronises the device and returns how many were timed and their summed duration.
+ * cvlc_profile_select(NULL, 0) switches it off and frees the events.  Single-threaded use. */
+int cvlc_profile_select(const char* kernel_name, uint32_t max_launches);
+int cvlc_profile_reset(void);
+int cvlc_profile_read(uint32_t* launches, double* total_ms);
+
 #ifdef __cplusplus
 }
 #endif

@@ -41,6 +41,7 @@ EXPORTS = [
     "cvlc_plan_workspace_bytes", "cvlc_encode_workspace_bytes", "cvlc_decode_workspace_bytes",
     "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math",
+    "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -118,6 +119,14 @@ def lib() -> C.CDLL:
     L.cvlc_selftest_philox.argtypes = [u64, u32, u32, u64, u64, vp, vp]
     L.cvlc_selftest_math.restype = C.c_int
     L.cvlc_selftest_math.argtypes = [vp, u64, vp, vp, vp, vp, vp]
+    L.cvlc_launch_count.restype = C.c_ulonglong
+    L.cvlc_launch_count.argtypes = [C.c_char_p]
+    L.cvlc_profile_select.restype = C.c_int
+    L.cvlc_profile_select.argtypes = [C.c_char_p, u32]
+    L.cvlc_profile_reset.restype = C.c_int
+    L.cvlc_profile_reset.argtypes = []
+    L.cvlc_profile_read.restype = C.c_int
+    L.cvlc_profile_read.argtypes = [C.POINTER(u32), C.POINTER(f64)]
     _lib = L
     return L
 
@@ -232,6 +241,24 @@ def cvlc_selftest_math(inp: torch.Tensor, log2_out: Optional[torch.Tensor], exp2
     assert inp.dtype == torch.float64
     _check(lib().cvlc_selftest_math(_ptr(inp), inp.numel(), _ptr(log2_out), _ptr(exp2_out), _ptr(div_out),
                                     _ptr(div_ref), _stream_handle(stream)), "cvlc_selftest_math")
+
+
+def cvlc_launch_count(kernel_name: str = "") -> int:
+    return int(lib().cvlc_launch_count(kernel_name.encode()))
+
+
+def cvlc_profile_select(kernel_name: Optional[str], max_launches: int) -> None:
+    _check(lib().cvlc_profile_select((kernel_name or "").encode(), int(max_launches)), "cvlc_profile_select")
+
+
+def cvlc_profile_reset() -> None:
+    _check(lib().cvlc_profile_reset(), "cvlc_profile_reset")
+
+
+def cvlc_profile_read():
+    n, ms = C.c_uint32(), C.c_double()
+    _check(lib().cvlc_profile_read(C.byref(n), C.byref(ms)), "cvlc_profile_read")
+    return int(n.value), float(ms.value)
 
 
 # ---- buffer helpers (allocation only) ---------------------------------------------------

@@ -94,6 +94,25 @@ struct PlanTables {
   uint32_t cap[CVLC_MAX_CODE_BITS + 1];      // cap(y) for every y
 };
 
+// ---- launch accounting and optional per-kernel timing ------------------------------
+
+enum KernelId {
+  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSortHist, kKSortPass, kKPack, kKDecodePrepare,
+  kKFillZero, kKDecode, kKSelftest, kNumKernelIds
+};
+
+// Called around every kernel launch.  Counts launches; when a kernel has been selected with
+// cvlc_profile_select, records a CUDA event pair on the launching stream around it.
+void launch_begin(int kernel_id, cudaStream_t st);
+void launch_end(int kernel_id, cudaStream_t st);
+
+struct LaunchScope {
+  int id;
+  cudaStream_t st;
+  LaunchScope(int id_, cudaStream_t st_) : id(id_), st(st_) { launch_begin(id, st); }
+  ~LaunchScope() { launch_end(id, st); }
+};
+
 // ---- launchers (one per translation unit) ---------------------------------------
 
 cudaError_t launch_plan(const float* x, const PlanTables& T, cvlc_plan_t* plan, void* ws, cudaStream_t st);

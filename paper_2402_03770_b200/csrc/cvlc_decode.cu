@@ -183,14 +183,15 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
                           void* ws, cudaStream_t st) {
   unsigned char* w = static_cast<unsigned char*>(ws);
-  k_decode_prepare<<<1, kPrepThreads, 0, st>>>(streams, stream_bytes, weights, n, weight_total, d, s, w);
+  { LaunchScope ls(kKDecodePrepare, st); k_decode_prepare<<<1, kPrepThreads, 0, st>>>(streams, stream_bytes, weights, n, weight_total, d, s, w); }
   if (!accumulate) {
     const uint64_t nvec = d >> 2;
     uint64_t want = (nvec + 255) / 256;
     const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? (want ? want : 1) : 8 * kNumSM);
+    LaunchScope ls(kKFillZero, st);
     k_fill_zero<<<grid, 256, 0, st>>>(out, d);
   }
-  k_decode<<<8 * kNumSM, kDecodeThreads, ((size_t)n + 1) * 4, st>>>(streams, n, d, s, out, w);
+  { LaunchScope ls(kKDecode, st); k_decode<<<8 * kNumSM, kDecodeThreads, ((size_t)n + 1) * 4, st>>>(streams, n, d, s, out, w); }
   return cudaGetLastError();
 }
 

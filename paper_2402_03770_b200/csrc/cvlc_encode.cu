@@ -532,21 +532,24 @@ cudaError_t launch_encode(const float* x, const cvlc_params& p, uint32_t s, uint
   unsigned long long* buf_a = reinterpret_cast<unsigned long long*>(w + L.off_buf_a);
   unsigned long long* buf_b = reinterpret_cast<unsigned long long*>(w + L.off_buf_b);
 
-  k_encode_init<<<2 * kNumSM, 256, 0, st>>>(w, plan, L, p.d, s, R);
+  { LaunchScope ls(kKEncodeInit, st); k_encode_init<<<2 * kNumSM, 256, 0, st>>>(w, plan, L, p.d, s, R); }
   {
     const uint64_t want = L.n_select_tiles;
     const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? want : 8 * kNumSM);
+    LaunchScope ls(kKSelect, st);
     k_select<<<grid, kSelectThreads, 0, st>>>(x, p.d, plan, hdr, sel_state, L.n_select_tiles, buf_a, p.d);
   }
   {
     const uint64_t want = L.max_sort_tiles;
     const int grid = (int)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
-    k_sort_hist<<<grid, 256, 0, st>>>(buf_a, plan, hdr, ghist);
-    for (int pass = 0; pass < kSortPasses; ++pass)
+    { LaunchScope ls(kKSortHist, st); k_sort_hist<<<grid, 256, 0, st>>>(buf_a, plan, hdr, ghist); }
+    for (int pass = 0; pass < kSortPasses; ++pass) {
+      LaunchScope ls(kKSortPass, st);
       k_sort_pass<<<grid, kSortThreads, 0, st>>>(pass, buf_a, buf_b, plan, hdr, ghist,
                                                  sort_state + (size_t)pass * L.max_sort_tiles * 256);
+    }
   }
-  k_pack<<<R, kPackThreads, pack_smem, st>>>(buf_a, buf_b, plan, hdr, ghist, p, s, R, reinterpret_cast<uint32_t*>(stream));
+  { LaunchScope ls(kKPack, st); k_pack<<<R, kPackThreads, pack_smem, st>>>(buf_a, buf_b, plan, hdr, ghist, p, s, R, reinterpret_cast<uint32_t*>(stream)); }
   return cudaGetLastError();
 }
 

@@ -451,23 +451,26 @@ k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__
 // ===================================================================================
 
 cudaError_t launch_plan(const float* x, const PlanTables& T, cvlc_plan_t* plan, void* ws, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
+  static bool attr_done[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+    e = cudaFuncSetAttribute(k_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev] = true;
   }
   unsigned char* w = static_cast<unsigned char*>(ws);
   unsigned long long* hist = reinterpret_cast<unsigned long long*>(w + kPlanWsHist);
   uint32_t* flag = reinterpret_cast<uint32_t*>(w + kPlanWsStatus + 4);
-  k_zero_words<<<8, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsBytes / 4);
+  { LaunchScope ls(kKZeroWords, st); k_zero_words<<<8, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsBytes / 4); }
   const uint64_t nvec = T.d >> 2;
   uint64_t want = (nvec + kHistThreads - 1) / kHistThreads;
   int grid = (int)(want < (uint64_t)(2 * kNumSM) ? (want ? want : 1) : 2 * kNumSM);
-  k_hist<<<grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(x, T.d, hist, flag);
-  k_plan<<<1, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flag, T, plan);
+  { LaunchScope ls(kKHist, st); k_hist<<<grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(x, T.d, hist, flag); }
+  { LaunchScope ls(kKPlan, st); k_plan<<<1, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flag, T, plan); }
   return cudaGetLastError();
 }
 
@@ -502,14 +505,14 @@ __global__ void k_selftest_math(const double* in, uint64_t n, double* l2, double
 cudaError_t launch_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t first, uint64_t n,
                                    uint32_t* out, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
-  k_selftest_philox<<<kNumSM, 256, 0, st>>>(seed, client_id, round, first, n, out);
+  { LaunchScope ls(kKSelftest, st); k_selftest_philox<<<kNumSM, 256, 0, st>>>(seed, client_id, round, first, n, out); }
   return cudaGetLastError();
 }
 
 cudaError_t launch_selftest_math(const double* in, uint64_t n, double* l2, double* e2, double* dv, double* dr,
                                  cudaStream_t st) {
   if (n == 0) return cudaSuccess;
-  k_selftest_math<<<kNumSM, 256, 0, st>>>(in, n, l2, e2, dv, dr);
+  { LaunchScope ls(kKSelftest, st); k_selftest_math<<<kNumSM, 256, 0, st>>>(in, n, l2, e2, dv, dr); }
   return cudaGetLastError();
 }
 

@@ -161,7 +161,7 @@ def test_ties_zeros_and_negative_zero(torch_cuda):
     x = (np.round(rng.standard_normal(d) * 4) / 4).astype(np.float32)          # heavy ties, both signs
     x[5000:30000] = 0.0
     x[5000:30000:3] = -0.0
-    pd = params_dict(d, 30 * 2048, packet_bits=2048, seed=9)
+    pd = params_dict(d, 220 * 2048, packet_bits=2048, seed=9)
     of, ost = run_case(x, pd)
     assert of["k"] > np.count_nonzero(x)                                         # zeros are in the stream
     pd2 = params_dict(d, 12 * 2048, packet_bits=2048, seed=9)

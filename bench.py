@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the Fed-CVLC compression path on B200.
+
+One step = one federated round's compression work for one batch of clients:
+plan + encode of every client's fp32 update, then decode-aggregate of all their
+streams into the dense averaged update.  Inputs are synthetic (seeded, shaped like
+CNN updates) and resident in HBM when the timed region starts; the `e2e` figure
+repeats the step with every update copied from pinned host memory and the
+aggregate copied back inside the timed region.
+
+    python bench.py --gpus 1 --steps 5 --warmup 3
+    python bench.py --impl reference          # the CPU oracle, timed on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2402_03770_b200 import workloads as W  # noqa: E402
+
+METRIC = "encode+decode_aggregate throughput (4*d*clients / step time)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the
+# kernel named by --profile-kernel (profiles/); None when no capture matches the current kernel.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18")
+    ap.add_argument("--bits-per-coord", type=float, default=2.0)
+    ap.add_argument("--clients", type=int, default=0, help="0 = the workload's client count")
+    ap.add_argument("--d", type=int, default=0, help="0 = the workload's d (smaller values are for profiling)")
+    ap.add_argument("--streams", type=int, default=8, help="CUDA streams the clients' encodes are spread over")
+    ap.add_argument("--profile-kernel", default="k_select")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample-clients", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle as it stands, on a bounded sample of the workload
+# --------------------------------------------------------------------------------------------
+
+def oracle_step(w, d, bpc, clients):
+    """plan + encode of `clients`, then decode-aggregate of their streams; returns seconds"""
+    import oracle as O
+    xs = [W.client_update(w, c, d=d) for c in clients]
+    weights = W.client_weights(w)[[c % w.n_clients for c in clients]]
+    t0 = time.perf_counter()
+    streams = []
+    for c, x in zip(clients, xs):
+        seed, cid, rnd = W.philox_ids(w, c)
+        p = O.make_params(d, int(np.floor(bpc * d)), seed=seed, client_id=cid, round=rnd)
+        streams.append(O.encode(x, p, O.plan(x, p)))
+    O.decode_aggregate(streams, weights, d)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = W.WORKLOADS[args.workload]
+    d = args.d or w.d
+    n = max(1, args.cpu_sample_clients)
+    clients = list(range(n))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(w, d, args.bits_per_coord, clients[:1])
+    times = [oracle_step(w, d, args.bits_per_coord, clients) for _ in range(args.steps)]
+    t = float(np.mean(times))
+    value = 4.0 * d * n / t / 1e9
+    sample = f"{n} of {args.clients or w.n_clients} clients per step (plan+encode each, decode-aggregate of those {n})"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64 plan / f32 data", "data": "synthetic",
+        "config": {"workload": f"{w.name} d={d} bits_per_coord={args.bits_per_coord}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "params_per_s": d * n / t,
+    }))
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2402_03770_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.lib()
+    B.cvlc_set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = W.WORKLOADS[args.workload]
+    d = args.d or w.d
+    n_clients = args.clients or w.n_clients
+    bpc = args.bits_per_coord
+    budget = int(np.floor(bpc * d))
+    first_client = rank * n_clients  # every rank is an independent replica with its own clients
+
+    # ---- inputs: seeded host generation (threads; numpy releases the GIL), then HBM-resident
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 4)) as ex:
+        host_x = list(ex.map(lambda c: W.client_update(w, first_client + c, d=d), range(n_clients)))
+    pinned = [torch.from_numpy(x).pin_memory() for x in host_x] if not args.no_e2e else None
+    dev_x = [torch.from_numpy(x).to(dev) for x in host_x]
+    weights = torch.from_numpy(W.client_weights(w)[[(first_client + c) % w.n_clients for c in range(n_clients)]].copy())
+
+    params = []
+    for c in range(n_clients):
+        seed, cid, rnd = W.philox_ids(w, first_client + c)
+        params.append(B.make_params(d, budget, seed=seed, client_id=cid, round=rnd))
+    n_streams = max(1, min(args.streams, n_clients))
+    streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams)]
+    encoders = [B.ClientEncoder(params[0], dev) for _ in range(n_streams)]
+    stage = [torch.empty(d, dtype=torch.float32, device=dev) for _ in range(n_streams)] if not args.no_e2e else None
+    out_streams = [B.alloc_bytes(B.cvlc_stream_bytes(params[0]), dev) for _ in range(n_clients)]
+    agg = B.Aggregator(n_clients, d, dev)
+    agg.set_clients(out_streams, weights)
+    result = torch.empty(d, dtype=torch.float32, device=dev)
+    result_host = torch.empty(d, dtype=torch.float32).pin_memory() if not args.no_e2e else None
+    main = torch.cuda.current_stream(dev)
+    done = [torch.cuda.Event() for _ in range(n_streams)]
+    fork = torch.cuda.Event()
+
+    def step(from_host: bool):
+        fork.record(main)
+        for s in streams:
+            s.wait_event(fork)
+        for c in range(n_clients):
+            slot = c % n_streams
+            s = streams[slot]
+            if from_host:
+                with torch.cuda.stream(s):
+                    stage[slot].copy_(pinned[c], non_blocking=True)
+                x = stage[slot]
+            else:
+                x = dev_x[c]
+            encoders[slot].run(x, p=params[c], out=out_streams[c], stream=s)
+        for s, e in zip(streams, done):
+            e.record(s)
+            main.wait_event(e)
+        agg.run(n_clients, result, stream=main)
+        if from_host:
+            result_host.copy_(result, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(n_steps: int, from_host: bool):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        barrier()
+        ev[0].record(main)
+        for i in range(n_steps):
+            step(from_host)
+            ev[i + 1].record(main)
+        barrier()
+        total_ms = ev[0].elapsed_time(ev[-1])
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(n_steps)]
+        if world > 1:
+            t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms, per
+
+    for _ in range(max(args.warmup, 3)):
+        step(False)
+    barrier()
+    for enc in encoders:
+        assert enc.status() == B.CVLC_OK, "encode reported a device-side error"
+    assert agg.status() == B.CVLC_OK, "decode-aggregate reported a device-side error"
+
+    launches_before = B.cvlc_launch_count()
+    per_step_launch_cap = 8 * n_clients + 8
+    B.cvlc_profile_select(args.profile_kernel, per_step_launch_cap * args.steps)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    total_ms, per = timed(args.steps, False)
+    clocks = sampler.stop() if rank == 0 else None
+    gpu_launches = B.cvlc_launch_count() - launches_before
+    prof_n, prof_ms = B.cvlc_profile_read()
+    B.cvlc_profile_select(None, 0)
+
+    ms_per_step = total_ms / args.steps
+    units = d * n_clients * world
+    value = 4.0 * units / (ms_per_step * 1e-3) / 1e9
+
+    e2e = None
+    if not args.no_e2e:
+        step(True)
+        e2e_ms, _ = timed(max(1, args.e2e_steps), True)
+        e2e_ms /= max(1, args.e2e_steps)
+        e2e = {"value": 4.0 * units / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": 4 * d * n_clients, "d2h_bytes_per_step": 4 * d}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the profiled kernel: algorithmic bytes per launch / mean launch duration
+    plan0 = B.read_plan(encoders[0].plan)
+    stream_bytes = B.cvlc_stream_bytes(params[0])
+    alg_bytes = {
+        "k_hist": 4.0 * d,
+        "k_select": 4.0 * d + 8.0 * plan0.n_candidates,
+        "k_sort_pass": 16.0 * plan0.n_candidates,
+        "k_pack": 8.0 * plan0.k + stream_bytes,
+        "k_decode": float(n_clients) * stream_bytes + 4.0 * d,
+        "k_fill_zero": 4.0 * d,
+    }.get(args.profile_kernel)
+    peak, peak_kind = measured_hbm_peak()
+    roofline = None
+    if alg_bytes and prof_n:
+        achieved = alg_bytes / (prof_ms / prof_n * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": args.profile_kernel, "achieved": achieved, "peak": peak,
+                    "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": NCU_TRAFFIC_BYTES.get(args.profile_kernel), "launches_timed": prof_n,
+                    "mean_launch_us": prof_ms / prof_n * 1e3, "algorithmic_bytes_per_launch": alg_bytes}
+    # whole-step minimum bytes (read every update once, write every stream; read the streams, write the aggregate)
+    step_min_bytes = n_clients * (4.0 * d + stream_bytes) + n_clients * stream_bytes + 4.0 * d
+    step_frac = step_min_bytes / (ms_per_step * 1e-3) / 1e9 / peak
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_s = max(1, min(args.cpu_sample_clients, n_clients))
+        t = oracle_step(w, d, bpc, list(range(n_s)))
+        cpu_baseline = {"value": 4.0 * d * n_s / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"{n_s} of {n_clients} clients: plan+encode each, decode-aggregate of those {n_s}; {t:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 data / f64 plan+quantizer / u32 keys", "data": "synthetic",
+        "config": {"workload": f"{w.name} d={d} clients={n_clients} bits_per_coord={bpc} packet=1500B",
+                   "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams,
+                   "multi_gpu": "replicas only: every rank runs its own clients and aggregator"},
+        "params_per_s": units / (ms_per_step * 1e-3),
+        "step_min_bytes_frac_of_hbm_peak": step_frac,
+        "per_step_ms": per,
+        "plan": {"k": int(plan0.k), "R": int(plan0.R), "n_candidates": int(plan0.n_candidates), "alpha_q": plan0.alpha_q,
+                 "lengths": {str(y): int(plan0.n_y[y]) for y in range(33) if plan0.n_y[y]}},
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(gpu_launches),
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -170,6 +170,32 @@ int cvlc_decode_aggregate(const uint8_t* const* streams_dev, const uint64_t* str
                           uint64_t d, float* out_dev, int accumulate, void* ws_dev, size_t ws_bytes,
                           void* cuda_stream);
 
+/*
+ * The same aggregation as cvlc_decode_aggregate for callers that cannot allocate device
+ * memory (the paper has no counterpart to this entry point; it exists for integration).
+ * Such callers are, for example, code that runs inside another framework's memory pool
+ * with no spare capacity, a plugin that is forbidden to call cudaMalloc after start-up,
+ * or a real-time serving loop where an allocation could stall on the driver.  Instead of
+ * a workspace argument the call uses a scratch array built into the library (a few KB per
+ * GPU, held from library load to process exit), so it handles at most
+ * CVLC_NOALLOC_MAX_CLIENTS clients per call; more returns CVLC_ERR_WORKSPACE_TOO_SMALL
+ * and launches nothing.  It calls no cudaMalloc / cudaFree and no allocating routine.
+ *  - All arguments as in cvlc_decode_aggregate, plus status_dev: one int32 of the
+ *    caller's device memory that receives the device status (0 or CVLC_ERR_BAD_STREAM,
+ *    ...) when the stream reaches that point; read it after synchronising.
+ *  - The first call on each device looks the scratch's device address up (with that
+ *    device current); make that first call outside of any stream capture.
+ *  - Every call on a device shares the one scratch.  Each call resets what it needs, so
+ *    calls that run one after another are independent, but two calls whose kernels may
+ *    overlap on the GPU (different streams, no ordering between them) race on it: order
+ *    them, or use cvlc_decode_aggregate with separate workspaces.
+ */
+#define CVLC_NOALLOC_MAX_CLIENTS 256
+int cvlc_decode_aggregate_noalloc(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev,
+                                  const float* weights_dev, uint32_t n_clients, double weight_total,
+                                  uint64_t d, float* out_dev, int accumulate, int32_t* status_dev,
+                                  void* cuda_stream);
+
 /* Waits for cuda_stream and returns the status word at byte 0 of a plan or workspace. */
 int cvlc_read_status(const void* plan_or_ws_dev, void* cuda_stream);
 

@@ -41,7 +41,7 @@ EXPORTS = [
     "cvlc_plan_workspace_bytes", "cvlc_encode_workspace_bytes", "cvlc_decode_workspace_bytes",
     "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math",
-    "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
+    "cvlc_decode_aggregate_noalloc", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -113,6 +113,8 @@ def lib() -> C.CDLL:
     L.cvlc_encode.argtypes = [vp, PP, vp, vp, sz, vp, sz, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
     L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
+    L.cvlc_decode_aggregate_noalloc.restype = C.c_int
+    L.cvlc_decode_aggregate_noalloc.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, vp]
     L.cvlc_read_status.restype = C.c_int
     L.cvlc_read_status.argtypes = [vp, vp]
     L.cvlc_selftest_philox.restype = C.c_int
@@ -222,6 +224,25 @@ def cvlc_decode_aggregate(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor,
                                        float(weight_total), int(d), _ptr(out), 1 if accumulate else 0,
                                        _ptr(ws), ws.numel() * ws.element_size(), _stream_handle(stream)),
            "cvlc_decode_aggregate")
+
+
+NOALLOC_MAX_CLIENTS = 256
+
+
+def cvlc_decode_aggregate_noalloc(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor,
+                                  n_clients: int, weight_total: float, d: int, out: torch.Tensor,
+                                  accumulate: bool, status: torch.Tensor,
+                                  stream: Optional[torch.cuda.Stream] = None) -> None:
+    """cvlc_decode_aggregate without a workspace argument: for callers that may not allocate
+    device memory.  Uses the library's built-in scratch (at most NOALLOC_MAX_CLIENTS clients);
+    `status` is one int32 device word that receives the device status.  Calls on one device
+    must not overlap on the GPU."""
+    assert status.dtype == torch.int32 and status.numel() >= 1
+    assert weights.dtype == torch.float32 and out.dtype == torch.float32 and out.numel() == d
+    _check(lib().cvlc_decode_aggregate_noalloc(_ptr(stream_ptrs), _ptr(stream_bytes), _ptr(weights), int(n_clients),
+                                               float(weight_total), int(d), _ptr(out), 1 if accumulate else 0,
+                                               _ptr(status), _stream_handle(stream)),
+           "cvlc_decode_aggregate_noalloc")
 
 
 def cvlc_read_status(plan_or_ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:

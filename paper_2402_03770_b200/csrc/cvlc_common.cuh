@@ -55,7 +55,7 @@ struct EncLayout {
 #define CVLC_HD
 #endif
 
-CVLC_HD static inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+CVLC_HD constexpr size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 static inline EncLayout enc_layout(uint64_t d) {
   EncLayout L;
@@ -73,10 +73,10 @@ static inline EncLayout enc_layout(uint64_t d) {
 constexpr size_t kDecWsStatus = 0;     // int32 status
 constexpr size_t kDecWsTotalPkts = 8;  // uint32 total packets
 constexpr size_t kDecWsCoef = 256;     // float[n]
-CVLC_HD static inline size_t dec_off_prefix(uint32_t n) { return align256(kDecWsCoef + (size_t)n * 4); }  // uint32[n+1]
-CVLC_HD static inline size_t dec_off_meta(uint32_t n) { return align256(dec_off_prefix(n) + ((size_t)n + 1) * 4); }
+CVLC_HD constexpr size_t dec_off_prefix(uint32_t n) { return align256(kDecWsCoef + (size_t)n * 4); }  // uint32[n+1]
+CVLC_HD constexpr size_t dec_off_meta(uint32_t n) { return align256(dec_off_prefix(n) + ((size_t)n + 1) * 4); }
 // per client: packet_bits, header_bits (uint32 each)
-CVLC_HD static inline size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta(n) + (size_t)n * 8); }
+CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta(n) + (size_t)n * 8); }
 
 // ---- host-side tables handed to the planning kernel -----------------------------
 

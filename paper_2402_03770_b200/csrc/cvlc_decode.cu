@@ -196,3 +196,71 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
 }
 
 }  // namespace cvlc
+
+// ===================================================================================
+// Decode-aggregate for callers that cannot allocate device memory
+// ===================================================================================
+
+namespace cvlc {
+
+// Scratch of cvlc_decode_aggregate_noalloc: the decode workspace for up to
+// CVLC_NOALLOC_MAX_CLIENTS clients (a few KB), resident in every GPU that loads the
+// library until the process exits.
+constexpr size_t kNoAllocScratchBytes = dec_ws_bytes(CVLC_NOALLOC_MAX_CLIENTS);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// copies the status word of the scratch to the caller's word (device code names the array directly)
+__global__ void k_noalloc_publish_status(int32_t* status_out) {
+  *status_out = *reinterpret_cast<const int32_t*>(g_noalloc_scratch + kDecWsStatus);
+}
+
+// Device address of the scratch on the current device.  In host code the array's name is only a
+// handle for the runtime, so the address is asked for once per device and cached.
+static cudaError_t noalloc_scratch_address(void** out) {
+  static void* cached[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return cudaSuccess;
+}
+
+}  // namespace cvlc
+
+extern "C" int cvlc_decode_aggregate_noalloc(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev,
+                                             const float* weights_dev, uint32_t n_clients, double weight_total,
+                                             uint64_t d, float* out_dev, int accumulate, int32_t* status_dev,
+                                             void* cuda_stream) {
+  using namespace cvlc;
+  if (n_clients == 0) return CVLC_ERR_INVALID_ARG;
+  if (n_clients > CVLC_NOALLOC_MAX_CLIENTS) return CVLC_ERR_WORKSPACE_TOO_SMALL;  // beyond the built-in scratch
+  if (d < 2 || d > (1ull << 31)) return CVLC_ERR_INVALID_ARG;
+  if (!(weight_total >= 0.0) || !(weight_total < 1e300)) return CVLC_ERR_INVALID_ARG;
+  auto aligned = [](const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; };
+  if (!aligned(streams_dev, 8) || !aligned(stream_bytes_dev, 8) || !aligned(weights_dev, 4) || !aligned(out_dev, 16) ||
+      !aligned(status_dev, 4))
+    return CVLC_ERR_INVALID_ARG;
+  void* scratch = nullptr;
+  if (noalloc_scratch_address(&scratch) != cudaSuccess) return CVLC_ERR_CUDA;
+  uint32_t s = 1;
+  while ((1ull << s) < d) ++s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // k_decode_prepare resets the status word and rewrites every table entry it later reads,
+  // so nothing of the previous call's contents is used
+  if (launch_decode(streams_dev, stream_bytes_dev, weights_dev, n_clients, weight_total, d, s, out_dev,
+                    accumulate ? 1 : 0, scratch, st) != cudaSuccess)
+    return CVLC_ERR_CUDA;
+  {
+    LaunchScope ls(kKDecodePrepare, st);
+    k_noalloc_publish_status<<<1, 1, 0, st>>>(status_dev);
+  }
+  return cudaGetLastError() == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+}
+

@@ -49,7 +49,10 @@ def parse_args():
     ap.add_argument("--bits-per-coord", type=float, default=2.0)
     ap.add_argument("--clients", type=int, default=0, help="0 = the workload's client count")
     ap.add_argument("--d", type=int, default=0, help="0 = the workload's d (smaller values are for profiling)")
-    ap.add_argument("--streams", type=int, default=8, help="CUDA streams the clients' encodes are spread over")
+    ap.add_argument("--batch", type=int, default=0, help="clients per plan/encode call; 0 = all clients in one call")
+    ap.add_argument("--streams", type=int, default=2, help="CUDA streams the batches are spread over")
+    ap.add_argument("--max-candidates", type=int, default=0,
+                    help="candidate slots per client in the encode workspace; 0 = 3 * R * cap(1)")
     ap.add_argument("--profile-kernel", default="k_select")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-clients", type=int, default=3)
@@ -200,11 +203,17 @@ def run_ours(args):
     for c in range(n_clients):
         seed, cid, rnd = W.philox_ids(w, first_client + c)
         params.append(B.make_params(d, budget, seed=seed, client_id=cid, round=rnd))
-    n_streams = max(1, min(args.streams, n_clients))
+    batch = args.batch or n_clients
+    groups = [list(range(i, min(i + batch, n_clients))) for i in range(0, n_clients, batch)]
+    n_streams = max(1, min(args.streams, len(groups)))
     streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams)]
-    encoders = [B.ClientEncoder(params[0], dev) for _ in range(n_streams)]
-    stage = [torch.empty(d, dtype=torch.float32, device=dev) for _ in range(n_streams)] if not args.no_e2e else None
-    out_streams = [B.alloc_bytes(B.cvlc_stream_bytes(params[0]), dev) for _ in range(n_clients)]
+    if args.max_candidates:
+        max_cand = args.max_candidates
+    else:
+        s_bits = max(1, int(np.ceil(np.log2(d))))
+        max_cand = min(d, 3 * (budget // 12000) * ((12000 - 80) // (s_bits + 1)))
+    encoders = [B.BatchEncoder([params[c] for c in g], dev, max_candidates=max_cand) for g in groups]
+    out_streams = [o for enc in encoders for o in enc.outs]
     agg = B.Aggregator(n_clients, d, dev)
     agg.set_clients(out_streams, weights)
     result = torch.empty(d, dtype=torch.float32, device=dev)
@@ -217,16 +226,13 @@ def run_ours(args):
         fork.record(main)
         for s in streams:
             s.wait_event(fork)
-        for c in range(n_clients):
-            slot = c % n_streams
-            s = streams[slot]
+        for gi, g in enumerate(groups):
+            s = streams[gi % n_streams]
             if from_host:
                 with torch.cuda.stream(s):
-                    stage[slot].copy_(pinned[c], non_blocking=True)
-                x = stage[slot]
-            else:
-                x = dev_x[c]
-            encoders[slot].run(x, p=params[c], out=out_streams[c], stream=s)
+                    for c in g:
+                        dev_x[c].copy_(pinned[c], non_blocking=True)
+            encoders[gi].run([dev_x[c] for c in g], stream=s)
         for s, e in zip(streams, done):
             e.record(s)
             main.wait_event(e)
@@ -264,7 +270,7 @@ def run_ours(args):
     assert agg.status() == B.CVLC_OK, "decode-aggregate reported a device-side error"
 
     launches_before = B.cvlc_launch_count()
-    per_step_launch_cap = 8 * n_clients + 8
+    per_step_launch_cap = 8 * len(groups) + 8
     B.cvlc_profile_select(args.profile_kernel, per_step_launch_cap * args.steps)
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -294,13 +300,13 @@ def run_ours(args):
         return
 
     # ---- roofline of the profiled kernel: algorithmic bytes per launch / mean launch duration
-    plan0 = B.read_plan(encoders[0].plan)
+    plan0 = encoders[0].read_plan(0)
     stream_bytes = B.cvlc_stream_bytes(params[0])
     alg_bytes = {
-        "k_hist": 4.0 * d,
-        "k_select": 4.0 * d + 8.0 * plan0.n_candidates,
-        "k_sort_pass": 16.0 * plan0.n_candidates,
-        "k_pack": 8.0 * plan0.k + stream_bytes,
+        "k_hist": 4.0 * d * n_clients / len(groups),
+        "k_select": (4.0 * d + 8.0 * plan0.n_candidates) * n_clients / len(groups),
+        "k_sort_pass": 16.0 * plan0.n_candidates * n_clients / len(groups),
+        "k_pack": (8.0 * plan0.k + stream_bytes) * n_clients / len(groups),
         "k_decode": float(n_clients) * stream_bytes + 4.0 * d,
         "k_fill_zero": 4.0 * d,
     }.get(args.profile_kernel)
@@ -328,7 +334,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 data / f64 plan+quantizer / u32 keys", "data": "synthetic",
         "config": {"workload": f"{w.name} d={d} clients={n_clients} bits_per_coord={bpc} packet=1500B",
-                   "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams,
+                   "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams, "clients_per_call": batch, "max_candidates": int(max_cand),
                    "multi_gpu": "replicas only: every rank runs its own clients and aggregator"},
         "params_per_s": units / (ms_per_step * 1e-3),
         "step_min_bytes_frac_of_hbm_peak": step_frac,

@@ -58,6 +58,7 @@ enum {
 #define CVLC_STREAM_HEADER_BYTES 64
 #define CVLC_STREAM_MAGIC 0x434C5643u
 #define CVLC_MAX_CLIENTS_PER_CALL 4096
+#define CVLC_MAX_BATCH 512
 
 /* Problem statement of Section IV-C: the update has d coordinates, the client may
  * send budget_bits this round in packets of packet_bits (b) with header_bits (H)
@@ -150,6 +151,32 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev,
                 uint8_t* stream_dev, size_t stream_capacity, void* ws_dev, size_t ws_bytes,
                 void* cuda_stream);
+
+/*
+ * Batched forms: the same kernels over n clients (n <= CVLC_MAX_BATCH) in one set of
+ * launches, for a process that compresses many clients' updates on one GPU.  All clients
+ * of a batch share d, the packet count floor(budget_bits / b), b, H, the quantizer and
+ * max_code_bits (else INVALID_ARG); scale_B, seed, client_id and round are per client.
+ *  x_dev        HOST array of n device pointers (each update d fp32, 16-byte aligned)
+ *  params       HOST array of n cvlc_params
+ *  fixed_y      0 = tune the lengths (cvlc_plan); 1..32 = every packet at this length
+ *  plans_dev    DEVICE array of n plans; plans_dev[i].status carries client i's status and
+ *               byte 0 of the workspace the first error of the batch
+ *  streams_dev  HOST array of n device pointers, each with stream_capacity bytes
+ *  max_candidates  candidate slots per client in the encode workspace; 0 = d (always
+ *               enough).  A plan whose n_candidates exceeds it makes the whole batch fail
+ *               with WORKSPACE_TOO_SMALL (device-detected, byte 0 of the workspace).
+ * A device-detected error in one client (non-finite input, plan mismatch) stops the
+ * encoding of the whole batch.  After cvlc_plan_batch the histogram of client i sits at
+ * byte 256 + 32768 * i of the workspace.
+ */
+size_t cvlc_plan_batch_workspace_bytes(const cvlc_params* p, uint32_t n);
+size_t cvlc_encode_batch_workspace_bytes(const cvlc_params* p, uint32_t n, uint64_t max_candidates);
+int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint32_t fixed_y,
+                    cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n,
+                      const cvlc_plan_t* plans_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                      uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream);
 
 /*
  * Parameter-server aggregation (Section III, step 3) fused with decoding: for every

@@ -32,6 +32,7 @@ CVLC_ERR_SCALE_TOO_SMALL = 12
 CVLC_ERR_PLAN_MISMATCH = 13
 
 MAX_CODE_BITS = 32
+MAX_BATCH = 512
 HIST_BINS = 4096
 PLAN_BYTES = 512
 PLAN_WS_HIST_OFFSET = 256
@@ -39,7 +40,8 @@ PLAN_WS_HIST_OFFSET = 256
 EXPORTS = [
     "cvlc_version", "cvlc_status_string", "cvlc_set_device", "cvlc_stream_bytes", "cvlc_default_scale",
     "cvlc_plan_workspace_bytes", "cvlc_encode_workspace_bytes", "cvlc_decode_workspace_bytes",
-    "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_decode_aggregate", "cvlc_read_status",
+    "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_plan_batch_workspace_bytes",
+    "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math",
     "cvlc_decode_aggregate_noalloc", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
@@ -111,6 +113,14 @@ def lib() -> C.CDLL:
     L.cvlc_plan_fixed.argtypes = [vp, PP, u32, vp, vp, sz, vp]
     L.cvlc_encode.restype = C.c_int
     L.cvlc_encode.argtypes = [vp, PP, vp, vp, sz, vp, sz, vp]
+    L.cvlc_plan_batch_workspace_bytes.restype = sz
+    L.cvlc_plan_batch_workspace_bytes.argtypes = [PP, u32]
+    L.cvlc_encode_batch_workspace_bytes.restype = sz
+    L.cvlc_encode_batch_workspace_bytes.argtypes = [PP, u32, u64]
+    L.cvlc_plan_batch.restype = C.c_int
+    L.cvlc_plan_batch.argtypes = [vp, PP, u32, u32, vp, vp, sz, vp]
+    L.cvlc_encode_batch.restype = C.c_int
+    L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, sz, u64, vp, sz, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
     L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
     L.cvlc_decode_aggregate_noalloc.restype = C.c_int
@@ -212,6 +222,44 @@ def cvlc_encode(x: torch.Tensor, p: CvlcParams, plan: torch.Tensor, out_stream: 
     assert out_stream.dtype == torch.uint8
     _check(lib().cvlc_encode(_ptr(x), C.byref(p), _ptr(plan), _ptr(out_stream), out_stream.numel(),
                              _ptr(ws), ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode")
+
+
+def cvlc_plan_batch_workspace_bytes(p: CvlcParams, n: int) -> int:
+    return int(lib().cvlc_plan_batch_workspace_bytes(C.byref(p), int(n)))
+
+
+def cvlc_encode_batch_workspace_bytes(p: CvlcParams, n: int, max_candidates: int = 0) -> int:
+    return int(lib().cvlc_encode_batch_workspace_bytes(C.byref(p), int(n), int(max_candidates)))
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    return (C.c_void_p * len(tensors))(*[_ptr(t) for t in tensors])
+
+
+def _params_array(params: Sequence[CvlcParams]):
+    return (CvlcParams * len(params))(*params)
+
+
+def cvlc_plan_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor, ws: torch.Tensor,
+                    fixed_y: int = 0, stream: Optional[torch.cuda.Stream] = None, _cache=None) -> None:
+    """xs: n device tensors; params: n CvlcParams; plans: device uint8 tensor of n * 512 bytes."""
+    n = len(xs)
+    assert len(params) == n and plans.dtype == torch.uint8 and plans.numel() >= n * PLAN_BYTES
+    xa, pa = _cache if _cache is not None else (_ptr_array(xs), _params_array(params))
+    _check(lib().cvlc_plan_batch(xa, pa, n, int(fixed_y), _ptr(plans), _ptr(ws), ws.numel() * ws.element_size(),
+                                 _stream_handle(stream)), "cvlc_plan_batch")
+
+
+def cvlc_encode_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor,
+                      outs: Sequence[torch.Tensor], ws: torch.Tensor, max_candidates: int = 0,
+                      stream: Optional[torch.cuda.Stream] = None, _cache=None) -> None:
+    """outs: n device uint8 tensors of cvlc_stream_bytes(params[0]) bytes each."""
+    n = len(xs)
+    assert len(params) == n and len(outs) == n
+    xa, pa, oa = _cache if _cache is not None else (_ptr_array(xs), _params_array(params), _ptr_array(outs))
+    cap = min(o.numel() for o in outs)
+    _check(lib().cvlc_encode_batch(xa, pa, n, _ptr(plans), oa, cap, int(max_candidates), _ptr(ws),
+                                   ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode_batch")
 
 
 def cvlc_decode_aggregate(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor,
@@ -320,6 +368,37 @@ class ClientEncoder:
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         rc = cvlc_read_status(self.plan, stream)
         return rc if rc != CVLC_OK else cvlc_read_status(self.enc_ws, stream)
+
+
+class BatchEncoder:
+    """Buffers for plan + encode of a batch of n clients that share a problem shape."""
+
+    def __init__(self, params: Sequence[CvlcParams], device: torch.device, max_candidates: int = 0):
+        self.params = list(params)
+        self.n = len(self.params)
+        self.device = device
+        self.max_candidates = max_candidates
+        p0 = self.params[0]
+        self.plans = alloc_bytes(PLAN_BYTES * self.n, device)
+        self.plan_ws = alloc_bytes(cvlc_plan_batch_workspace_bytes(p0, self.n), device)
+        self.enc_ws = alloc_bytes(cvlc_encode_batch_workspace_bytes(p0, self.n, max_candidates), device)
+        self.outs = [alloc_bytes(cvlc_stream_bytes(p0), device) for _ in range(self.n)]
+        self._pa = _params_array(self.params)
+        self._oa = _ptr_array(self.outs)
+
+    def run(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0):
+        xa = _ptr_array(xs)
+        cvlc_plan_batch(xs, self.params, self.plans, self.plan_ws, fixed_y, stream, _cache=(xa, self._pa))
+        cvlc_encode_batch(xs, self.params, self.plans, self.outs, self.enc_ws, self.max_candidates, stream,
+                          _cache=(xa, self._pa, self._oa))
+        return self.outs
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        rc = cvlc_read_status(self.plan_ws, stream)
+        return rc if rc != CVLC_OK else cvlc_read_status(self.enc_ws, stream)
+
+    def read_plan(self, i: int) -> CvlcPlan:
+        return read_plan(self.plans[i * PLAN_BYTES:(i + 1) * PLAN_BYTES])
 
 
 class Aggregator:

@@ -57,51 +57,40 @@ double coeff_g(double Q, double B) {
   return 1.0 - c;
 }
 
-int build_tables(const cvlc_params* p, uint32_t fixed_y, PlanTables* T) {
+// Checks one client's parameters and fills the shape shared by a batch.  The per-length
+// coefficients are rebuilt on the device from scale_B with the same IEEE operations; the host
+// evaluates them here only to reject parameters for which no length is usable.
+int build_shape(const cvlc_params* p, uint32_t fixed_y, Shape* S) {
   Derived D;
   const int rc = derive(p, &D);
   if (rc != CVLC_OK) return rc;
-  memset(T, 0, sizeof *T);
-  T->d = p->d;
-  T->s = D.s;
-  T->R = D.R;
-  T->fixed_y = fixed_y;
-  for (uint32_t y = 0; y <= CVLC_MAX_CODE_BITS; ++y) T->cap[y] = D.cap[y];
+  memset(S, 0, sizeof *S);
+  S->d = p->d;
+  S->s = D.s;
+  S->R = D.R;
+  S->packet_bits = p->packet_bits;
+  S->header_bits = p->header_bits;
+  S->quantizer = p->quantizer;
+  S->max_code_bits = p->max_code_bits;
+  S->fixed_y = fixed_y;
+  for (uint32_t y = 0; y <= CVLC_MAX_CODE_BITS; ++y) S->cap[y] = D.cap[y];
   if (fixed_y) {
     if (fixed_y > p->max_code_bits) return CVLC_ERR_INVALID_ARG;
     if ((uint64_t)D.R * D.cap[fixed_y] > p->d) return CVLC_ERR_BUDGET_TOO_LARGE;
-    T->nY = 1;
-    T->y_min = fixed_y;
-    T->Y[0] = fixed_y;
-    T->capY[0] = D.cap[fixed_y];
-    T->QY[0] = quant_Q(D.cap[fixed_y], fixed_y);
-    T->gY[0] = coeff_g(T->QY[0], p->scale_B);
     return CVLC_OK;
   }
-  double Q[CVLC_MAX_CODE_BITS + 1], g[CVLC_MAX_CODE_BITS + 1];
-  uint32_t y_min = 0;
-  for (uint32_t y = 1; y <= p->max_code_bits; ++y) {
-    Q[y] = quant_Q(D.cap[y], y);
-    g[y] = coeff_g(Q[y], p->scale_B);
-    if (y_min == 0 && g[y] > 0.0) y_min = y;
-  }
-  if (y_min == 0) return CVLC_ERR_SCALE_TOO_SMALL;
-  T->y_min = y_min;
-  uint32_t nY = 0;
-  for (uint32_t y = y_min; y <= p->max_code_bits; ++y) {
-    // a length that fits no more records than the next longer one is dominated
-    if (y == p->max_code_bits || D.cap[y] > D.cap[y + 1]) {
-      T->Y[nY] = y;
-      T->capY[nY] = D.cap[y];
-      T->QY[nY] = Q[y];
-      T->gY[nY] = g[y];
-      ++nY;
-    }
-  }
-  T->nY = nY;
+  bool usable = false;
+  for (uint32_t y = 1; y <= p->max_code_bits; ++y)
+    if (coeff_g(quant_Q(D.cap[y], y), p->scale_B) > 0.0) usable = true;
+  if (!usable) return CVLC_ERR_SCALE_TOO_SMALL;
   // an admissible single-length plan must exist: the longest code sends the fewest coordinates
   if ((uint64_t)D.R * D.cap[p->max_code_bits] > p->d) return CVLC_ERR_BUDGET_TOO_LARGE;
   return CVLC_OK;
+}
+
+bool same_shape(const cvlc_params& a, const cvlc_params& b) {
+  return a.d == b.d && a.budget_bits / a.packet_bits == b.budget_bits / b.packet_bits && a.packet_bits == b.packet_bits &&
+         a.header_bits == b.header_bits && a.quantizer == b.quantizer && a.max_code_bits == b.max_code_bits;
 }
 
 bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -151,52 +140,105 @@ double cvlc_default_scale(const cvlc_params* p) {
   return 1.0 + quant_Q(cap8, 8);
 }
 
-size_t cvlc_plan_workspace_bytes(const cvlc_params* p) { return params_ok(p) ? kPlanWsBytes : 0; }
+size_t cvlc_plan_workspace_bytes(const cvlc_params* p) { return cvlc_plan_batch_workspace_bytes(p, 1); }
 
-size_t cvlc_encode_workspace_bytes(const cvlc_params* p) { return params_ok(p) ? enc_layout(p->d).total : 0; }
+size_t cvlc_plan_batch_workspace_bytes(const cvlc_params* p, uint32_t n) {
+  if (!params_ok(p) || n == 0 || n > CVLC_MAX_BATCH) return 0;
+  return plan_ws_bytes(n);
+}
+
+size_t cvlc_encode_workspace_bytes(const cvlc_params* p) { return cvlc_encode_batch_workspace_bytes(p, 1, 0); }
+
+size_t cvlc_encode_batch_workspace_bytes(const cvlc_params* p, uint32_t n, uint64_t max_candidates) {
+  if (!params_ok(p) || n == 0 || n > CVLC_MAX_BATCH) return 0;
+  const uint64_t cap = (max_candidates == 0 || max_candidates > p->d) ? p->d : max_candidates;
+  return enc_layout(p->d, n, cap).total;
+}
 
 size_t cvlc_decode_workspace_bytes(uint32_t n_clients) {
   if (n_clients == 0 || n_clients > CVLC_MAX_CLIENTS_PER_CALL) return 0;
   return dec_ws_bytes(n_clients);
 }
 
-static int plan_common(const float* x_dev, const cvlc_params* p, uint32_t fixed_y, cvlc_plan_t* plan_dev, void* ws_dev,
-                       size_t ws_bytes, void* cuda_stream) {
-  PlanTables T;
-  const int rc = build_tables(p, fixed_y, &T);
-  if (rc != CVLC_OK) return rc;
-  if (!aligned(x_dev, 16) || !aligned(plan_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
-  if (ws_bytes < kPlanWsBytes) return CVLC_ERR_WORKSPACE_TOO_SMALL;
-  return launch_plan(x_dev, T, plan_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
-                                                                                                        : CVLC_ERR_CUDA;
+int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint32_t fixed_y,
+                    cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!x_dev || !params || n == 0 || n > CVLC_MAX_BATCH || fixed_y > CVLC_MAX_CODE_BITS) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  for (uint32_t i = 0; i < n; ++i) {
+    Shape Si;
+    const int rc = build_shape(&params[i], fixed_y, i == 0 ? &S : &Si);
+    if (rc != CVLC_OK) return rc;
+    if (i && !same_shape(params[0], params[i])) return CVLC_ERR_INVALID_ARG;
+    if (!aligned(x_dev[i], 16)) return CVLC_ERR_INVALID_ARG;
+    desc[i].x = x_dev[i];
+    desc[i].plan = plans_dev + i;
+    desc[i].stream = nullptr;
+    desc[i].seed = params[i].seed;
+    desc[i].scale_B = params[i].scale_B;
+    desc[i].client_id = params[i].client_id;
+    desc[i].round = params[i].round;
+  }
+  if (!aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (ws_bytes < plan_ws_bytes(n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  return launch_plan(desc, n, S, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
 int cvlc_plan(const float* x_dev, const cvlc_params* p, cvlc_plan_t* plan_dev, void* ws_dev, size_t ws_bytes,
               void* cuda_stream) {
-  return plan_common(x_dev, p, 0, plan_dev, ws_dev, ws_bytes, cuda_stream);
+  return cvlc_plan_batch(&x_dev, p, 1, 0, plan_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
 int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_plan_t* plan_dev, void* ws_dev,
                     size_t ws_bytes, void* cuda_stream) {
   if (y < 1 || y > CVLC_MAX_CODE_BITS) return CVLC_ERR_INVALID_ARG;
-  return plan_common(x_dev, p, y, plan_dev, ws_dev, ws_bytes, cuda_stream);
+  return cvlc_plan_batch(&x_dev, p, 1, y, plan_dev, ws_dev, ws_bytes, cuda_stream);
+}
+
+int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                      uint8_t* const* streams_dev, size_t stream_capacity, uint64_t max_candidates, void* ws_dev,
+                      size_t ws_bytes, void* cuda_stream) {
+  if (!x_dev || !params || !streams_dev || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  for (uint32_t i = 0; i < n; ++i) {
+    Derived D;
+    const int rc = derive(&params[i], &D);
+    if (rc != CVLC_OK) return rc;
+    if (i && !same_shape(params[0], params[i])) return CVLC_ERR_INVALID_ARG;
+    if (!aligned(x_dev[i], 16) || !aligned(streams_dev[i], 16)) return CVLC_ERR_INVALID_ARG;
+    if (i == 0) {
+      memset(&S, 0, sizeof S);
+      S.d = params[0].d;
+      S.s = D.s;
+      S.R = D.R;
+      S.packet_bits = params[0].packet_bits;
+      S.header_bits = params[0].header_bits;
+      S.quantizer = params[0].quantizer;
+      S.max_code_bits = params[0].max_code_bits;
+      for (uint32_t y = 0; y <= CVLC_MAX_CODE_BITS; ++y) S.cap[y] = D.cap[y];
+    }
+    desc[i].x = x_dev[i];
+    desc[i].plan = const_cast<cvlc_plan_t*>(plans_dev) + i;
+    desc[i].stream = streams_dev[i];
+    desc[i].seed = params[i].seed;
+    desc[i].scale_B = params[i].scale_B;
+    desc[i].client_id = params[i].client_id;
+    desc[i].round = params[i].round;
+  }
+  if (!aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
+  const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
+  if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if ((size_t)S.cap[1] * 8 > 200 * 1024) return CVLC_ERR_INVALID_ARG;  // a packet's records are staged in shared memory
+  if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
+  return launch_encode(desc, n, S, cap, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
+                                                                                                       : CVLC_ERR_CUDA;
 }
 
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, uint8_t* stream_dev,
                 size_t stream_capacity, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
-  Derived D;
-  const int rc = derive(p, &D);
-  if (rc != CVLC_OK) return rc;
-  if (!aligned(x_dev, 16) || !aligned(plan_dev, 8) || !aligned(stream_dev, 16) || !aligned(ws_dev, 256))
-    return CVLC_ERR_INVALID_ARG;
-  if (stream_capacity < cvlc_stream_bytes(p)) return CVLC_ERR_OUTPUT_TOO_SMALL;
-  if (ws_bytes < enc_layout(p->d).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
-  const uint32_t max_cap = D.cap[1];
-  if ((size_t)max_cap * 8 > 200 * 1024) return CVLC_ERR_INVALID_ARG;  // a packet's records are staged in shared memory
-  return launch_encode(x_dev, *p, D.s, D.R, max_cap, plan_dev, stream_dev, ws_dev,
-                       static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
-             ? CVLC_OK
-             : CVLC_ERR_CUDA;
+  return cvlc_encode_batch(&x_dev, p, 1, plan_dev, &stream_dev, stream_capacity, 0, ws_dev, ws_bytes, cuda_stream);
 }
 
 int cvlc_decode_aggregate(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev, const float* weights_dev,

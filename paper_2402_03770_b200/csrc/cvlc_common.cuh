@@ -11,44 +11,6 @@ namespace cvlc {
 
 constexpr int kNumSM = 148;  // B200: grids are sized in multiples of this
 
-// ---- workspace layouts (byte offsets; every region 256-byte aligned) ----------
-
-// plan workspace
-constexpr size_t kPlanWsStatus = 0;      // int32 status, uint32 nonfinite flag at +4
-constexpr size_t kPlanWsHist = 256;      // uint64[4096]
-constexpr size_t kPlanWsBytes = kPlanWsHist + CVLC_HIST_BINS * 8;
-
-// encode workspace header (first 256 bytes), all zeroed at the start of a call
-struct EncHeader {
-  int32_t status;            // byte 0
-  uint32_t pad0;
-  uint32_t select_ticket;    // tile tickets of the selection kernel
-  uint32_t sort_ticket[4];   // tile tickets of the four digit passes
-  uint32_t pad1;
-  unsigned long long n_selected;  // candidates written by the selection kernel
-};
-constexpr size_t kEncWsSortHist = 256;                 // uint64[4][256] digit histograms
-constexpr size_t kEncWsSelectState = 256 + 4 * 256 * 8;  // uint64[n_select_tiles]
-
-constexpr int kSelectThreads = 256;
-constexpr int kSelectVecPerThread = 4;                       // float4 loads per thread per tile
-constexpr int kSelectTile = kSelectThreads * kSelectVecPerThread * 4;  // 4096 coordinates
-
-constexpr int kSortThreads = 256;
-constexpr int kSortItemsPerThread = 8;
-constexpr int kSortTile = kSortThreads * kSortItemsPerThread;  // 2048 pairs
-constexpr int kSortPasses = 4;                                 // digits of 8,8,8,7 bits
-
-struct EncLayout {
-  uint64_t n_select_tiles;
-  uint64_t max_sort_tiles;
-  size_t off_select_state;
-  size_t off_sort_state;   // uint64[4][max_sort_tiles][256]
-  size_t off_buf_a;        // uint64[d]
-  size_t off_buf_b;        // uint64[d]
-  size_t total;
-};
-
 #ifdef __CUDACC__
 #define CVLC_HD __host__ __device__
 #else
@@ -57,15 +19,98 @@ struct EncLayout {
 
 CVLC_HD constexpr size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-static inline EncLayout enc_layout(uint64_t d) {
+// ---- a batch of clients -------------------------------------------------------------
+// Every kernel of the plan / encode path works on a batch of clients that share the problem
+// shape (d, budget, packet and header size, candidate lengths) and differ in their update,
+// scale and Philox identifiers.  The per-client descriptors travel as a kernel parameter
+// (no host-to-device copy, no device-side table to keep alive); kernels are instantiated
+// for a small and a large descriptor capacity.
+
+struct ClientDesc {
+  const float* x;      // the update, d fp32
+  cvlc_plan_t* plan;   // written by the plan kernels, read by the encode kernels
+  uint8_t* stream;     // encode output (unused while planning)
+  uint64_t seed;       // Philox key
+  double scale_B;      // B of the scaling operation
+  uint32_t client_id;  // Philox counter word 2
+  uint32_t round;      // Philox counter word 3
+};
+
+constexpr int kSmallBatch = 4;
+constexpr int kLargeBatch = CVLC_MAX_BATCH;
+
+template <int CAP>
+struct BatchDesc {
+  uint32_t n;
+  uint32_t pad;
+  ClientDesc c[CAP];
+};
+
+struct Shape {
+  uint64_t d;
+  uint32_t s, R;
+  uint32_t packet_bits, header_bits, quantizer, max_code_bits;
+  uint32_t fixed_y;  // 0 = tune the lengths; otherwise every packet at this length
+  uint32_t pad;
+  uint32_t cap[CVLC_MAX_CODE_BITS + 1];  // records per packet per code length
+};
+
+// ---- workspace layouts (byte offsets; every region 256-byte aligned) ----------
+
+// plan workspace: [0] int32 status | [256] uint64 hist[n][4096] | uint32 nonfinite[n]
+constexpr size_t kPlanWsHist = 256;
+CVLC_HD constexpr size_t plan_off_flags(uint32_t n) { return kPlanWsHist + (size_t)n * CVLC_HIST_BINS * 8; }
+CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n) { return align256(plan_off_flags(n) + (size_t)n * 4); }
+
+// encode workspace header (first 256 bytes), zeroed at the start of a call
+struct EncHeader {
+  int32_t status;           // byte 0
+  uint32_t select_ticket;   // tile tickets of the selection kernel
+  uint32_t sort_ticket[4];  // tile tickets of the four digit passes
+  uint32_t total_sort_tiles;
+};
+
+constexpr int kSelectThreads = 512;
+constexpr int kSelectVecPerThread = 4;                                 // float4 loads per thread per tile
+constexpr int kSelectTile = kSelectThreads * kSelectVecPerThread * 4;  // 8192 coordinates
+
+constexpr int kSortThreads = 256;
+constexpr int kSortItemsPerThread = 8;
+constexpr int kSortTile = kSortThreads * kSortItemsPerThread;  // 2048 pairs
+constexpr int kSortPasses = 4;                                 // digits of 8,8,8,7 bits
+
+struct EncLayout {
+  uint32_t n;
+  uint64_t capacity;             // candidate slots per client
+  uint64_t select_tiles;         // per client
+  uint64_t sort_tiles_max;       // per client
+  size_t off_n_selected;         // uint64[n]
+  size_t off_sort_prefix;        // uint32[n + 1]: first sort tile of every client
+  size_t off_pass_mask;          // uint32[n]: digit passes that are constant for the client
+  size_t off_ghist;              // uint64[n][4][256] digit histograms
+  size_t off_gbase;              // uint64[n][4][256] their exclusive scans
+  size_t off_select_state;       // uint64[n][select_tiles]
+  size_t off_sort_state;         // uint64[4][n * sort_tiles_max][256]
+  size_t off_buf_a, off_buf_b;   // uint64[n][capacity]
+  size_t total;
+};
+
+static inline EncLayout enc_layout(uint64_t d, uint32_t n, uint64_t capacity) {
   EncLayout L;
-  L.n_select_tiles = (d + kSelectTile - 1) / kSelectTile;
-  L.max_sort_tiles = (d + kSortTile - 1) / kSortTile;
-  L.off_select_state = kEncWsSelectState;
-  L.off_sort_state = align256(L.off_select_state + L.n_select_tiles * 8);
-  L.off_buf_a = align256(L.off_sort_state + (size_t)kSortPasses * L.max_sort_tiles * 256 * 8);
-  L.off_buf_b = align256(L.off_buf_a + d * 8);
-  L.total = align256(L.off_buf_b + d * 8);
+  L.n = n;
+  L.capacity = capacity;
+  L.select_tiles = (d + kSelectTile - 1) / kSelectTile;
+  L.sort_tiles_max = (capacity + kSortTile - 1) / kSortTile;
+  L.off_n_selected = 256;
+  L.off_sort_prefix = align256(L.off_n_selected + (size_t)n * 8);
+  L.off_pass_mask = align256(L.off_sort_prefix + ((size_t)n + 1) * 4);
+  L.off_ghist = align256(L.off_pass_mask + (size_t)n * 4);
+  L.off_gbase = align256(L.off_ghist + (size_t)n * kSortPasses * 256 * 8);
+  L.off_select_state = align256(L.off_gbase + (size_t)n * kSortPasses * 256 * 8);
+  L.off_sort_state = align256(L.off_select_state + (size_t)n * L.select_tiles * 8);
+  L.off_buf_a = align256(L.off_sort_state + (size_t)kSortPasses * n * L.sort_tiles_max * 256 * 8);
+  L.off_buf_b = align256(L.off_buf_a + (size_t)n * capacity * 8);
+  L.total = align256(L.off_buf_b + (size_t)n * capacity * 8);
   return L;
 }
 
@@ -78,27 +123,11 @@ CVLC_HD constexpr size_t dec_off_meta(uint32_t n) { return align256(dec_off_pref
 // per client: packet_bits, header_bits (uint32 each)
 CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta(n) + (size_t)n * 8); }
 
-// ---- host-side tables handed to the planning kernel -----------------------------
-
-struct PlanTables {
-  uint64_t d;
-  uint32_t s, R;
-  uint32_t nY;                               // candidate lengths
-  uint32_t y_min;
-  uint32_t fixed_y;                          // 0 = tune; otherwise every packet at this length
-  uint32_t pad;
-  uint32_t Y[CVLC_MAX_CODE_BITS];            // candidate lengths, ascending
-  uint32_t capY[CVLC_MAX_CODE_BITS];         // cap(Y[i])
-  double gY[CVLC_MAX_CODE_BITS];             // coefficient g(Y[i]) of Eq. (5)
-  double QY[CVLC_MAX_CODE_BITS];             // PQ error factor Q(Y[i])
-  uint32_t cap[CVLC_MAX_CODE_BITS + 1];      // cap(y) for every y
-};
-
 // ---- launch accounting and optional per-kernel timing ------------------------------
 
 enum KernelId {
-  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSortHist, kKSortPass, kKPack, kKDecodePrepare,
-  kKFillZero, kKDecode, kKSelftest, kNumKernelIds
+  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSortHist, kKSortScan, kKSortPass, kKPack,
+  kKDecodePrepare, kKFillZero, kKDecode, kKSelftest, kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -115,9 +144,9 @@ struct LaunchScope {
 
 // ---- launchers (one per translation unit) ---------------------------------------
 
-cudaError_t launch_plan(const float* x, const PlanTables& T, cvlc_plan_t* plan, void* ws, cudaStream_t st);
-cudaError_t launch_encode(const float* x, const cvlc_params& p, uint32_t s, uint32_t R, uint32_t max_cap,
-                          const cvlc_plan_t* plan, uint8_t* stream, void* ws, cudaStream_t st);
+cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
+cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
+                          cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
                           void* ws, cudaStream_t st);

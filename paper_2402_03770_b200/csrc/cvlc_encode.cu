@@ -1,6 +1,6 @@
-// Encoding kernels (Algorithm 1, steps 15-17): top-k candidate selection by the
-// plan's histogram threshold, stable LSD radix ranking of the candidates by |x|,
-// per-packet minimum/maximum, PQ stochastic quantization with Philox4x32-10 and
+// Encoding kernels (Algorithm 1, steps 15-17), batched over clients: top-k candidate
+// selection by the plan's histogram threshold, stable LSD radix ranking of the candidates
+// by |x|, per-packet minimum/maximum, PQ stochastic quantization with Philox4x32-10 and
 // bit packing of (position ID, centroid ID) pairs into fixed-size packets (Fig. 2).
 #include "cvlc_common.cuh"
 
@@ -37,39 +37,78 @@ __device__ __forceinline__ unsigned long long wait_state(const unsigned long lon
   return v;
 }
 
-// ===================================================================================
-// K0  workspace reset + plan validation
-// ===================================================================================
+__device__ __forceinline__ uint32_t sort_tiles_of(unsigned long long n_candidates, unsigned long long capacity) {
+  const unsigned long long nc = n_candidates < capacity ? n_candidates : capacity;
+  return (uint32_t)((nc + kSortTile - 1) / kSortTile);
+}
 
-__global__ void k_encode_init(unsigned char* ws, const cvlc_plan_t* __restrict__ plan, EncLayout L, uint64_t d,
-                              uint32_t s, uint32_t R) {
+// ===================================================================================
+// K0  workspace reset, plan validation, sort-tile prefix over the clients
+// ===================================================================================
+// The grid zeroes the per-client counters, digit histograms and look-back states; block 0
+// alone owns the 256-byte header and the sort-tile prefix (nobody else writes them).
+
+template <int CAP>
+__global__ void __launch_bounds__(256)
+k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
+              const __grid_constant__ EncLayout L) {
+  __shared__ unsigned long long s_total;
+  __shared__ int s_bad;
+  const uint32_t n = batch.n;
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+    for (uint32_t c = 0; c < n; ++c) t += sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
+    s_total = t;
+    s_bad = 0;
+  }
+  __syncthreads();
   const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t gstride = (size_t)gridDim.x * blockDim.x;
-  unsigned long long* w64 = reinterpret_cast<unsigned long long*>(ws);
-  const size_t n_head = L.off_sort_state / 8;  // header, digit histograms, selection tile states
-  for (size_t i = gtid; i < n_head; i += gstride) w64[i] = 0ull;
-  unsigned long long nc = plan->n_candidates;
-  if (nc > d) nc = d;
-  const size_t tiles = (size_t)((nc + kSortTile - 1) / kSortTile);
-  const size_t per_pass = tiles * 256;
+  {
+    unsigned long long* a = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
+    for (size_t i = gtid; i < n; i += gstride) a[i] = 0ull;
+    unsigned long long* b = reinterpret_cast<unsigned long long*>(ws + L.off_ghist);
+    const size_t nb = (L.off_sort_state - L.off_ghist) / 8;  // digit histograms, their scans, selection tile states
+    for (size_t i = gtid; i < nb; i += gstride) b[i] = 0ull;
+  }
+  const size_t per_pass = (size_t)s_total * 256;
   for (int p = 0; p < kSortPasses; ++p) {
-    unsigned long long* st = reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)p * L.max_sort_tiles * 256;
+    unsigned long long* st = reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)p * n * L.sort_tiles_max * 256;
     for (size_t i = gtid; i < per_pass; i += gstride) st[i] = 0ull;
   }
-  if (gtid == 0) {
-    // the plan must belong to these parameters (status is written after the zeroing above
-    // by the same thread, so it survives)
-    int32_t bad = 0;
-    if (plan->status != CVLC_OK) bad = plan->status;
+  if (blockIdx.x != 0) return;
+
+  EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
+  uint32_t* prefix = reinterpret_cast<uint32_t*>(ws + L.off_sort_prefix);
+  for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+    const cvlc_plan_t* plan = batch.c[c].plan;
     unsigned long long k = 0, nsum = 0;
     for (int y = 1; y <= CVLC_MAX_CODE_BITS; ++y) {
       k += (unsigned long long)plan->n_y[y] * plan->cap[y];
       nsum += plan->n_y[y];
     }
-    if (!bad && (plan->s != s || plan->R != R || nsum != R || k != plan->k || k == 0 || k > plan->n_candidates ||
-                 plan->n_candidates > d || plan->thresh_bin >= CVLC_HIST_BINS))
+    int bad = 0;
+    if (plan->status != CVLC_OK)
+      bad = plan->status;
+    else if (plan->s != shape.s || plan->R != shape.R || nsum != shape.R || k != plan->k || k == 0 ||
+             k > plan->n_candidates || plan->n_candidates > shape.d || plan->thresh_bin >= CVLC_HIST_BINS)
       bad = CVLC_ERR_PLAN_MISMATCH;
-    if (bad) reinterpret_cast<EncHeader*>(ws)->status = bad;
+    else if (plan->n_candidates > L.capacity)
+      bad = CVLC_ERR_WORKSPACE_TOO_SMALL;
+    if (bad) atomicCAS(&s_bad, 0, bad);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t run = 0;
+    for (uint32_t c = 0; c < n; ++c) {
+      prefix[c] = run;
+      run += sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
+    }
+    prefix[n] = run;
+    hdr->status = s_bad;
+    hdr->select_ticket = 0;
+    for (int p = 0; p < kSortPasses; ++p) hdr->sort_ticket[p] = 0;
+    hdr->total_sort_tiles = run;
   }
 }
 
@@ -78,23 +117,36 @@ __global__ void k_encode_init(unsigned char* ws, const cvlc_plan_t* __restrict__
 // ===================================================================================
 // Emits (key << 32 | sign << 31 | index) for every coordinate whose histogram bin is at or
 // above the plan's threshold bin, in ascending index order.  4 bytes read per coordinate.
+// Tiles of 8192 coordinates are handed out by an atomic ticket (client-major), so every
+// predecessor of a tile is running or done; the look-back reads 512 predecessors per step.
 
+template <int CAP>
 __global__ void __launch_bounds__(kSelectThreads)
-k_select(const float* __restrict__ x, uint64_t d, const cvlc_plan_t* __restrict__ plan, EncHeader* hdr,
-         unsigned long long* tile_state, uint64_t n_tiles, unsigned long long* __restrict__ out, uint64_t out_capacity) {
+k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ uint32_t s_tile;
   __shared__ unsigned long long s_warp_incl[kSelectThreads / 32];
-  __shared__ unsigned long long s_tile_excl;
+  __shared__ unsigned long long s_look_sum[kSelectThreads / 32];
+  __shared__ uint32_t s_look_flag[kSelectThreads / 32];
+  EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t thresh = plan->thresh_bin << 19;
-  const float4* xv = reinterpret_cast<const float4*>(x);
+  const uint64_t tiles_per_client = L.select_tiles;
+  const uint64_t total_tiles = tiles_per_client * batch.n;
+  unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
 
   while (true) {
     if (tid == 0) s_tile = atomicAdd(&hdr->select_ticket, 1u);
     __syncthreads();
-    const uint64_t tile = s_tile;
-    if (tile >= n_tiles) break;
+    const uint64_t gt = s_tile;
+    if (gt >= total_tiles) break;
+    const uint32_t c = (uint32_t)(gt / tiles_per_client);
+    const uint64_t tile = gt - (uint64_t)c * tiles_per_client;
+    const float* __restrict__ x = batch.c[c].x;
+    const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
+    const float4* xv = reinterpret_cast<const float4*>(x);
+    const uint32_t thresh = plan->thresh_bin << 19;
+    unsigned long long* tile_state = reinterpret_cast<unsigned long long*>(ws + L.off_select_state) + (size_t)c * tiles_per_client;
+    unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     const uint64_t base_vec = tile * (uint64_t)(kSelectThreads * kSelectVecPerThread);
 
     uint32_t bits[kSelectVecPerThread][4];
@@ -113,20 +165,20 @@ k_select(const float* __restrict__ x, uint64_t d, const cvlc_plan_t* __restrict_
         valid = 0xF;
       } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          bits[v][c] = 0;
-          if (e0 + c < d) {
-            bits[v][c] = __float_as_uint(x[e0 + c]);
-            valid |= 1u << c;
+        for (int cc = 0; cc < 4; ++cc) {
+          bits[v][cc] = 0;
+          if (e0 + cc < d) {
+            bits[v][cc] = __float_as_uint(x[e0 + cc]);
+            valid |= 1u << cc;
           }
         }
       }
       uint32_t m = 0;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) m |= (((bits[v][c] & 0x7FFFFFFFu) >= thresh) ? 1u : 0u) << c;
+      for (int cc = 0; cc < 4; ++cc) m |= (((bits[v][cc] & 0x7FFFFFFFu) >= thresh) ? 1u : 0u) << cc;
       mask[v] = m & valid;
     }
-    // block scan of the four per-vector counts, packed 16 bits each (tile totals <= 1024)
+    // block scan of the four per-vector counts, packed 16 bits each (tile totals <= 2048)
     unsigned long long packed = 0;
 #pragma unroll
     for (int v = 0; v < kSelectVecPerThread; ++v) packed |= (unsigned long long)__popc(mask[v]) << (16 * v);
@@ -148,60 +200,68 @@ k_select(const float* __restrict__ x, uint64_t d, const cvlc_plan_t* __restrict_
     const unsigned long long excl = below + incl - packed;  // per-vector exclusive counts over threads
     const uint32_t tile_total = (uint32_t)((tot & 0xFFFF) + ((tot >> 16) & 0xFFFF) + ((tot >> 32) & 0xFFFF) + (tot >> 48));
 
-    // decoupled look-back over the preceding tiles (warp 0, 32 tiles per step)
-    if (warp == 0) {
-      if (lane == 0) st_relaxed(tile_state + tile, (tile == 0 ? kFlagPrefix : kFlagAgg) | tile_total);
-      unsigned long long run = 0;
-      if (tile > 0) {
-        long long base = (long long)tile - 1;
-        while (true) {
-          const long long idx = base - lane;
-          unsigned long long sv = kFlagPrefix;  // before tile 0: empty prefix
-          if (idx >= 0) sv = wait_state(tile_state + idx, &hdr->status);
-          const unsigned timed_out = __ballot_sync(kFull, sv == 0);
-          const unsigned is_prefix = __ballot_sync(kFull, (sv & kFlagMask) == kFlagPrefix);
-          if (timed_out) break;
-          unsigned long long val = sv & kValMask;
-          if (is_prefix) {
-            const int firstp = __ffs(is_prefix) - 1;
-            if (lane > firstp) val = 0;
-          }
+    // decoupled look-back: thread i inspects predecessor (tile - 1 - i) of this client
+    if (tid == 0) st_relaxed(tile_state + tile, (tile == 0 ? kFlagPrefix : kFlagAgg) | tile_total);
+    unsigned long long run = 0;
+    if (tile > 0) {
+      long long base = (long long)tile - 1;
+      while (true) {
+        const long long idx = base - tid;
+        unsigned long long sv = kFlagPrefix;  // before tile 0: empty prefix
+        if (idx >= 0) sv = wait_state(tile_state + idx, &hdr->status);
+        const bool to = (sv == 0);
+        const unsigned is_prefix = __ballot_sync(kFull, (sv & kFlagMask) == kFlagPrefix);
+        unsigned long long val = sv & kValMask;
+        if (is_prefix) {
+          const int firstp = __ffs(is_prefix) - 1;
+          if (lane > firstp) val = 0;
+        }
 #pragma unroll
-          for (int off = 16; off > 0; off >>= 1) val += __shfl_xor_sync(kFull, val, off);
-          run += val;
-          if (is_prefix) break;
-          base -= 32;
+        for (int off = 16; off > 0; off >>= 1) val += __shfl_xor_sync(kFull, val, off);
+        if (lane == 0) {
+          s_look_sum[warp] = val;
+          s_look_flag[warp] = is_prefix ? 1u : 0u;
         }
-        if (lane == 0) st_relaxed(tile_state + tile, kFlagPrefix | (run + tile_total));
-      }
-      if (lane == 0) {
-        s_tile_excl = run;
-        if (tile == n_tiles - 1) {
-          hdr->n_selected = run + tile_total;
-          if (run + tile_total != plan->n_candidates) set_status(&hdr->status, CVLC_ERR_PLAN_MISMATCH);
+        const int any_to = __syncthreads_or(to);
+        // the nearest warp (smallest distance) that saw a prefix ends the walk
+        bool found = false;
+        unsigned long long add = 0;
+#pragma unroll
+        for (int w = 0; w < kSelectThreads / 32; ++w) {
+          if (!found) {
+            add += s_look_sum[w];
+            found = s_look_flag[w] != 0;
+          }
         }
+        run += add;
+        __syncthreads();
+        if (any_to || found) break;  // after a timeout the status is set and the results are void
+        base -= kSelectThreads;
       }
+      if (tid == 0) st_relaxed(tile_state + tile, kFlagPrefix | (run + tile_total));
     }
-    __syncthreads();
-    unsigned long long pos = s_tile_excl;
+    if (tid == 0 && tile == tiles_per_client - 1) {
+      n_selected[c] = run + tile_total;
+      if (run + tile_total != plan->n_candidates) set_status(&hdr->status, CVLC_ERR_PLAN_MISMATCH);
+    }
     unsigned long long vec_base = 0;
 #pragma unroll
     for (int v = 0; v < kSelectVecPerThread; ++v) {
-      unsigned long long o = pos + vec_base + ((excl >> (16 * v)) & 0xFFFF);
+      unsigned long long o = run + vec_base + ((excl >> (16 * v)) & 0xFFFF);
       const uint64_t e0 = (base_vec + (uint64_t)v * kSelectThreads + tid) * 4;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        if (mask[v] & (1u << c)) {
-          const uint32_t b = bits[v][c];
+      for (int cc = 0; cc < 4; ++cc) {
+        if (mask[v] & (1u << cc)) {
+          const uint32_t b = bits[v][cc];
           const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) |
-                                          (unsigned long long)(e0 + c);
-          if (o < out_capacity) out[o] = pair;
+                                          (unsigned long long)(e0 + cc);
+          if (o < L.capacity) out[o] = pair;
           ++o;
         }
       }
       vec_base += (tot >> (16 * v)) & 0xFFFF;
     }
-    __syncthreads();  // s_tile / s_tile_excl are reused by the next tile
+    __syncthreads();  // s_tile and the look-back scratch are reused by the next tile
   }
 }
 
@@ -209,73 +269,76 @@ k_select(const float* __restrict__ x, uint64_t d, const cvlc_plan_t* __restrict_
 // K4  stable LSD radix ranking of the candidates, |x| descending (ties keep ascending index)
 // ===================================================================================
 // Key digit = digit of (0x7FFFFFFF - key): 8, 8, 8, 7 bits.  One histogram kernel for all
-// four digits, then one single-pass kernel per digit (decoupled look-back per digit value).
-// A pass whose digit is the same for every candidate is skipped; which buffer holds the
-// data after pass q therefore follows from the digit histograms alone.
+// four digits and all clients, a small scan kernel, then one single-pass kernel per digit
+// (tiles of all clients handed out by ticket, decoupled look-back per digit value).  A pass
+// whose digit is the same for every candidate of a client is skipped for that client; which
+// buffer holds its data after pass q follows from the mask of skipped passes.
 
 __device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass) {
   const uint32_t inv = 0x7FFFFFFFu - (uint32_t)(pair >> 32);
   return (inv >> (8 * pass)) & 0xFFu;
 }
 
+// The clients' candidate arrays are concatenated in units of sort tiles (2048 pairs) and cut
+// into equal contiguous chunks, one per block; a block that crosses a client boundary merges
+// its shared histograms into that client's and starts afresh.
+template <int CAP>
 __global__ void __launch_bounds__(256)
-k_sort_hist(const unsigned long long* __restrict__ in, const cvlc_plan_t* __restrict__ plan, const EncHeader* hdr,
-            unsigned long long* __restrict__ ghist) {
+k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ uint32_t sh[kSortPasses * 256];
+  const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
+  const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + L.off_sort_prefix);
+  unsigned long long* ghist_all = reinterpret_cast<unsigned long long*>(ws + L.off_ghist);
   for (int i = threadIdx.x; i < kSortPasses * 256; i += 256) sh[i] = 0;
   __syncthreads();
-  const unsigned long long n = plan->n_candidates;
-  for (unsigned long long i = (unsigned long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (unsigned long long)gridDim.x * 256) {
-    const unsigned long long pair = in[i];
+  const uint32_t total_tiles = prefix[batch.n];
+  const uint32_t chunk = (total_tiles + gridDim.x - 1) / gridDim.x;
+  uint32_t t = blockIdx.x * chunk;
+  const uint32_t t_end = (t + chunk < total_tiles) ? t + chunk : total_tiles;
+  uint32_t c = 0;
+  while (t < t_end) {
+    while (prefix[c + 1] <= t) ++c;  // client of tile t (clients without tiles are passed over)
+    const uint32_t seg_end = prefix[c + 1] < t_end ? prefix[c + 1] : t_end;
+    const unsigned long long n = batch.c[c].plan->n_candidates;
+    const unsigned long long* __restrict__ in = reinterpret_cast<const unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
+    const unsigned long long i0 = (unsigned long long)(t - prefix[c]) * kSortTile;
+    unsigned long long i1 = (unsigned long long)(seg_end - prefix[c]) * kSortTile;
+    if (i1 > n) i1 = n;
+    for (unsigned long long i = i0 + threadIdx.x; i < i1; i += 256) {
+      const unsigned long long pair = in[i];
 #pragma unroll
-    for (int p = 0; p < kSortPasses; ++p) atomicAdd(&sh[p * 256 + sort_digit(pair, p)], 1u);
+      for (int p = 0; p < kSortPasses; ++p) atomicAdd(&sh[p * 256 + sort_digit(pair, p)], 1u);
+    }
+    __syncthreads();
+    unsigned long long* ghist = ghist_all + (size_t)c * kSortPasses * 256;
+    for (int i = threadIdx.x; i < kSortPasses * 256; i += 256) {
+      const uint32_t v = sh[i];
+      sh[i] = 0;
+      if (v) atomicAdd(ghist + i, (unsigned long long)v);
+    }
+    __syncthreads();
+    t = seg_end;
   }
-  __syncthreads();
-  for (int i = threadIdx.x; i < kSortPasses * 256; i += 256)
-    if (sh[i]) atomicAdd(ghist + i, (unsigned long long)sh[i]);
 }
 
-// number of passes before `pass` that moved data, and whether `pass` itself is skipped
-__device__ __forceinline__ void sort_pass_parity(const unsigned long long* ghist, unsigned long long n, int pass, int* flips,
-                                                 bool* skip) {
-  int f = 0;
-  bool sk = false;
-  for (int q = 0; q <= pass; ++q) {
-    int hit = 0;
-    for (int b = threadIdx.x; b < 256; b += blockDim.x) hit |= (ghist[q * 256 + b] == n);
-    const int trivial = __syncthreads_or(hit);
-    if (q < pass)
-      f += trivial ? 0 : 1;
-    else
-      sk = trivial != 0;
-  }
-  *flips = f;
-  *skip = sk;
-}
-
-__global__ void __launch_bounds__(kSortThreads)
-k_sort_pass(int pass, unsigned long long* buf_a, unsigned long long* buf_b, const cvlc_plan_t* __restrict__ plan, EncHeader* hdr,
-            const unsigned long long* __restrict__ ghist, unsigned long long* state /* [tiles][256] */) {
-  __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_wc[kSortThreads / 32][256];  // per-warp digit counters -> per-warp offsets
-  __shared__ unsigned long long s_base[256];         // global position of this tile's first item per digit
-  __shared__ unsigned long long s_scan[256];
+// per client: exclusive scans of the four digit histograms and the mask of constant digits
+template <int CAP>
+__global__ void __launch_bounds__(256)
+k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
+  __shared__ unsigned long long s_scan[8];
+  const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
+  const uint32_t c = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const unsigned long long n = plan->n_candidates;
-  const unsigned long long n_tiles = (n + kSortTile - 1) / kSortTile;
-  int flips;
-  bool skip;
-  sort_pass_parity(ghist, n, pass, &flips, &skip);
-  if (skip) return;
-  const unsigned long long* src = (flips & 1) ? buf_b : buf_a;
-  unsigned long long* dst = (flips & 1) ? buf_a : buf_b;
-
-  // exclusive scan of this digit's histogram: first position of every digit value
-  {
-    const unsigned long long c = ghist[pass * 256 + tid];
-    unsigned long long incl = c;
+  const unsigned long long n = batch.c[c].plan->n_candidates;
+  const unsigned long long* ghist = reinterpret_cast<const unsigned long long*>(ws + L.off_ghist) + (size_t)c * kSortPasses * 256;
+  unsigned long long* gbase = reinterpret_cast<unsigned long long*>(ws + L.off_gbase) + (size_t)c * kSortPasses * 256;
+  uint32_t mask = 0;
+  for (int p = 0; p < kSortPasses; ++p) {
+    const unsigned long long cnt = ghist[p * 256 + tid];
+    if (__syncthreads_or(cnt == n)) mask |= 1u << p;
+    unsigned long long incl = cnt;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
       const unsigned long long o = __shfl_up_sync(kFull, incl, off);
@@ -285,19 +348,63 @@ k_sort_pass(int pass, unsigned long long* buf_a, unsigned long long* buf_b, cons
     __syncthreads();
     unsigned long long below = 0;
     for (int w = 0; w < warp; ++w) below += s_scan[w];
+    gbase[p * 256 + tid] = below + incl - cnt;
     __syncthreads();
-    s_scan[tid] = below + incl - c;
+  }
+  if (tid == 0) reinterpret_cast<uint32_t*>(ws + L.off_pass_mask)[c] = mask;
+}
+
+template <int CAP>
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
+  __shared__ uint32_t s_tile;
+  __shared__ uint32_t s_wc[kSortThreads / 32][256];  // per-warp digit counters -> per-warp offsets
+  __shared__ unsigned long long s_base[256];         // position of this tile's first item per digit
+  extern __shared__ uint32_t s_prefix[];             // [n + 1] first sort tile of every client
+  EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
+  if (hdr->status != 0) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t n_clients = batch.n;
+  {
+    const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + L.off_sort_prefix);
+    for (uint32_t i = tid; i <= n_clients; i += kSortThreads) s_prefix[i] = prefix[i];
   }
   __syncthreads();
-  const unsigned long long gbase = s_scan[tid];
+  const uint32_t total_tiles = s_prefix[n_clients];
+  const uint32_t* pass_mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask);
+  unsigned long long* state_all =
+      reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)pass * n_clients * L.sort_tiles_max * 256;
   const unsigned lanemask_lt = (1u << lane) - 1u;
 
   while (true) {
     if (tid == 0) s_tile = atomicAdd(&hdr->sort_ticket[pass], 1u);
+#pragma unroll
     for (int w = 0; w < kSortThreads / 32; ++w) s_wc[w][tid] = 0;
     __syncthreads();
-    const unsigned long long tile = s_tile;
-    if (tile >= n_tiles) break;
+    const uint32_t gt = s_tile;
+    if (gt >= total_tiles) break;
+    // client of tile gt: last c with prefix[c] <= gt
+    uint32_t lo_c = 0, hi_c = n_clients;
+    while (hi_c - lo_c > 1) {
+      const uint32_t mid = (lo_c + hi_c) >> 1;
+      if (s_prefix[mid] <= gt) lo_c = mid; else hi_c = mid;
+    }
+    const uint32_t c = lo_c;
+    const uint32_t mask = pass_mask[c];
+    if (mask & (1u << pass)) {  // constant digit for this client: nothing to move
+      __syncthreads();          // everyone has read s_tile before the next ticket overwrites it
+      continue;
+    }
+    const unsigned long long tile = gt - s_prefix[c];
+    const unsigned long long n = batch.c[c].plan->n_candidates;
+    const int flips = __popc(~mask & ((1u << pass) - 1u));
+    unsigned long long* buf_a = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
+    unsigned long long* buf_b = reinterpret_cast<unsigned long long*>(ws + L.off_buf_b) + (size_t)c * L.capacity;
+    const unsigned long long* __restrict__ src = (flips & 1) ? buf_b : buf_a;
+    unsigned long long* __restrict__ dst = (flips & 1) ? buf_a : buf_b;
+    unsigned long long* state = state_all + (size_t)s_prefix[c] * 256;
+    const unsigned long long gbase =
+        reinterpret_cast<const unsigned long long*>(ws + L.off_gbase)[(size_t)c * kSortPasses * 256 + pass * 256 + tid];
 
     unsigned long long item[kSortItemsPerThread];
     uint32_t rank[kSortItemsPerThread];
@@ -327,9 +434,9 @@ k_sort_pass(int pass, unsigned long long* buf_a, unsigned long long* buf_b, cons
       uint32_t tot = 0;
 #pragma unroll
       for (int w = 0; w < kSortThreads / 32; ++w) {
-        const uint32_t c = s_wc[w][tid];
+        const uint32_t cnt = s_wc[w][tid];
         s_wc[w][tid] = tot;
-        tot += c;
+        tot += cnt;
       }
       unsigned long long* my_state = state + tile * 256 + tid;
       st_relaxed(my_state, (tile == 0 ? kFlagPrefix : kFlagAgg) | tot);
@@ -351,7 +458,7 @@ k_sort_pass(int pass, unsigned long long* buf_a, unsigned long long* buf_b, cons
       if ((first + i * 32 + lane) < n) {
         const uint32_t dig = sort_digit(item[i], pass);
         const unsigned long long o = s_base[dig] + s_wc[warp][dig] + rank[i];
-        if (o < n) dst[o] = item[i];
+        if (o < n && o < L.capacity) dst[o] = item[i];
       }
     }
     __syncthreads();
@@ -361,27 +468,30 @@ k_sort_pass(int pass, unsigned long long* buf_a, unsigned long long* buf_b, cons
 // ===================================================================================
 // K5  per-packet min/max, PQ stochastic quantization, bit packing
 // ===================================================================================
-// One CTA per packet.  Packet r (longest codes first) holds ranks [Z, Z + cap(y_r)).
+// One CTA per (packet, client).  Packet r (longest codes first) holds ranks [Z, Z + cap(y_r)).
 
 constexpr int kPackThreads = 128;
 
+template <int CAP>
 __global__ void __launch_bounds__(kPackThreads)
-k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* __restrict__ buf_b,
-       const cvlc_plan_t* __restrict__ plan, const EncHeader* hdr, const unsigned long long* __restrict__ ghist,
-       const __grid_constant__ cvlc_params prm, uint32_t s, uint32_t R, uint32_t* __restrict__ stream_words) {
+k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
+       const __grid_constant__ EncLayout L) {
   extern __shared__ unsigned long long recs[];  // [cap(1)]
   __shared__ float s_red[2][kPackThreads / 32];
   __shared__ uint32_t s_y;
   __shared__ unsigned long long s_Z;
+  const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t r = blockIdx.x;
+  const uint32_t r = blockIdx.x, c = blockIdx.y;
+  const ClientDesc& cd = batch.c[c];
+  const cvlc_plan_t* __restrict__ plan = cd.plan;
+  const uint32_t s = shape.s;
 
-  int flips;
-  bool skip;
-  sort_pass_parity(ghist, plan->n_candidates, kSortPasses - 1, &flips, &skip);
-  if (!skip) flips += 1;
-  const unsigned long long* sorted = (flips & 1) ? buf_b : buf_a;
+  const uint32_t mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask)[c];
+  const int flips = __popc(~mask & ((1u << kSortPasses) - 1u));
+  const unsigned long long* __restrict__ sorted =
+      reinterpret_cast<const unsigned long long*>(ws + ((flips & 1) ? L.off_buf_b : L.off_buf_a)) + (size_t)c * L.capacity;
 
   if (tid == 0) {
     unsigned long long cum = 0, Z = 0;
@@ -435,7 +545,7 @@ k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* _
   }
 
   // stochastic rounding onto the 2^y uniform centroids of [lo, hi]
-  const double L = (double)((1ull << y) - 1ull);
+  const double Lc = (double)((1ull << y) - 1ull);
   const double dlo = (double)lo;
   const double den = __dsub_rn((double)hi, dlo);
   for (uint32_t j = tid; j < P; j += kPackThreads) {
@@ -445,11 +555,11 @@ k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* _
     const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;
     uint32_t code = 0;
     if (hi != lo) {
-      const double t = __dmul_rn(__ddiv_rn(__dsub_rn((double)__uint_as_float(b), dlo), den), L);
+      const double t = __dmul_rn(__ddiv_rn(__dsub_rn((double)__uint_as_float(b), dlo), den), Lc);
       double j0 = floor(t);
-      if (j0 > L) j0 = L;
+      if (j0 > Lc) j0 = Lc;
       const double frac = __dsub_rn(t, j0);
-      const double u = __dmul_rn((double)philox_coord(prm.seed, prm.client_id, prm.round, pid), 1.0 / 4294967296.0);
+      const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
       code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
     }
     recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
@@ -457,8 +567,9 @@ k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* _
   __syncthreads();
 
   // gather the packet's 32-bit words: header {s, y, lo, hi}, then records of wd bits from bit H
-  const uint32_t H = prm.header_bits;
-  const uint32_t n_words = prm.packet_bits / 32;
+  const uint32_t H = shape.header_bits;
+  const uint32_t n_words = shape.packet_bits / 32;
+  uint32_t* stream_words = reinterpret_cast<uint32_t*>(cd.stream);
   uint32_t* pkt = stream_words + CVLC_STREAM_HEADER_BYTES / 4 + (size_t)r * n_words;
   const uint32_t blo = __float_as_uint(lo), bhi = __float_as_uint(hi);
   const uint32_t payload_end = H + P * wd;
@@ -480,23 +591,23 @@ k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* _
     pkt[w] = val;
   }
 
-  // global header (64 bytes), written once
+  // global header (64 bytes), written once per client
   if (r == 0 && tid < 16) {
     uint32_t v = 0;
-    const unsigned long long Bbits = (unsigned long long)__double_as_longlong(prm.scale_B);
+    const unsigned long long Bbits = (unsigned long long)__double_as_longlong(cd.scale_B);
     const unsigned long long k = plan->k;
     switch (tid) {
       case 0: v = CVLC_STREAM_MAGIC; break;
-      case 1: v = 1u | (prm.quantizer << 16) | (s << 24); break;
-      case 2: v = (uint32_t)prm.d; break;
-      case 3: v = (uint32_t)(prm.d >> 32); break;
-      case 4: v = R; break;
-      case 5: v = prm.packet_bits; break;
-      case 6: v = prm.header_bits; break;
-      case 7: v = prm.client_id; break;
-      case 8: v = (uint32_t)prm.seed; break;
-      case 9: v = (uint32_t)(prm.seed >> 32); break;
-      case 10: v = prm.round; break;
+      case 1: v = 1u | (shape.quantizer << 16) | (s << 24); break;
+      case 2: v = (uint32_t)shape.d; break;
+      case 3: v = (uint32_t)(shape.d >> 32); break;
+      case 4: v = shape.R; break;
+      case 5: v = shape.packet_bits; break;
+      case 6: v = shape.header_bits; break;
+      case 7: v = cd.client_id; break;
+      case 8: v = (uint32_t)cd.seed; break;
+      case 9: v = (uint32_t)(cd.seed >> 32); break;
+      case 10: v = cd.round; break;
       case 11: v = 0; break;
       case 12: v = (uint32_t)Bbits; break;
       case 13: v = (uint32_t)(Bbits >> 32); break;
@@ -511,46 +622,63 @@ k_pack(const unsigned long long* __restrict__ buf_a, const unsigned long long* _
 // launcher
 // ===================================================================================
 
-cudaError_t launch_encode(const float* x, const cvlc_params& p, uint32_t s, uint32_t R, uint32_t max_cap,
-                          const cvlc_plan_t* plan, uint8_t* stream, void* ws, cudaStream_t st) {
+template <int CAP>
+static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
+                                   cudaStream_t st) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  const size_t pack_smem = (size_t)max_cap * 8;
   if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-    e = cudaFuncSetAttribute(k_pack, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = cudaFuncSetAttribute(k_pack<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
-  const EncLayout L = enc_layout(p.d);
+  BatchDesc<CAP> batch;
+  batch.n = n;
+  batch.pad = 0;
+  for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
+  const EncLayout L = enc_layout(shape.d, n, capacity);
   unsigned char* w = static_cast<unsigned char*>(ws);
-  EncHeader* hdr = reinterpret_cast<EncHeader*>(w);
-  unsigned long long* ghist = reinterpret_cast<unsigned long long*>(w + kEncWsSortHist);
-  unsigned long long* sel_state = reinterpret_cast<unsigned long long*>(w + L.off_select_state);
-  unsigned long long* sort_state = reinterpret_cast<unsigned long long*>(w + L.off_sort_state);
-  unsigned long long* buf_a = reinterpret_cast<unsigned long long*>(w + L.off_buf_a);
-  unsigned long long* buf_b = reinterpret_cast<unsigned long long*>(w + L.off_buf_b);
+  const size_t pack_smem = (size_t)shape.cap[1] * 8;
 
-  { LaunchScope ls(kKEncodeInit, st); k_encode_init<<<2 * kNumSM, 256, 0, st>>>(w, plan, L, p.d, s, R); }
   {
-    const uint64_t want = L.n_select_tiles;
-    const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? want : 8 * kNumSM);
-    LaunchScope ls(kKSelect, st);
-    k_select<<<grid, kSelectThreads, 0, st>>>(x, p.d, plan, hdr, sel_state, L.n_select_tiles, buf_a, p.d);
+    LaunchScope ls(kKEncodeInit, st);
+    k_encode_init<CAP><<<2 * kNumSM, 256, 0, st>>>(w, batch, shape, L);
   }
   {
-    const uint64_t want = L.max_sort_tiles;
-    const int grid = (int)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
-    { LaunchScope ls(kKSortHist, st); k_sort_hist<<<grid, 256, 0, st>>>(buf_a, plan, hdr, ghist); }
+    const uint64_t want = L.select_tiles * n;
+    const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
+    LaunchScope ls(kKSelect, st);
+    k_select<CAP><<<grid, kSelectThreads, 0, st>>>(batch, shape.d, w, L);
+  }
+  {
+    const uint64_t want = L.sort_tiles_max * n;
+    const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
+    {
+      LaunchScope ls(kKSortHist, st);
+      k_sort_hist<CAP><<<grid, 256, 0, st>>>(batch, w, L);
+    }
+    {
+      LaunchScope ls(kKSortScan, st);
+      k_sort_scan<CAP><<<n, 256, 0, st>>>(batch, w, L);
+    }
     for (int pass = 0; pass < kSortPasses; ++pass) {
       LaunchScope ls(kKSortPass, st);
-      k_sort_pass<<<grid, kSortThreads, 0, st>>>(pass, buf_a, buf_b, plan, hdr, ghist,
-                                                 sort_state + (size_t)pass * L.max_sort_tiles * 256);
+      k_sort_pass<CAP><<<grid, kSortThreads, ((size_t)n + 1) * 4, st>>>(pass, batch, w, L);
     }
   }
-  { LaunchScope ls(kKPack, st); k_pack<<<R, kPackThreads, pack_smem, st>>>(buf_a, buf_b, plan, hdr, ghist, p, s, R, reinterpret_cast<uint32_t*>(stream)); }
+  {
+    LaunchScope ls(kKPack, st);
+    k_pack<CAP><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+  }
   return cudaGetLastError();
+}
+
+cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
+                          cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, ws, st);
+  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, ws, st);
 }
 
 }  // namespace cvlc

@@ -16,57 +16,74 @@ namespace cvlc {
 constexpr int kHistThreads = 512;
 constexpr int kHistSub = 4;  // shared sub-histograms per block (64 KB)
 
+// The clients' updates are treated as one concatenated array of units (a unit = one float4,
+// plus one ragged-tail unit per client) that is cut into equal contiguous chunks, one per
+// block, so the load is even whatever the number of clients; a block that crosses a client
+// boundary merges its shared histogram into that client's global one and starts afresh.
+__device__ __forceinline__ uint32_t hist_add4(uint32_t* my, const float4 a) {
+  const uint32_t k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
+  const uint32_t k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
+  atomicAdd(my + (k0 >> 19), 1u);
+  atomicAdd(my + (k1 >> 19), 1u);
+  atomicAdd(my + (k2 >> 19), 1u);
+  atomicAdd(my + (k3 >> 19), 1u);
+  return (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
+}
+
+template <int CAP>
 __global__ void __launch_bounds__(kHistThreads, 2)
-k_hist(const float* __restrict__ x, uint64_t d, unsigned long long* __restrict__ hist, uint32_t* __restrict__ nonfinite) {
+k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned long long* __restrict__ hist_all,
+       uint32_t* __restrict__ nonfinite_all) {
   extern __shared__ uint32_t sh_hist[];  // [kHistSub][4096]
   for (int i = threadIdx.x; i < kHistSub * CVLC_HIST_BINS; i += kHistThreads) sh_hist[i] = 0;
   __syncthreads();
   uint32_t* my = sh_hist + ((threadIdx.x >> 5) & (kHistSub - 1)) * CVLC_HIST_BINS;
 
   const uint64_t nvec = d >> 2;
-  const float4* xv = reinterpret_cast<const float4*>(x);
-  const uint64_t stride = (uint64_t)gridDim.x * kHistThreads;
-  uint32_t bad = 0;
-  uint64_t v = (uint64_t)blockIdx.x * kHistThreads + threadIdx.x;
-  // four independent 128-bit loads in flight per thread
-  for (; v + 3 * stride < nvec; v += 4 * stride) {
-    float4 a[4];
+  const uint64_t units = nvec + 1;  // per client: nvec float4 units and one tail unit
+  const uint64_t total = units * batch.n;
+  const uint64_t chunk = (total + gridDim.x - 1) / gridDim.x;
+  uint64_t pos = (uint64_t)blockIdx.x * chunk;
+  const uint64_t end = (pos + chunk < total) ? pos + chunk : total;
+
+  while (pos < end) {
+    const uint64_t c = pos / units;
+    const uint64_t seg_end = ((c + 1) * units < end) ? (c + 1) * units : end;
+    const uint64_t u0 = pos - c * units, u1 = seg_end - c * units;
+    const float* __restrict__ x = batch.c[c].x;
+    const float4* xv = reinterpret_cast<const float4*>(x);
+    const uint64_t v1 = (u1 < nvec) ? u1 : nvec;  // float4 units of this segment: [u0, v1)
+    uint32_t bad = 0;
+    uint64_t v = u0 + threadIdx.x;
+    // four independent 128-bit loads in flight per thread
+    for (; v + 3 * kHistThreads < v1; v += 4 * kHistThreads) {
+      float4 a[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * stride);
+      for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * kHistThreads);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t k0 = __float_as_uint(a[u].x) & 0x7FFFFFFFu, k1 = __float_as_uint(a[u].y) & 0x7FFFFFFFu;
-      const uint32_t k2 = __float_as_uint(a[u].z) & 0x7FFFFFFFu, k3 = __float_as_uint(a[u].w) & 0x7FFFFFFFu;
-      bad |= (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
-      atomicAdd(my + (k0 >> 19), 1u);
-      atomicAdd(my + (k1 >> 19), 1u);
-      atomicAdd(my + (k2 >> 19), 1u);
-      atomicAdd(my + (k3 >> 19), 1u);
+      for (int u = 0; u < 4; ++u) bad |= hist_add4(my, a[u]);
     }
-  }
-  for (; v < nvec; v += stride) {
-    const float4 a = __ldg(xv + v);
-    const uint32_t k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
-    const uint32_t k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
-    bad |= (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
-    atomicAdd(my + (k0 >> 19), 1u);
-    atomicAdd(my + (k1 >> 19), 1u);
-    atomicAdd(my + (k2 >> 19), 1u);
-    atomicAdd(my + (k3 >> 19), 1u);
-  }
-  // ragged tail (d not a multiple of 4)
-  if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
-    const uint32_t k0 = __float_as_uint(x[(nvec << 2) + threadIdx.x]) & 0x7FFFFFFFu;
-    bad |= (k0 >= 0x7F800000u);
-    atomicAdd(my + (k0 >> 19), 1u);
-  }
-  if (bad) atomicOr(nonfinite, 1u);
-  __syncthreads();
-  for (int b = threadIdx.x; b < CVLC_HIST_BINS; b += kHistThreads) {
-    uint32_t c = 0;
+    for (; v < v1; v += kHistThreads) bad |= hist_add4(my, __ldg(xv + v));
+    // ragged tail of the client (d not a multiple of 4)
+    if (u1 == units && threadIdx.x < (d & 3)) {
+      const uint32_t k0 = __float_as_uint(x[(nvec << 2) + threadIdx.x]) & 0x7FFFFFFFu;
+      bad |= (k0 >= 0x7F800000u);
+      atomicAdd(my + (k0 >> 19), 1u);
+    }
+    if (bad) atomicOr(nonfinite_all + c, 1u);
+    __syncthreads();
+    unsigned long long* __restrict__ hist = hist_all + (size_t)c * CVLC_HIST_BINS;
+    for (int b = threadIdx.x; b < CVLC_HIST_BINS; b += kHistThreads) {
+      uint32_t cnt = 0;
 #pragma unroll
-    for (int s = 0; s < kHistSub; ++s) c += sh_hist[s * CVLC_HIST_BINS + b];
-    if (c) atomicAdd(hist + b, (unsigned long long)c);
+      for (int sub = 0; sub < kHistSub; ++sub) {
+        cnt += sh_hist[sub * CVLC_HIST_BINS + b];
+        sh_hist[sub * CVLC_HIST_BINS + b] = 0;
+      }
+      if (cnt) atomicAdd(hist + b, (unsigned long long)cnt);
+    }
+    __syncthreads();
+    pos = seg_end;
   }
 }
 
@@ -176,16 +193,73 @@ struct PlanShared {
   uint32_t n_points;
 };
 
+// candidate lengths of one client and their coefficients (Eq. (5)), built by warp 0
+struct PlanTab {
+  uint64_t d;
+  uint32_t s, R, nY, y_min, fixed_y;
+  uint32_t Y[32];     // candidate lengths, ascending
+  uint32_t capY[32];  // cap(Y[i])
+  double gY[32];      // g(Y[i]) = 1 - (Q/B^2 + (1 - 1/B)^2)
+  double QY[32];      // PQ error factor Q(Y[i]) = cap / (2^y - 1)^2
+};
+
+template <int CAP>
 __global__ void __launch_bounds__(kPlanThreads, 1)
-k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__ nonfinite,
-       const __grid_constant__ PlanTables T, cvlc_plan_t* __restrict__ plan) {
+k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restrict__ nonfinite_all,
+       const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, int32_t* ws_status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned long long* Nsuf = reinterpret_cast<unsigned long long*>(smem_raw);  // [4096] survival counts
   double* ptX = reinterpret_cast<double*>(smem_raw + 4096 * 8);                // fit points, ascending bin
   double* ptY = ptX + 4096;
   __shared__ PlanShared S;
+  __shared__ PlanTab T;
+
+  // blockIdx.x = client
+  const unsigned long long* __restrict__ hist = hist_all + (size_t)blockIdx.x * CVLC_HIST_BINS;
+  const uint32_t* __restrict__ nonfinite = nonfinite_all + blockIdx.x;
+  cvlc_plan_t* __restrict__ plan = batch.c[blockIdx.x].plan;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- candidate lengths: g(y) > 0 (the paper's B > (Q+1)/2) and not dominated --------
+  if (warp == 0) {
+    const uint32_t y = lane + 1;
+    const double B = batch.c[blockIdx.x].scale_B;
+    const bool in_range = y <= shape.max_code_bits;
+    const uint32_t cap_y = in_range ? shape.cap[y] : 0u;
+    const double L = (double)((1ull << y) - 1ull);
+    const double Q = __ddiv_rn((double)cap_y, __dmul_rn(L, L));
+    const double one_m = __dsub_rn(1.0, __ddiv_rn(1.0, B));
+    const double g = __dsub_rn(1.0, __dadd_rn(__ddiv_rn(Q, __dmul_rn(B, B)), __dmul_rn(one_m, one_m)));
+    unsigned member;
+    uint32_t y_min;
+    if (shape.fixed_y) {
+      y_min = shape.fixed_y;
+      member = 1u << (shape.fixed_y - 1);
+    } else {
+      const unsigned pos = __ballot_sync(kFull, in_range && g > 0.0);
+      y_min = pos ? (uint32_t)__ffs(pos) : 1u;  // the host has checked that one exists
+      const uint32_t cap_next = __shfl_down_sync(kFull, cap_y, 1);
+      const bool keep = in_range && y >= y_min && (y == shape.max_code_bits || cap_y > cap_next);
+      member = __ballot_sync(kFull, keep);
+    }
+    if (member & (1u << lane)) {
+      const int i = __popc(member & ((1u << lane) - 1u));
+      T.Y[i] = y;
+      T.capY[i] = cap_y;
+      T.gY[i] = g;
+      T.QY[i] = Q;
+    }
+    if (lane == 0) {
+      T.d = shape.d;
+      T.s = shape.s;
+      T.R = shape.R;
+      T.nY = (uint32_t)__popc(member);
+      T.y_min = y_min;
+      T.fixed_y = shape.fixed_y;
+    }
+  }
+  __syncthreads();
 
   // ---- survival counts N_j = #{bin >= j} ------------------------------------------
   unsigned long long h[4];
@@ -417,6 +491,7 @@ k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__
     for (int i = 0; i < nY; ++i)
       if (S.n[i] > 0 && T.QY[i] > Qmax) Qmax = T.QY[i];
     plan->status = (*nonfinite) ? CVLC_ERR_NONFINITE_INPUT : CVLC_OK;
+    if (*nonfinite) set_status(ws_status, CVLC_ERR_NONFINITE_INPUT);
     plan->s = T.s;
     plan->R = T.R;
     plan->y_min = T.y_min;
@@ -429,7 +504,7 @@ k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__
     plan->B_next = __dadd_rn(1.0, Qmax);
     for (int y = 0; y <= CVLC_MAX_CODE_BITS; ++y) {
       plan->n_y[y] = 0;
-      plan->cap[y] = T.cap[y];
+      plan->cap[y] = shape.cap[y];
     }
     for (int i = 0; i < nY; ++i) plan->n_y[T.Y[i]] = S.n[i];
   }
@@ -450,28 +525,48 @@ k_plan(const unsigned long long* __restrict__ hist, const uint32_t* __restrict__
 // launchers
 // ===================================================================================
 
-cudaError_t launch_plan(const float* x, const PlanTables& T, cvlc_plan_t* plan, void* ws, cudaStream_t st) {
+template <int CAP>
+static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-    e = cudaFuncSetAttribute(k_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
+    e = cudaFuncSetAttribute(k_hist<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
+    e = cudaFuncSetAttribute(k_plan<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
+  BatchDesc<CAP> batch;
+  batch.n = n;
+  batch.pad = 0;
+  for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
   unsigned char* w = static_cast<unsigned char*>(ws);
   unsigned long long* hist = reinterpret_cast<unsigned long long*>(w + kPlanWsHist);
-  uint32_t* flag = reinterpret_cast<uint32_t*>(w + kPlanWsStatus + 4);
-  { LaunchScope ls(kKZeroWords, st); k_zero_words<<<8, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsBytes / 4); }
-  const uint64_t nvec = T.d >> 2;
-  uint64_t want = (nvec + kHistThreads - 1) / kHistThreads;
-  int grid = (int)(want < (uint64_t)(2 * kNumSM) ? (want ? want : 1) : 2 * kNumSM);
-  { LaunchScope ls(kKHist, st); k_hist<<<grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(x, T.d, hist, flag); }
-  { LaunchScope ls(kKPlan, st); k_plan<<<1, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flag, T, plan); }
+  uint32_t* flags = reinterpret_cast<uint32_t*>(w + plan_off_flags(n));
+  {
+    LaunchScope ls(kKZeroWords, st);
+    k_zero_words<<<2 * kNumSM, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), plan_ws_bytes(n) / 4);
+  }
+  // two resident blocks per SM share the concatenated updates evenly
+  const uint64_t total_units = ((shape.d >> 2) + 1) * n;
+  uint64_t grid = (total_units + 4 * kHistThreads - 1) / (4 * kHistThreads);
+  if (grid > (uint64_t)(2 * kNumSM)) grid = 2 * kNumSM;
+  {
+    LaunchScope ls(kKHist, st);
+    k_hist<CAP><<<(unsigned)grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, hist, flags);
+  }
+  {
+    LaunchScope ls(kKPlan, st);
+    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, reinterpret_cast<int32_t*>(w));
+  }
   return cudaGetLastError();
+}
+
+cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, st);
+  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, st);
 }
 
 // ---- diagnostics ---------------------------------------------------------------------

@@ -196,6 +196,55 @@ def test_other_packet_and_header_sizes(torch_cuda):
         run_case(x, pd)
 
 
+@pytest.mark.parametrize("n", [2, 4, 5, 23])
+def test_batched_plan_encode_matches_oracle_per_client(torch_cuda, n):
+    """one set of launches for n clients (different data, scales and Philox ids) = n oracle runs"""
+    torch = torch_cuda
+    from paper_2402_03770_b200 import binding as B
+    from gpu_util import gpu_params
+    w = W.WORKLOADS["resnet18"]
+    d = 120_001                                                                  # ragged: not a multiple of 4
+    dev = torch.device("cuda:0")
+    xs, pds = [], []
+    for c in range(n):
+        x = W.client_update(w, c, d=d)
+        if c == 1:
+            x[:] = 0.0                                                           # one all-zero client inside the batch
+        xs.append(x)
+        pds.append(params_dict(d, 20 * 12000 + 7 * c, seed=100 + c, client_id=c, round=c % 3, scale_B=1.0 + 0.002 * c))
+    params = [gpu_params(pd) for pd in pds]
+    for max_cand in (0, 60_000 if n != 5 else 0):
+        enc = B.BatchEncoder(params, dev, max_candidates=max_cand)
+        for o in enc.outs:
+            o.fill_(0xCD)
+        dxs = [torch.from_numpy(x).to(dev) for x in xs]
+        outs = enc.run(dxs)
+        status = enc.status()
+        if max_cand:
+            # the all-zero client has d candidates: more than the reduced workspace holds
+            assert status == B.CVLC_ERR_WORKSPACE_TOO_SMALL
+            continue
+        assert status == 0
+        for c in range(n):
+            of, ost = oracle_plan_encode(xs[c], pds[c])
+            assert_plan_equal(enc.read_plan(c), of)
+            assert (outs[c].cpu().numpy() == ost).all(), c
+
+
+def test_batch_rejects_mixed_shapes(torch_cuda):
+    torch = torch_cuda
+    from paper_2402_03770_b200 import binding as B
+    dev = torch.device("cuda:0")
+    d = 50_000
+    xs = [torch.zeros(d, device=dev), torch.zeros(d, device=dev)]
+    params = [B.make_params(d, 10 * 12000), B.make_params(d, 11 * 12000)]
+    plans = B.alloc_bytes(2 * B.PLAN_BYTES, dev)
+    ws = B.alloc_bytes(B.cvlc_plan_batch_workspace_bytes(params[0], 2), dev)
+    with pytest.raises(B.CvlcError) as e:
+        B.cvlc_plan_batch(xs, params, plans, ws)
+    assert e.value.code == B.CVLC_ERR_INVALID_ARG
+
+
 def test_encode_is_deterministic(torch_cuda):
     w = W.WORKLOADS["small_cnn"]
     x = W.client_update(w, 3, d=500_000)

@@ -94,7 +94,9 @@ typedef struct cvlc_plan_t {
   double B_next;          /* 1 + max Q over the used lengths: scale_B for the next round */
   uint32_t n_y[CVLC_MAX_CODE_BITS + 1]; /* packets per code length; packets are laid out longest code first */
   uint32_t cap[CVLC_MAX_CODE_BITS + 1]; /* records per packet per code length: floor((b - H) / (s + y)) */
-  uint8_t reserved[512 - 80 - 2 * 4 * (CVLC_MAX_CODE_BITS + 1)];
+  uint32_t top_bin;       /* highest non-empty histogram bin */
+  uint32_t reserved0;
+  uint8_t reserved[512 - 88 - 2 * 4 * (CVLC_MAX_CODE_BITS + 1)];
 } cvlc_plan_t;
 
 /* --- host-only helpers (no GPU work) --------------------------------------- */
@@ -145,12 +147,16 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
  * packs (position ID, centroid ID) pairs behind the packet header (Fig. 2).
  * stream_dev (16-byte aligned) receives cvlc_stream_bytes(p) bytes.
  * plan_dev must come from cvlc_plan / cvlc_plan_fixed on the same x_dev and params.
+ * plan_ws_dev: the workspace that call used, untouched since (it holds per-chunk candidate
+ * counts that let the selection run without any exchange between thread blocks), or NULL
+ * when it is gone or the plan came from elsewhere: the selection then computes its output
+ * offsets itself with a decoupled look-back scan across blocks (slower).
  * Errors: INVALID_ARG, OUTPUT_TOO_SMALL, WORKSPACE_TOO_SMALL (host); PLAN_MISMATCH,
  * DEVICE_TIMEOUT (device, at byte 0 of ws_dev).
  */
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev,
-                uint8_t* stream_dev, size_t stream_capacity, void* ws_dev, size_t ws_bytes,
-                void* cuda_stream);
+                const void* plan_ws_dev, uint8_t* stream_dev, size_t stream_capacity, void* ws_dev,
+                size_t ws_bytes, void* cuda_stream);
 
 /*
  * Batched forms: the same kernels over n clients (n <= CVLC_MAX_BATCH) in one set of
@@ -168,15 +174,17 @@ int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* pla
  *               with WORKSPACE_TOO_SMALL (device-detected, byte 0 of the workspace).
  * A device-detected error in one client (non-finite input, plan mismatch) stops the
  * encoding of the whole batch.  After cvlc_plan_batch the histogram of client i sits at
- * byte 256 + 32768 * i of the workspace.
+ * byte 256 + 32768 * i of the workspace.  plan_ws_dev (see cvlc_encode) must be the workspace
+ * of the cvlc_plan_batch call on the same n clients in the same order, or NULL.
  */
 size_t cvlc_plan_batch_workspace_bytes(const cvlc_params* p, uint32_t n);
 size_t cvlc_encode_batch_workspace_bytes(const cvlc_params* p, uint32_t n, uint64_t max_candidates);
 int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint32_t fixed_y,
                     cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream);
 int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n,
-                      const cvlc_plan_t* plans_dev, uint8_t* const* streams_dev, size_t stream_capacity,
-                      uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+                      const cvlc_plan_t* plans_dev, const void* plan_ws_dev, uint8_t* const* streams_dev,
+                      size_t stream_capacity, uint64_t max_candidates, void* ws_dev, size_t ws_bytes,
+                      void* cuda_stream);
 
 /*
  * Parameter-server aggregation (Section III, step 3) fused with decoding: for every

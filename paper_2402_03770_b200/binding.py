@@ -65,7 +65,8 @@ class CvlcPlan(C.Structure):
         ("alpha", C.c_double), ("alpha_q", C.c_double), ("beta", C.c_double),
         ("gamma", C.c_double), ("B_next", C.c_double),
         ("n_y", C.c_uint32 * (MAX_CODE_BITS + 1)), ("cap", C.c_uint32 * (MAX_CODE_BITS + 1)),
-        ("reserved", C.c_uint8 * (512 - 80 - 2 * 4 * (MAX_CODE_BITS + 1))),
+        ("top_bin", C.c_uint32), ("reserved0", C.c_uint32),
+        ("reserved", C.c_uint8 * (512 - 88 - 2 * 4 * (MAX_CODE_BITS + 1))),
     ]
 
 
@@ -112,7 +113,7 @@ def lib() -> C.CDLL:
     L.cvlc_plan_fixed.restype = C.c_int
     L.cvlc_plan_fixed.argtypes = [vp, PP, u32, vp, vp, sz, vp]
     L.cvlc_encode.restype = C.c_int
-    L.cvlc_encode.argtypes = [vp, PP, vp, vp, sz, vp, sz, vp]
+    L.cvlc_encode.argtypes = [vp, PP, vp, vp, vp, sz, vp, sz, vp]
     L.cvlc_plan_batch_workspace_bytes.restype = sz
     L.cvlc_plan_batch_workspace_bytes.argtypes = [PP, u32]
     L.cvlc_encode_batch_workspace_bytes.restype = sz
@@ -120,7 +121,7 @@ def lib() -> C.CDLL:
     L.cvlc_plan_batch.restype = C.c_int
     L.cvlc_plan_batch.argtypes = [vp, PP, u32, u32, vp, vp, sz, vp]
     L.cvlc_encode_batch.restype = C.c_int
-    L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, sz, u64, vp, sz, vp]
+    L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
     L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
     L.cvlc_decode_aggregate_noalloc.restype = C.c_int
@@ -217,10 +218,12 @@ def cvlc_plan_fixed(x: torch.Tensor, p: CvlcParams, y: int, plan: torch.Tensor, 
 
 
 def cvlc_encode(x: torch.Tensor, p: CvlcParams, plan: torch.Tensor, out_stream: torch.Tensor,
-                ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+                ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+                plan_ws: Optional[torch.Tensor] = None) -> None:
+    """plan_ws: the workspace cvlc_plan used for this plan (fast selection) or None (look-back selection)."""
     assert x.dtype == torch.float32 and x.numel() == p.d
     assert out_stream.dtype == torch.uint8
-    _check(lib().cvlc_encode(_ptr(x), C.byref(p), _ptr(plan), _ptr(out_stream), out_stream.numel(),
+    _check(lib().cvlc_encode(_ptr(x), C.byref(p), _ptr(plan), _ptr(plan_ws), _ptr(out_stream), out_stream.numel(),
                              _ptr(ws), ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode")
 
 
@@ -252,13 +255,14 @@ def cvlc_plan_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], pl
 
 def cvlc_encode_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor,
                       outs: Sequence[torch.Tensor], ws: torch.Tensor, max_candidates: int = 0,
-                      stream: Optional[torch.cuda.Stream] = None, _cache=None) -> None:
+                      stream: Optional[torch.cuda.Stream] = None, _cache=None,
+                      plan_ws: Optional[torch.Tensor] = None) -> None:
     """outs: n device uint8 tensors of cvlc_stream_bytes(params[0]) bytes each."""
     n = len(xs)
     assert len(params) == n and len(outs) == n
     xa, pa, oa = _cache if _cache is not None else (_ptr_array(xs), _params_array(params), _ptr_array(outs))
     cap = min(o.numel() for o in outs)
-    _check(lib().cvlc_encode_batch(xa, pa, n, _ptr(plans), oa, cap, int(max_candidates), _ptr(ws),
+    _check(lib().cvlc_encode_batch(xa, pa, n, _ptr(plans), _ptr(plan_ws), oa, cap, int(max_candidates), _ptr(ws),
                                    ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode_batch")
 
 
@@ -355,14 +359,14 @@ class ClientEncoder:
         self.out = alloc_bytes(cvlc_stream_bytes(p), device)
 
     def run(self, x: torch.Tensor, p: Optional[CvlcParams] = None, out: Optional[torch.Tensor] = None,
-            stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0) -> torch.Tensor:
+            stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0, use_plan_ws: bool = True) -> torch.Tensor:
         p = self.p if p is None else p
         out = self.out if out is None else out
         if fixed_y:
             cvlc_plan_fixed(x, p, fixed_y, self.plan, self.plan_ws, stream)
         else:
             cvlc_plan(x, p, self.plan, self.plan_ws, stream)
-        cvlc_encode(x, p, self.plan, out, self.enc_ws, stream)
+        cvlc_encode(x, p, self.plan, out, self.enc_ws, stream, plan_ws=self.plan_ws if use_plan_ws else None)
         return out
 
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
@@ -386,11 +390,12 @@ class BatchEncoder:
         self._pa = _params_array(self.params)
         self._oa = _ptr_array(self.outs)
 
-    def run(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0):
+    def run(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0,
+            use_plan_ws: bool = True):
         xa = _ptr_array(xs)
         cvlc_plan_batch(xs, self.params, self.plans, self.plan_ws, fixed_y, stream, _cache=(xa, self._pa))
         cvlc_encode_batch(xs, self.params, self.plans, self.outs, self.enc_ws, self.max_candidates, stream,
-                          _cache=(xa, self._pa, self._oa))
+                          _cache=(xa, self._pa, self._oa), plan_ws=self.plan_ws if use_plan_ws else None)
         return self.outs
 
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:

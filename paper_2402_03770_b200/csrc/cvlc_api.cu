@@ -144,7 +144,7 @@ size_t cvlc_plan_workspace_bytes(const cvlc_params* p) { return cvlc_plan_batch_
 
 size_t cvlc_plan_batch_workspace_bytes(const cvlc_params* p, uint32_t n) {
   if (!params_ok(p) || n == 0 || n > CVLC_MAX_BATCH) return 0;
-  return plan_ws_bytes(n);
+  return plan_ws_bytes(n, make_partition(p->d, n).max_segments);
 }
 
 size_t cvlc_encode_workspace_bytes(const cvlc_params* p) { return cvlc_encode_batch_workspace_bytes(p, 1, 0); }
@@ -180,7 +180,7 @@ int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32
     desc[i].round = params[i].round;
   }
   if (!aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
-  if (ws_bytes < plan_ws_bytes(n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   return launch_plan(desc, n, S, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
@@ -196,8 +196,8 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
 }
 
 int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
-                      uint8_t* const* streams_dev, size_t stream_capacity, uint64_t max_candidates, void* ws_dev,
-                      size_t ws_bytes, void* cuda_stream) {
+                      const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                      uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
   if (!x_dev || !params || !streams_dev || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
   Shape S;
   ClientDesc desc[CVLC_MAX_BATCH];
@@ -227,18 +227,20 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
     desc[i].round = params[i].round;
   }
   if (!aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (plan_ws_dev && !aligned(plan_ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
   if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
   const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
   if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   if ((size_t)S.cap[1] * 8 > 200 * 1024) return CVLC_ERR_INVALID_ARG;  // a packet's records are staged in shared memory
   if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
-  return launch_encode(desc, n, S, cap, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
+  return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
                                                                                                        : CVLC_ERR_CUDA;
 }
 
-int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, uint8_t* stream_dev,
-                size_t stream_capacity, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
-  return cvlc_encode_batch(&x_dev, p, 1, plan_dev, &stream_dev, stream_capacity, 0, ws_dev, ws_bytes, cuda_stream);
+int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, const void* plan_ws_dev,
+                uint8_t* stream_dev, size_t stream_capacity, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  return cvlc_encode_batch(&x_dev, p, 1, plan_dev, plan_ws_dev, &stream_dev, stream_capacity, 0, ws_dev, ws_bytes,
+                           cuda_stream);
 }
 
 int cvlc_decode_aggregate(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev, const float* weights_dev,

@@ -57,10 +57,51 @@ struct Shape {
 
 // ---- workspace layouts (byte offsets; every region 256-byte aligned) ----------
 
-// plan workspace: [0] int32 status | [256] uint64 hist[n][4096] | uint32 nonfinite[n]
+// The histogram and the selection kernel stream the clients' updates as one concatenated
+// array of units (a unit = one float4; every client ends with one ragged-tail unit) cut into
+// equal contiguous chunks, one per thread block.  A segment is the part of one client inside
+// one chunk; with block b and client c both non-decreasing along the array, b + c numbers the
+// segments uniquely.
+constexpr int kStreamThreads = 512;
+struct Partition {
+  uint64_t units;   // per client: d / 4 float4 units + 1 tail unit
+  uint64_t total;   // units * n
+  uint64_t chunk;   // units per block
+  uint32_t grid;    // blocks
+  uint32_t max_segments;  // grid + n
+};
+CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
+  Partition P;
+  P.units = (d >> 2) + 1;
+  P.total = P.units * n;
+  uint64_t grid = (P.total + 4 * kStreamThreads - 1) / (4 * kStreamThreads);
+  if (grid > (uint64_t)(2 * kNumSM)) grid = 2 * kNumSM;
+  if (grid == 0) grid = 1;
+  P.grid = (uint32_t)grid;
+  P.chunk = (P.total + grid - 1) / grid;
+  P.max_segments = P.grid + n;
+  return P;
+}
+
+// plan workspace:
+//   [0] PlanWsHeader | [256] uint64 hist[n][4096] | uint32 nonfinite[n] | uint32 seg_count[S]
+//   | uint64 seg_prefix[S] | uint32 seg_hist[S][4096]          (S = max_segments)
+struct PlanWsHeader {
+  int32_t status;   // byte 0
+  uint32_t n;       // clients of the batch the workspace was filled for
+  uint64_t d;
+  uint32_t grid;
+  uint32_t magic;   // set when the segment tables are valid
+};
+constexpr uint32_t kPlanWsMagic = 0x53454743u;
 constexpr size_t kPlanWsHist = 256;
 CVLC_HD constexpr size_t plan_off_flags(uint32_t n) { return kPlanWsHist + (size_t)n * CVLC_HIST_BINS * 8; }
-CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n) { return align256(plan_off_flags(n) + (size_t)n * 4); }
+CVLC_HD constexpr size_t plan_off_seg_count(uint32_t n) { return align256(plan_off_flags(n) + (size_t)n * 4); }
+CVLC_HD constexpr size_t plan_off_seg_prefix(uint32_t n, uint32_t S) { return align256(plan_off_seg_count(n) + (size_t)S * 4); }
+CVLC_HD constexpr size_t plan_off_seg_hist(uint32_t n, uint32_t S) { return align256(plan_off_seg_prefix(n, S) + (size_t)S * 8); }
+CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n, uint32_t S) {
+  return align256(plan_off_seg_hist(n, S) + (size_t)S * CVLC_HIST_BINS * 4);
+}
 
 // encode workspace header (first 256 bytes), zeroed at the start of a call
 struct EncHeader {
@@ -68,6 +109,7 @@ struct EncHeader {
   uint32_t select_ticket;   // tile tickets of the selection kernel
   uint32_t sort_ticket[4];  // tile tickets of the four digit passes
   uint32_t total_sort_tiles;
+  uint32_t max_sort_tiles;  // largest per-client tile count of this batch
 };
 
 constexpr int kSelectThreads = 512;
@@ -77,7 +119,9 @@ constexpr int kSelectTile = kSelectThreads * kSelectVecPerThread * 4;  // 8192 c
 constexpr int kSortThreads = 256;
 constexpr int kSortItemsPerThread = 8;
 constexpr int kSortTile = kSortThreads * kSortItemsPerThread;  // 2048 pairs
-constexpr int kSortPasses = 4;                                 // digits of 8,8,8,7 bits
+constexpr int kSortPasses = 4;                                 // digits of 9,9,9,4 bits
+constexpr int kDigitBits = 9;
+constexpr int kDigits = 1 << kDigitBits;                       // 512 digit values
 
 struct EncLayout {
   uint32_t n;
@@ -87,10 +131,10 @@ struct EncLayout {
   size_t off_n_selected;         // uint64[n]
   size_t off_sort_prefix;        // uint32[n + 1]: first sort tile of every client
   size_t off_pass_mask;          // uint32[n]: digit passes that are constant for the client
-  size_t off_ghist;              // uint64[n][4][256] digit histograms
-  size_t off_gbase;              // uint64[n][4][256] their exclusive scans
+  size_t off_ghist;              // uint64[n][4][512] digit histograms
+  size_t off_gbase;              // uint64[n][4][512] their exclusive scans
   size_t off_select_state;       // uint64[n][select_tiles]
-  size_t off_sort_state;         // uint64[4][n * sort_tiles_max][256]
+  size_t off_sort_state;         // uint64[4][n * sort_tiles_max][512]
   size_t off_buf_a, off_buf_b;   // uint64[n][capacity]
   size_t total;
 };
@@ -105,10 +149,10 @@ static inline EncLayout enc_layout(uint64_t d, uint32_t n, uint64_t capacity) {
   L.off_sort_prefix = align256(L.off_n_selected + (size_t)n * 8);
   L.off_pass_mask = align256(L.off_sort_prefix + ((size_t)n + 1) * 4);
   L.off_ghist = align256(L.off_pass_mask + (size_t)n * 4);
-  L.off_gbase = align256(L.off_ghist + (size_t)n * kSortPasses * 256 * 8);
-  L.off_select_state = align256(L.off_gbase + (size_t)n * kSortPasses * 256 * 8);
+  L.off_gbase = align256(L.off_ghist + (size_t)n * kSortPasses * kDigits * 8);
+  L.off_select_state = align256(L.off_gbase + (size_t)n * kSortPasses * kDigits * 8);
   L.off_sort_state = align256(L.off_select_state + (size_t)n * L.select_tiles * 8);
-  L.off_buf_a = align256(L.off_sort_state + (size_t)kSortPasses * n * L.sort_tiles_max * 256 * 8);
+  L.off_buf_a = align256(L.off_sort_state + (size_t)kSortPasses * n * L.sort_tiles_max * kDigits * 8);
   L.off_buf_b = align256(L.off_buf_a + (size_t)n * capacity * 8);
   L.total = align256(L.off_buf_b + (size_t)n * capacity * 8);
   return L;
@@ -126,7 +170,7 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 // ---- launch accounting and optional per-kernel timing ------------------------------
 
 enum KernelId {
-  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSortHist, kKSortScan, kKSortPass, kKPack,
+  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan, kKSortPass, kKPack,
   kKDecodePrepare, kKFillZero, kKDecode, kKSelftest, kNumKernelIds
 };
 
@@ -145,8 +189,8 @@ struct LaunchScope {
 // ---- launchers (one per translation unit) ---------------------------------------
 
 cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
-cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
-                          cudaStream_t st);
+cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
+                          const void* plan_ws, void* ws, cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
                           void* ws, cudaStream_t st);

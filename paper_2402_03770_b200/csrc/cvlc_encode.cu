@@ -51,7 +51,7 @@ __device__ __forceinline__ uint32_t sort_tiles_of(unsigned long long n_candidate
 template <int CAP>
 __global__ void __launch_bounds__(256)
 k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
-              const __grid_constant__ EncLayout L) {
+              const __grid_constant__ EncLayout L, const unsigned char* plan_ws, const __grid_constant__ Partition part) {
   __shared__ unsigned long long s_total;
   __shared__ int s_bad;
   const uint32_t n = batch.n;
@@ -71,9 +71,9 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
     const size_t nb = (L.off_sort_state - L.off_ghist) / 8;  // digit histograms, their scans, selection tile states
     for (size_t i = gtid; i < nb; i += gstride) b[i] = 0ull;
   }
-  const size_t per_pass = (size_t)s_total * 256;
+  const size_t per_pass = (size_t)s_total * kDigits;
   for (int p = 0; p < kSortPasses; ++p) {
-    unsigned long long* st = reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)p * n * L.sort_tiles_max * 256;
+    unsigned long long* st = reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)p * n * L.sort_tiles_max * kDigits;
     for (size_t i = gtid; i < per_pass; i += gstride) st[i] = 0ull;
   }
   if (blockIdx.x != 0) return;
@@ -99,12 +99,20 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    uint32_t run = 0;
+    uint32_t run = 0, mx = 0;
     for (uint32_t c = 0; c < n; ++c) {
       prefix[c] = run;
-      run += sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
+      const uint32_t t = sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
+      run += t;
+      if (t > mx) mx = t;
     }
     prefix[n] = run;
+    if (plan_ws && !s_bad) {
+      // the segment tables must have been made for this very batch
+      const PlanWsHeader* ph = reinterpret_cast<const PlanWsHeader*>(plan_ws);
+      if (ph->magic != kPlanWsMagic || ph->n != n || ph->d != shape.d || ph->grid != part.grid) s_bad = CVLC_ERR_PLAN_MISMATCH;
+    }
+    hdr->max_sort_tiles = mx;
     hdr->status = s_bad;
     hdr->select_ticket = 0;
     for (int p = 0; p < kSortPasses; ++p) hdr->sort_ticket[p] = 0;
@@ -117,12 +125,14 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
 // ===================================================================================
 // Emits (key << 32 | sign << 31 | index) for every coordinate whose histogram bin is at or
 // above the plan's threshold bin, in ascending index order.  4 bytes read per coordinate.
-// Tiles of 8192 coordinates are handed out by an atomic ticket (client-major), so every
+// Tiles of 8192 coordinates are handed out by an atomic ticket (tile-major, clients interleaved:
+// the tiles in flight at any time are a few consecutive tiles of every client), so every
 // predecessor of a tile is running or done; the look-back reads 512 predecessors per step.
+// Used when the plan's workspace (and with it the per-segment counts) is not available.
 
 template <int CAP>
 __global__ void __launch_bounds__(kSelectThreads)
-k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned char* ws, const __grid_constant__ EncLayout L) {
+k_select_lookback(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ uint32_t s_tile;
   __shared__ unsigned long long s_warp_incl[kSelectThreads / 32];
   __shared__ unsigned long long s_look_sum[kSelectThreads / 32];
@@ -139,8 +149,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned char
     __syncthreads();
     const uint64_t gt = s_tile;
     if (gt >= total_tiles) break;
-    const uint32_t c = (uint32_t)(gt / tiles_per_client);
-    const uint64_t tile = gt - (uint64_t)c * tiles_per_client;
+    const uint64_t tile = gt / batch.n;
+    const uint32_t c = (uint32_t)(gt - tile * batch.n);
     const float* __restrict__ x = batch.c[c].x;
     const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
     const float4* xv = reinterpret_cast<const float4*>(x);
@@ -266,17 +276,194 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned char
 }
 
 // ===================================================================================
+// K3' threshold selection with offsets known in advance (no exchange between blocks)
+// ===================================================================================
+// Same chunking of the concatenated updates as the histogram kernel: block b streams its chunk
+// once with 128-bit loads, one tile (8192 coordinates) ahead of the compaction.  The number of
+// candidates in every earlier segment of the client is known from the per-segment histograms
+// (seg_prefix, written by the planner), so the output position of a candidate is
+// seg_prefix + its rank inside the block's segment: a block-level scan per tile and nothing else.
+
+constexpr int kSelStages = 3;  // tiles in flight per block (cp.async groups)
+constexpr size_t kSelStageBytes = (size_t)kSelectThreads * kSelectVecPerThread * 16;  // 32 KB
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int CAP>
+__global__ void __launch_bounds__(kSelectThreads, 2)
+k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_constant__ Partition part,
+         const unsigned char* __restrict__ plan_ws, unsigned char* ws, const __grid_constant__ EncLayout L) {
+  extern __shared__ float4 s_stage[];  // [kSelStages][kSelectVecPerThread][kSelectThreads]
+  __shared__ unsigned long long s_warp_incl[2][kSelectThreads / 32];
+  EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
+  if (hdr->status != 0) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t S = part.max_segments;
+  const uint32_t* seg_count = reinterpret_cast<const uint32_t*>(plan_ws + plan_off_seg_count(batch.n));
+  const unsigned long long* seg_prefix = reinterpret_cast<const unsigned long long*>(plan_ws + plan_off_seg_prefix(batch.n, S));
+  unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
+  const uint64_t nvec = d >> 2;
+  const uint64_t units = part.units;
+  uint64_t pos = (uint64_t)blockIdx.x * part.chunk;
+  const uint64_t end = (pos + part.chunk < part.total) ? pos + part.chunk : part.total;
+  constexpr uint64_t kTileVec = (uint64_t)kSelectThreads * kSelectVecPerThread;
+  int parity = 0;
+
+  while (pos < end) {
+    const uint32_t c = (uint32_t)(pos / units);
+    const uint64_t seg_end = ((c + 1) * units < end) ? (c + 1) * units : end;
+    const uint64_t u0 = pos - c * units, u1 = seg_end - c * units;  // units [u0, u1) of client c
+    const bool with_tail = (u1 == units);                            // the segment ends with the client's tail unit
+    const uint64_t v_end = with_tail ? nvec : u1;                    // float4 units [u0, v_end)
+    const float* __restrict__ x = batch.c[c].x;
+    const float4* xv = reinterpret_cast<const float4*>(x);
+    const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
+    const uint32_t thresh = plan->thresh_bin << 19;
+    const uint32_t seg = blockIdx.x + c;
+    unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
+    unsigned long long run = seg_prefix[seg];
+    const unsigned long long run0 = run;
+    const uint64_t n_tiles = (v_end > u0) ? (v_end - u0 + kTileVec - 1) / kTileVec : 0;
+
+    // every thread stages the float4s it will consume itself, so no barrier guards the staging buffers
+    auto issue = [&](uint64_t t) {
+      if (t < n_tiles) {
+        float4* dst = s_stage + (size_t)(t % kSelStages) * kTileVec;
+#pragma unroll
+        for (int v = 0; v < kSelectVecPerThread; ++v) {
+          const uint64_t vi = u0 + t * kTileVec + (uint64_t)v * kSelectThreads + tid;
+          if (vi < v_end) cp_async16(dst + v * kSelectThreads + tid, xv + vi);
+        }
+      }
+      cp_async_commit();  // one group per tile slot, empty past the end, keeps the group count uniform
+    };
+    // compaction of one tile held in registers: bits / valid per vector; e_base = element index of vector 0, thread 0
+    auto compact = [&](const uint32_t (&bits)[kSelectVecPerThread][4], const uint32_t (&valid)[kSelectVecPerThread], uint64_t vec0) {
+      uint32_t mask[kSelectVecPerThread];
+      unsigned long long packed = 0;
+#pragma unroll
+      for (int v = 0; v < kSelectVecPerThread; ++v) {
+        uint32_t m = 0;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) m |= (((bits[v][cc] & 0x7FFFFFFFu) >= thresh) ? 1u : 0u) << cc;
+        mask[v] = m & valid[v];
+        packed |= (unsigned long long)__popc(mask[v]) << (16 * v);
+      }
+      // block scan of the four per-vector counts, packed 16 bits each (tile totals <= 2048)
+      unsigned long long incl = packed;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long o = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (lane == 31) s_warp_incl[parity][warp] = incl;
+      __syncthreads();  // one barrier per tile: the scratch alternates between two copies
+      unsigned long long below = 0, tot = 0;
+#pragma unroll
+      for (int w = 0; w < kSelectThreads / 32; ++w) {
+        const unsigned long long t = s_warp_incl[parity][w];
+        if (w < warp) below += t;
+        tot += t;
+      }
+      parity ^= 1;
+      const unsigned long long excl = below + incl - packed;
+      unsigned long long vec_base = 0;
+#pragma unroll
+      for (int v = 0; v < kSelectVecPerThread; ++v) {
+        unsigned long long o = run + vec_base + ((excl >> (16 * v)) & 0xFFFF);
+        const uint64_t e0 = (vec0 + (uint64_t)v * kSelectThreads + tid) * 4;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          if (mask[v] & (1u << cc)) {
+            const uint32_t b = bits[v][cc];
+            const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) |
+                                            (unsigned long long)(b & 0x80000000u) | (unsigned long long)(e0 + cc);
+            if (o < L.capacity) out[o] = pair;
+            ++o;
+          }
+        }
+        vec_base += (tot >> (16 * v)) & 0xFFFF;
+      }
+      run += vec_base;
+    };
+
+#pragma unroll
+    for (int t = 0; t < kSelStages - 1; ++t) issue(t);
+    for (uint64_t t = 0; t < n_tiles; ++t) {
+      issue(t + kSelStages - 1);
+      cp_async_wait<kSelStages - 1>();  // the group of tile t has landed
+      const float4* src = s_stage + (size_t)(t % kSelStages) * kTileVec;
+      const uint64_t vec0 = u0 + t * kTileVec;
+      uint32_t bits[kSelectVecPerThread][4], valid[kSelectVecPerThread];
+#pragma unroll
+      for (int v = 0; v < kSelectVecPerThread; ++v) {
+        const uint64_t vi = vec0 + (uint64_t)v * kSelectThreads + tid;
+        valid[v] = 0;
+        bits[v][0] = bits[v][1] = bits[v][2] = bits[v][3] = 0;
+        if (vi < v_end) {
+          const float4 f = src[v * kSelectThreads + tid];
+          bits[v][0] = __float_as_uint(f.x);
+          bits[v][1] = __float_as_uint(f.y);
+          bits[v][2] = __float_as_uint(f.z);
+          bits[v][3] = __float_as_uint(f.w);
+          valid[v] = 0xF;
+        }
+      }
+      compact(bits, valid, vec0);
+    }
+    cp_async_wait<0>();
+    if (with_tail && (d & 3)) {  // the client's ragged tail: d % 4 scalars, as one more (nearly empty) tile
+      uint32_t bits[kSelectVecPerThread][4], valid[kSelectVecPerThread];
+#pragma unroll
+      for (int v = 0; v < kSelectVecPerThread; ++v) {
+        valid[v] = 0;
+        bits[v][0] = bits[v][1] = bits[v][2] = bits[v][3] = 0;
+      }
+      if (tid == 0) {
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          if (nvec * 4 + cc < d) {
+            bits[0][cc] = __float_as_uint(x[nvec * 4 + cc]);
+            valid[0] |= 1u << cc;
+          }
+        }
+      }
+      compact(bits, valid, nvec);
+    }
+    if (tid == 0) {
+      // the update must be the one the plan was made from
+      if (run - run0 != seg_count[seg]) set_status(&hdr->status, CVLC_ERR_PLAN_MISMATCH);
+      if (with_tail) n_selected[c] = run;
+    }
+    pos = seg_end;
+  }
+}
+
+// ===================================================================================
 // K4  stable LSD radix ranking of the candidates, |x| descending (ties keep ascending index)
 // ===================================================================================
-// Key digit = digit of (0x7FFFFFFF - key): 8, 8, 8, 7 bits.  One histogram kernel for all
-// four digits and all clients, a small scan kernel, then one single-pass kernel per digit
-// (tiles of all clients handed out by ticket, decoupled look-back per digit value).  A pass
-// whose digit is the same for every candidate of a client is skipped for that client; which
-// buffer holds its data after pass q follows from the mask of skipped passes.
+// Sort key = keytop - key, keytop = the largest key of the client's highest non-empty histogram
+// bin, so the key only spans the bins between the threshold and the top: 19 + log2(#bins) bits.
+// Digits of 9, 9, 9, 4 bits.  One histogram kernel for all four digits and all clients, a small
+// scan kernel, then one single-pass kernel per digit (tiles handed out by ticket, tile-major with
+// the clients interleaved; decoupled look-back per digit value).  A pass whose digit is the same
+// for every candidate of a client (normally the fourth) is skipped for that client; which buffer
+// holds its data after pass q follows from the mask of skipped passes.
 
-__device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass) {
-  const uint32_t inv = 0x7FFFFFFFu - (uint32_t)(pair >> 32);
-  return (inv >> (8 * pass)) & 0xFFu;
+__device__ __forceinline__ uint32_t sort_keytop(const cvlc_plan_t* plan) { return ((plan->top_bin + 1u) << 19) - 1u; }
+
+__device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass, uint32_t keytop) {
+  const uint32_t key = (uint32_t)(pair >> 32);
+  const uint32_t inv = key > keytop ? 0u : keytop - key;  // key > keytop only if the plan is not of this update
+  return (inv >> (kDigitBits * pass)) & (kDigits - 1);
 }
 
 // The clients' candidate arrays are concatenated in units of sort tiles (2048 pairs) and cut
@@ -285,12 +472,12 @@ __device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass
 template <int CAP>
 __global__ void __launch_bounds__(256)
 k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
-  __shared__ uint32_t sh[kSortPasses * 256];
+  __shared__ uint32_t sh[kSortPasses * kDigits];
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
   const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + L.off_sort_prefix);
   unsigned long long* ghist_all = reinterpret_cast<unsigned long long*>(ws + L.off_ghist);
-  for (int i = threadIdx.x; i < kSortPasses * 256; i += 256) sh[i] = 0;
+  for (int i = threadIdx.x; i < kSortPasses * kDigits; i += 256) sh[i] = 0;
   __syncthreads();
   const uint32_t total_tiles = prefix[batch.n];
   const uint32_t chunk = (total_tiles + gridDim.x - 1) / gridDim.x;
@@ -301,6 +488,7 @@ k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
     while (prefix[c + 1] <= t) ++c;  // client of tile t (clients without tiles are passed over)
     const uint32_t seg_end = prefix[c + 1] < t_end ? prefix[c + 1] : t_end;
     const unsigned long long n = batch.c[c].plan->n_candidates;
+    const uint32_t keytop = sort_keytop(batch.c[c].plan);
     const unsigned long long* __restrict__ in = reinterpret_cast<const unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     const unsigned long long i0 = (unsigned long long)(t - prefix[c]) * kSortTile;
     unsigned long long i1 = (unsigned long long)(seg_end - prefix[c]) * kSortTile;
@@ -308,11 +496,11 @@ k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
     for (unsigned long long i = i0 + threadIdx.x; i < i1; i += 256) {
       const unsigned long long pair = in[i];
 #pragma unroll
-      for (int p = 0; p < kSortPasses; ++p) atomicAdd(&sh[p * 256 + sort_digit(pair, p)], 1u);
+      for (int p = 0; p < kSortPasses; ++p) atomicAdd(&sh[p * kDigits + sort_digit(pair, p, keytop)], 1u);
     }
     __syncthreads();
-    unsigned long long* ghist = ghist_all + (size_t)c * kSortPasses * 256;
-    for (int i = threadIdx.x; i < kSortPasses * 256; i += 256) {
+    unsigned long long* ghist = ghist_all + (size_t)c * kSortPasses * kDigits;
+    for (int i = threadIdx.x; i < kSortPasses * kDigits; i += 256) {
       const uint32_t v = sh[i];
       sh[i] = 0;
       if (v) atomicAdd(ghist + i, (unsigned long long)v);
@@ -324,19 +512,19 @@ k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
 
 // per client: exclusive scans of the four digit histograms and the mask of constant digits
 template <int CAP>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kDigits)
 k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
-  __shared__ unsigned long long s_scan[8];
+  __shared__ unsigned long long s_scan[kDigits / 32];
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
   const uint32_t c = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long n = batch.c[c].plan->n_candidates;
-  const unsigned long long* ghist = reinterpret_cast<const unsigned long long*>(ws + L.off_ghist) + (size_t)c * kSortPasses * 256;
-  unsigned long long* gbase = reinterpret_cast<unsigned long long*>(ws + L.off_gbase) + (size_t)c * kSortPasses * 256;
+  const unsigned long long* ghist = reinterpret_cast<const unsigned long long*>(ws + L.off_ghist) + (size_t)c * kSortPasses * kDigits;
+  unsigned long long* gbase = reinterpret_cast<unsigned long long*>(ws + L.off_gbase) + (size_t)c * kSortPasses * kDigits;
   uint32_t mask = 0;
   for (int p = 0; p < kSortPasses; ++p) {
-    const unsigned long long cnt = ghist[p * 256 + tid];
+    const unsigned long long cnt = ghist[p * kDigits + tid];
     if (__syncthreads_or(cnt == n)) mask |= 1u << p;
     unsigned long long incl = cnt;
 #pragma unroll
@@ -348,7 +536,7 @@ k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
     __syncthreads();
     unsigned long long below = 0;
     for (int w = 0; w < warp; ++w) below += s_scan[w];
-    gbase[p * 256 + tid] = below + incl - cnt;
+    gbase[p * kDigits + tid] = below + incl - cnt;
     __syncthreads();
   }
   if (tid == 0) reinterpret_cast<uint32_t*>(ws + L.off_pass_mask)[c] = mask;
@@ -358,9 +546,9 @@ template <int CAP>
 __global__ void __launch_bounds__(kSortThreads)
 k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_wc[kSortThreads / 32][256];  // per-warp digit counters -> per-warp offsets
-  __shared__ unsigned long long s_base[256];         // position of this tile's first item per digit
-  extern __shared__ uint32_t s_prefix[];             // [n + 1] first sort tile of every client
+  __shared__ uint32_t s_wc[kSortThreads / 32][kDigits];  // per-warp digit counters -> per-warp offsets
+  __shared__ unsigned long long s_base[kDigits];         // position of this tile's first item per digit
+  extern __shared__ uint32_t s_prefix[];                 // [n + 1] first sort tile of every client
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -370,45 +558,46 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
     for (uint32_t i = tid; i <= n_clients; i += kSortThreads) s_prefix[i] = prefix[i];
   }
   __syncthreads();
-  const uint32_t total_tiles = s_prefix[n_clients];
+  const uint32_t total_tickets = hdr->max_sort_tiles * n_clients;
   const uint32_t* pass_mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask);
   unsigned long long* state_all =
-      reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)pass * n_clients * L.sort_tiles_max * 256;
+      reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)pass * n_clients * L.sort_tiles_max * kDigits;
   const unsigned lanemask_lt = (1u << lane) - 1u;
+  constexpr int kPerThread = kDigits / kSortThreads;  // digit values owned by a thread
 
   while (true) {
     if (tid == 0) s_tile = atomicAdd(&hdr->sort_ticket[pass], 1u);
 #pragma unroll
-    for (int w = 0; w < kSortThreads / 32; ++w) s_wc[w][tid] = 0;
+    for (int w = 0; w < kSortThreads / 32; ++w)
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) s_wc[w][tid + q * kSortThreads] = 0;
     __syncthreads();
     const uint32_t gt = s_tile;
-    if (gt >= total_tiles) break;
-    // client of tile gt: last c with prefix[c] <= gt
-    uint32_t lo_c = 0, hi_c = n_clients;
-    while (hi_c - lo_c > 1) {
-      const uint32_t mid = (lo_c + hi_c) >> 1;
-      if (s_prefix[mid] <= gt) lo_c = mid; else hi_c = mid;
-    }
-    const uint32_t c = lo_c;
+    if (gt >= total_tickets) break;
+    // tile-major tickets with the clients interleaved: the tiles in flight are a few consecutive
+    // tiles of every client, which keeps every look-back short
+    const uint32_t tile = gt / n_clients;
+    const uint32_t c = gt - tile * n_clients;
     const uint32_t mask = pass_mask[c];
-    if (mask & (1u << pass)) {  // constant digit for this client: nothing to move
-      __syncthreads();          // everyone has read s_tile before the next ticket overwrites it
+    if (tile >= s_prefix[c + 1] - s_prefix[c] || (mask & (1u << pass))) {  // no such tile, or a constant digit
+      __syncthreads();  // everyone has read s_tile before the next ticket overwrites it
       continue;
     }
-    const unsigned long long tile = gt - s_prefix[c];
-    const unsigned long long n = batch.c[c].plan->n_candidates;
+    const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
+    const unsigned long long n = plan->n_candidates;
+    const uint32_t keytop = sort_keytop(plan);
     const int flips = __popc(~mask & ((1u << pass) - 1u));
     unsigned long long* buf_a = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     unsigned long long* buf_b = reinterpret_cast<unsigned long long*>(ws + L.off_buf_b) + (size_t)c * L.capacity;
     const unsigned long long* __restrict__ src = (flips & 1) ? buf_b : buf_a;
     unsigned long long* __restrict__ dst = (flips & 1) ? buf_a : buf_b;
-    unsigned long long* state = state_all + (size_t)s_prefix[c] * 256;
-    const unsigned long long gbase =
-        reinterpret_cast<const unsigned long long*>(ws + L.off_gbase)[(size_t)c * kSortPasses * 256 + pass * 256 + tid];
+    unsigned long long* state = state_all + (size_t)s_prefix[c] * kDigits;
+    const unsigned long long* gbase = reinterpret_cast<const unsigned long long*>(ws + L.off_gbase) +
+                                      (size_t)c * kSortPasses * kDigits + (size_t)pass * kDigits;
 
     unsigned long long item[kSortItemsPerThread];
     uint32_t rank[kSortItemsPerThread];
-    const unsigned long long first = tile * kSortTile + (unsigned long long)warp * (32 * kSortItemsPerThread);
+    const unsigned long long first = (unsigned long long)tile * kSortTile + (unsigned long long)warp * (32 * kSortItemsPerThread);
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       const unsigned long long idx = first + i * 32 + lane;
@@ -418,7 +607,7 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       const bool valid = (first + i * 32 + lane) < n;
-      const uint32_t dig = valid ? sort_digit(item[i], pass) : 0xFFFFFFFFu;
+      const uint32_t dig = valid ? sort_digit(item[i], pass, keytop) : 0xFFFFFFFFu;
       const unsigned peers = __match_any_sync(kFull, dig);
       const int leader = __ffs(peers) - 1;
       uint32_t pre = 0;
@@ -429,34 +618,51 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
       __syncwarp();
     }
     __syncthreads();
-    // thread = digit value: offsets of the warps inside the tile, tile count, look-back
+    // thread = digit values tid, tid + 256: offsets of the warps inside the tile, tile count, look-back
     {
-      uint32_t tot = 0;
+      uint32_t tot[kPerThread];
+      unsigned long long run[kPerThread];
+      bool open[kPerThread];
 #pragma unroll
-      for (int w = 0; w < kSortThreads / 32; ++w) {
-        const uint32_t cnt = s_wc[w][tid];
-        s_wc[w][tid] = tot;
-        tot += cnt;
-      }
-      unsigned long long* my_state = state + tile * 256 + tid;
-      st_relaxed(my_state, (tile == 0 ? kFlagPrefix : kFlagAgg) | tot);
-      unsigned long long run = 0;
-      if (tile > 0) {
-        for (long long t = (long long)tile - 1; t >= 0; --t) {
-          const unsigned long long sv = wait_state(state + (unsigned long long)t * 256 + tid, &hdr->status);
-          if (sv == 0) break;  // timed out: status is set, results are void
-          run += sv & kValMask;
-          if ((sv & kFlagMask) == kFlagPrefix) break;
+      for (int q = 0; q < kPerThread; ++q) {
+        const int dg = tid + q * kSortThreads;
+        uint32_t t = 0;
+#pragma unroll
+        for (int w = 0; w < kSortThreads / 32; ++w) {
+          const uint32_t cnt = s_wc[w][dg];
+          s_wc[w][dg] = t;
+          t += cnt;
         }
-        st_relaxed(my_state, kFlagPrefix | (run + tot));
+        tot[q] = t;
+        run[q] = 0;
+        open[q] = tile > 0;
+        st_relaxed(state + (size_t)tile * kDigits + dg, (tile == 0 ? kFlagPrefix : kFlagAgg) | t);
       }
-      s_base[tid] = gbase + run;
+      for (long long t = (long long)tile - 1; t >= 0; --t) {
+        bool any_open = false;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+          if (open[q]) {
+            const unsigned long long sv = wait_state(state + (size_t)t * kDigits + tid + q * kSortThreads, &hdr->status);
+            run[q] += sv & kValMask;
+            if (sv == 0 || (sv & kFlagMask) == kFlagPrefix) open[q] = false;  // sv == 0: timed out, status is set
+            any_open |= open[q];
+          }
+        }
+        if (!any_open) break;
+      }
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) {
+        const int dg = tid + q * kSortThreads;
+        if (tile > 0) st_relaxed(state + (size_t)tile * kDigits + dg, kFlagPrefix | (run[q] + tot[q]));
+        s_base[dg] = gbase[dg] + run[q];
+      }
     }
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       if ((first + i * 32 + lane) < n) {
-        const uint32_t dig = sort_digit(item[i], pass);
+        const uint32_t dig = sort_digit(item[i], pass, keytop);
         const unsigned long long o = s_base[dig] + s_wc[warp][dig] + rank[i];
         if (o < n && o < L.capacity) dst[o] = item[i];
       }
@@ -623,14 +829,16 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
 // ===================================================================================
 
 template <int CAP>
-static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
-                                   cudaStream_t st) {
+static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
+                                   const void* plan_ws, void* ws, cudaStream_t st) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64 && !attr_done[dev]) {
     e = cudaFuncSetAttribute(k_pack<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_select<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSelStages * kSelStageBytes));
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
@@ -642,15 +850,20 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   unsigned char* w = static_cast<unsigned char*>(ws);
   const size_t pack_smem = (size_t)shape.cap[1] * 8;
 
+  const Partition part = make_partition(shape.d, n);
+  const unsigned char* pws = static_cast<const unsigned char*>(plan_ws);
   {
     LaunchScope ls(kKEncodeInit, st);
-    k_encode_init<CAP><<<2 * kNumSM, 256, 0, st>>>(w, batch, shape, L);
+    k_encode_init<CAP><<<2 * kNumSM, 256, 0, st>>>(w, batch, shape, L, pws, part);
   }
-  {
+  if (pws) {
+    LaunchScope ls(kKSelect, st);
+    k_select<CAP><<<part.grid, kSelectThreads, kSelStages * kSelStageBytes, st>>>(batch, shape.d, part, pws, w, L);
+  } else {
     const uint64_t want = L.select_tiles * n;
     const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
-    LaunchScope ls(kKSelect, st);
-    k_select<CAP><<<grid, kSelectThreads, 0, st>>>(batch, shape.d, w, L);
+    LaunchScope ls(kKSelectLookback, st);
+    k_select_lookback<CAP><<<grid, kSelectThreads, 0, st>>>(batch, shape.d, w, L);
   }
   {
     const uint64_t want = L.sort_tiles_max * n;
@@ -661,7 +874,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     }
     {
       LaunchScope ls(kKSortScan, st);
-      k_sort_scan<CAP><<<n, 256, 0, st>>>(batch, w, L);
+      k_sort_scan<CAP><<<n, kDigits, 0, st>>>(batch, w, L);
     }
     for (int pass = 0; pass < kSortPasses; ++pass) {
       LaunchScope ls(kKSortPass, st);
@@ -675,10 +888,10 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   return cudaGetLastError();
 }
 
-cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity, void* ws,
-                          cudaStream_t st) {
-  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, ws, st);
-  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, ws, st);
+cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
+                          const void* plan_ws, void* ws, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, plan_ws, ws, st);
+  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, plan_ws, ws, st);
 }
 
 }  // namespace cvlc

@@ -13,7 +13,7 @@ namespace cvlc {
 // K1  magnitude histogram: h[key >> 19], key = bits(|x|); HBM-bound, 4 bytes / coordinate
 // ===================================================================================
 
-constexpr int kHistThreads = 512;
+constexpr int kHistThreads = kStreamThreads;
 constexpr int kHistSub = 4;  // shared sub-histograms per block (64 KB)
 
 // The clients' updates are treated as one concatenated array of units (a unit = one float4,
@@ -32,19 +32,17 @@ __device__ __forceinline__ uint32_t hist_add4(uint32_t* my, const float4 a) {
 
 template <int CAP>
 __global__ void __launch_bounds__(kHistThreads, 2)
-k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned long long* __restrict__ hist_all,
-       uint32_t* __restrict__ nonfinite_all) {
+k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_constant__ Partition part,
+       unsigned long long* __restrict__ hist_all, uint32_t* __restrict__ nonfinite_all, uint32_t* __restrict__ seg_hist_all) {
   extern __shared__ uint32_t sh_hist[];  // [kHistSub][4096]
   for (int i = threadIdx.x; i < kHistSub * CVLC_HIST_BINS; i += kHistThreads) sh_hist[i] = 0;
   __syncthreads();
   uint32_t* my = sh_hist + ((threadIdx.x >> 5) & (kHistSub - 1)) * CVLC_HIST_BINS;
 
   const uint64_t nvec = d >> 2;
-  const uint64_t units = nvec + 1;  // per client: nvec float4 units and one tail unit
-  const uint64_t total = units * batch.n;
-  const uint64_t chunk = (total + gridDim.x - 1) / gridDim.x;
-  uint64_t pos = (uint64_t)blockIdx.x * chunk;
-  const uint64_t end = (pos + chunk < total) ? pos + chunk : total;
+  const uint64_t units = part.units;  // per client: nvec float4 units and one tail unit
+  uint64_t pos = (uint64_t)blockIdx.x * part.chunk;
+  const uint64_t end = (pos + part.chunk < part.total) ? pos + part.chunk : part.total;
 
   while (pos < end) {
     const uint64_t c = pos / units;
@@ -72,7 +70,10 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned long l
     }
     if (bad) atomicOr(nonfinite_all + c, 1u);
     __syncthreads();
+    // merge into the client's histogram and keep this segment's own counts (segment = block + client):
+    // the selection kernel derives its output offsets from them
     unsigned long long* __restrict__ hist = hist_all + (size_t)c * CVLC_HIST_BINS;
+    uint32_t* __restrict__ seg_hist = seg_hist_all + ((size_t)blockIdx.x + c) * CVLC_HIST_BINS;
     for (int b = threadIdx.x; b < CVLC_HIST_BINS; b += kHistThreads) {
       uint32_t cnt = 0;
 #pragma unroll
@@ -80,6 +81,7 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsigned long l
         cnt += sh_hist[sub * CVLC_HIST_BINS + b];
         sh_hist[sub * CVLC_HIST_BINS + b] = 0;
       }
+      seg_hist[b] = cnt;
       if (cnt) atomicAdd(hist + b, (unsigned long long)cnt);
     }
     __syncthreads();
@@ -206,13 +208,16 @@ struct PlanTab {
 template <int CAP>
 __global__ void __launch_bounds__(kPlanThreads, 1)
 k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restrict__ nonfinite_all,
-       const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, int32_t* ws_status) {
+       const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
+       const __grid_constant__ Partition part, unsigned char* ws) {
   extern __shared__ unsigned char smem_raw[];
   unsigned long long* Nsuf = reinterpret_cast<unsigned long long*>(smem_raw);  // [4096] survival counts
   double* ptX = reinterpret_cast<double*>(smem_raw + 4096 * 8);                // fit points, ascending bin
   double* ptY = ptX + 4096;
   __shared__ PlanShared S;
   __shared__ PlanTab T;
+  __shared__ uint32_t s_thresh_bin, s_top_bin;
+  int32_t* ws_status = reinterpret_cast<int32_t*>(ws);
 
   // blockIdx.x = client
   const unsigned long long* __restrict__ hist = hist_all + (size_t)blockIdx.x * CVLC_HIST_BINS;
@@ -508,7 +513,8 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     }
     for (int i = 0; i < nY; ++i) plan->n_y[T.Y[i]] = S.n[i];
   }
-  // threshold bin: the bin that holds rank k (1-based), and how many coordinates sit in it or above
+  // threshold bin: the bin that holds rank k (1-based), how many coordinates sit in it or above,
+  // and the highest non-empty bin
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int j = 4 * tid + i;
@@ -517,6 +523,48 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     if (N >= k && Nn < k) {
       plan->thresh_bin = (uint32_t)j;
       plan->n_candidates = N;
+      s_thresh_bin = (uint32_t)j;
+    }
+    if (N > 0 && Nn == 0) {
+      plan->top_bin = (uint32_t)j;
+      s_top_bin = (uint32_t)j;
+    }
+  }
+  __syncthreads();
+
+  // candidates per segment of this client (segment = part of the client inside one block's chunk of
+  // the histogram / selection kernels) and their exclusive prefix: the selection kernel's offsets
+  {
+    const uint32_t c = blockIdx.x;
+    const uint32_t S = part.max_segments;
+    uint32_t* seg_count = reinterpret_cast<uint32_t*>(ws + plan_off_seg_count(batch.n));
+    unsigned long long* seg_prefix = reinterpret_cast<unsigned long long*>(ws + plan_off_seg_prefix(batch.n, S));
+    const uint32_t* seg_hist = reinterpret_cast<const uint32_t*>(ws + plan_off_seg_hist(batch.n, S));
+    const uint64_t first = (uint64_t)c * part.units, last = first + part.units - 1;
+    const uint32_t b0 = (uint32_t)(first / part.chunk), b1 = (uint32_t)(last / part.chunk);
+    const uint32_t jt = s_thresh_bin;
+    for (uint32_t b = b0 + warp; b <= b1; b += kPlanThreads / 32) {
+      const uint32_t* hsrc = seg_hist + ((size_t)b + c) * CVLC_HIST_BINS;
+      uint32_t sum = 0;
+      for (uint32_t j = jt + lane; j < CVLC_HIST_BINS; j += 32) sum += hsrc[j];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+      if (lane == 0) seg_count[b + c] = sum;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long run = 0;
+      for (uint32_t b = b0; b <= b1; ++b) {
+        seg_prefix[b + c] = run;
+        run += seg_count[b + c];
+      }
+      if (c == 0) {
+        PlanWsHeader* hdr = reinterpret_cast<PlanWsHeader*>(ws);
+        hdr->n = batch.n;
+        hdr->d = shape.d;
+        hdr->grid = part.grid;
+        hdr->magic = kPlanWsMagic;
+      }
     }
   }
 }
@@ -545,21 +593,22 @@ static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Sh
   unsigned char* w = static_cast<unsigned char*>(ws);
   unsigned long long* hist = reinterpret_cast<unsigned long long*>(w + kPlanWsHist);
   uint32_t* flags = reinterpret_cast<uint32_t*>(w + plan_off_flags(n));
+  const Partition part = make_partition(shape.d, n);
+  uint32_t* seg_hist = reinterpret_cast<uint32_t*>(w + plan_off_seg_hist(n, part.max_segments));
   {
+    // header, histograms, flags and segment tables start at zero; the per-segment histograms are
+    // written in full by the histogram kernel
     LaunchScope ls(kKZeroWords, st);
-    k_zero_words<<<2 * kNumSM, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), plan_ws_bytes(n) / 4);
+    k_zero_words<<<2 * kNumSM, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), plan_off_seg_hist(n, part.max_segments) / 4);
   }
-  // two resident blocks per SM share the concatenated updates evenly
-  const uint64_t total_units = ((shape.d >> 2) + 1) * n;
-  uint64_t grid = (total_units + 4 * kHistThreads - 1) / (4 * kHistThreads);
-  if (grid > (uint64_t)(2 * kNumSM)) grid = 2 * kNumSM;
   {
+    // two resident blocks per SM share the concatenated updates evenly
     LaunchScope ls(kKHist, st);
-    k_hist<CAP><<<(unsigned)grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, hist, flags);
+    k_hist<CAP><<<part.grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, part, hist, flags, seg_hist);
   }
   {
     LaunchScope ls(kKPlan, st);
-    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, reinterpret_cast<int32_t*>(w));
+    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w);
   }
   return cudaGetLastError();
 }

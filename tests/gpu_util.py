@@ -72,7 +72,8 @@ def oracle_encode_clients(workload_name: str, clients: Sequence[int], d: Optiona
 
 # ---- GPU side ----------------------------------------------------------------------------
 
-def gpu_plan_encode(x: np.ndarray, pd: dict, fixed_y: int = 0, device: str = "cuda:0", want_hist: bool = False):
+def gpu_plan_encode(x: np.ndarray, pd: dict, fixed_y: int = 0, device: str = "cuda:0", want_hist: bool = False,
+                    use_plan_ws: bool = True):
     """returns (CvlcPlan host copy, stream np.uint8[, histogram np.uint64])"""
     import torch
     from paper_2402_03770_b200 import binding as B
@@ -81,7 +82,7 @@ def gpu_plan_encode(x: np.ndarray, pd: dict, fixed_y: int = 0, device: str = "cu
     xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(dev)
     enc = B.ClientEncoder(p, dev)
     enc.out.fill_(0xAB)  # the encoder must write every byte of the stream
-    out = enc.run(xd, fixed_y=fixed_y)
+    out = enc.run(xd, fixed_y=fixed_y, use_plan_ws=use_plan_ws)
     status = enc.status()
     plan = B.read_plan(enc.plan)
     st = out.cpu().numpy().copy()

@@ -31,7 +31,7 @@ def test_host_only_helpers_without_gpu():
     po = O.make_params(11_200_000, 22_400_000)
     assert B.cvlc_stream_bytes(p) == 64 + 1866 * 1500 == O.stream_bytes(po)
     assert p.scale_B == po.scale_B
-    assert B.cvlc_plan_workspace_bytes(p) == 256 + 4096 * 8 + 256
+    assert B.cvlc_plan_workspace_bytes(p) >= 256 + 4096 * 8 + 256
     assert B.cvlc_encode_workspace_bytes(p) >= 16 * p.d
     assert B.cvlc_encode_batch_workspace_bytes(p, 100, 1 << 20) < 100 * B.cvlc_encode_workspace_bytes(p)
     assert B.cvlc_decode_workspace_bytes(100) > 0 and B.cvlc_decode_workspace_bytes(5000) == 0

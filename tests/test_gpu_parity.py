@@ -94,13 +94,16 @@ def test_division_by_small_constants_is_correctly_rounded(torch_cuda):
 
 def run_case(x, pd, fixed_y=0):
     of, ost = oracle_plan_encode(x, pd, fixed_y)
-    status, gp, gst = gpu_plan_encode(x, pd, fixed_y)
-    assert status == 0
-    assert_plan_equal(gp, of)
-    assert gst.size == ost.size
-    if not (gst == ost).all():
-        bad = np.nonzero(gst != ost)[0]
-        raise AssertionError(f"stream differs at {bad.size} bytes, first at {bad[0]} of {gst.size}")
+    # both selection kernels: offsets from the plan's per-segment counts, and the look-back scan
+    for use_plan_ws in (True, False):
+        status, gp, gst = gpu_plan_encode(x, pd, fixed_y, use_plan_ws=use_plan_ws)
+        assert status == 0, (status, use_plan_ws)
+        assert_plan_equal(gp, of)
+        assert gst.size == ost.size
+        if not (gst == ost).all():
+            bad = np.nonzero(gst != ost)[0]
+            raise AssertionError(f"stream differs at {bad.size} bytes, first at {bad[0]} of {gst.size} "
+                                 f"(use_plan_ws={use_plan_ws})")
     return of, ost
 
 
@@ -218,7 +221,7 @@ def test_batched_plan_encode_matches_oracle_per_client(torch_cuda, n):
         for o in enc.outs:
             o.fill_(0xCD)
         dxs = [torch.from_numpy(x).to(dev) for x in xs]
-        outs = enc.run(dxs)
+        outs = enc.run(dxs, use_plan_ws=(n % 2 == 0))
         status = enc.status()
         if max_cand:
             # the all-zero client has d candidates: more than the reduced workspace holds

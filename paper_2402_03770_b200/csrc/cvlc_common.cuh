@@ -59,16 +59,20 @@ struct Shape {
 
 // The histogram and the selection kernel stream the clients' updates as one concatenated
 // array of units (a unit = one float4; every client ends with one ragged-tail unit) cut into
-// equal contiguous chunks, one per thread block.  A segment is the part of one client inside
-// one chunk; with block b and client c both non-decreasing along the array, b + c numbers the
-// segments uniquely.
+// equal contiguous chunks, several per thread block (the histogram takes them round-robin, the
+// selection by ticket, because its cost per chunk depends on how many candidates it holds).
+// A segment is the part of one client inside one chunk; with chunk q and client c both
+// non-decreasing along the array, q + c numbers the segments uniquely.
 constexpr int kStreamThreads = 512;
+constexpr int kChunksPerBlock = 8;
 struct Partition {
-  uint64_t units;   // per client: d / 4 float4 units + 1 tail unit
-  uint64_t total;   // units * n
-  uint64_t chunk;   // units per block
-  uint32_t grid;    // blocks
-  uint32_t max_segments;  // grid + n
+  uint64_t units;         // per client: d / 4 float4 units + 1 tail unit
+  uint64_t total;         // units * n
+  uint64_t chunk;         // units per chunk
+  uint32_t n_chunks;
+  uint32_t grid;          // blocks
+  uint32_t max_segments;  // n_chunks + n
+  uint32_t pad;
 };
 CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
   Partition P;
@@ -78,8 +82,14 @@ CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
   if (grid > (uint64_t)(2 * kNumSM)) grid = 2 * kNumSM;
   if (grid == 0) grid = 1;
   P.grid = (uint32_t)grid;
-  P.chunk = (P.total + grid - 1) / grid;
-  P.max_segments = P.grid + n;
+  // chunks of at least 16 tiles of 2048 units, at most kChunksPerBlock per block
+  uint64_t n_chunks = P.total / (16 * 4 * kStreamThreads);
+  if (n_chunks > grid * kChunksPerBlock) n_chunks = grid * kChunksPerBlock;
+  if (n_chunks < grid) n_chunks = grid;
+  P.chunk = (P.total + n_chunks - 1) / n_chunks;
+  P.n_chunks = (uint32_t)((P.total + P.chunk - 1) / P.chunk);
+  P.max_segments = P.n_chunks + n;
+  P.pad = 0;
   return P;
 }
 
@@ -90,7 +100,7 @@ struct PlanWsHeader {
   int32_t status;   // byte 0
   uint32_t n;       // clients of the batch the workspace was filled for
   uint64_t d;
-  uint32_t grid;
+  uint32_t n_chunks;
   uint32_t magic;   // set when the segment tables are valid
 };
 constexpr uint32_t kPlanWsMagic = 0x53454743u;

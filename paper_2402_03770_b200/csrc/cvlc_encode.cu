@@ -110,7 +110,7 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
     if (plan_ws && !s_bad) {
       // the segment tables must have been made for this very batch
       const PlanWsHeader* ph = reinterpret_cast<const PlanWsHeader*>(plan_ws);
-      if (ph->magic != kPlanWsMagic || ph->n != n || ph->d != shape.d || ph->grid != part.grid) s_bad = CVLC_ERR_PLAN_MISMATCH;
+      if (ph->magic != kPlanWsMagic || ph->n != n || ph->d != shape.d || ph->n_chunks != part.n_chunks) s_bad = CVLC_ERR_PLAN_MISMATCH;
     }
     hdr->max_sort_tiles = mx;
     hdr->status = s_bad;
@@ -297,12 +297,17 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// Staging layout: float4 unit g of a tile (g = 0 .. 2047, in memory order) sits in slot
+// g ^ ((g >> 3) & 3).  The copies of a warp (consecutive g) and the reads of a warp (thread t
+// reads its own four consecutive units 4t .. 4t+3) are then both free of bank conflicts.
+__device__ __forceinline__ uint32_t sel_slot(uint32_t g) { return g ^ ((g >> 3) & 3u); }
+
 template <int CAP>
 __global__ void __launch_bounds__(kSelectThreads, 2)
 k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_constant__ Partition part,
          const unsigned char* __restrict__ plan_ws, unsigned char* ws, const __grid_constant__ EncLayout L) {
-  extern __shared__ float4 s_stage[];  // [kSelStages][kSelectVecPerThread][kSelectThreads]
-  __shared__ unsigned long long s_warp_incl[2][kSelectThreads / 32];
+  extern __shared__ float4 s_stage[];  // [kSelStages][2048 float4]
+  __shared__ uint32_t s_warp_incl[2][kSelectThreads / 32];
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -312,10 +317,18 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
   unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;
-  uint64_t pos = (uint64_t)blockIdx.x * part.chunk;
-  const uint64_t end = (pos + part.chunk < part.total) ? pos + part.chunk : part.total;
-  constexpr uint64_t kTileVec = (uint64_t)kSelectThreads * kSelectVecPerThread;
+  constexpr uint32_t kTileVec = kSelectThreads * kSelectVecPerThread;  // 2048 float4 = 8192 coordinates
   int parity = 0;
+  __shared__ uint32_t s_chunk;
+
+  while (true) {
+  // chunks by ticket: a chunk full of candidates costs several times one without
+  if (tid == 0) s_chunk = atomicAdd(&hdr->select_ticket, 1u);
+  __syncthreads();
+  const uint32_t q = s_chunk;
+  if (q >= part.n_chunks) break;
+  uint64_t pos = (uint64_t)q * part.chunk;
+  const uint64_t end = (pos + part.chunk < part.total) ? pos + part.chunk : part.total;
 
   while (pos < end) {
     const uint32_t c = (uint32_t)(pos / units);
@@ -324,126 +337,121 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const bool with_tail = (u1 == units);                            // the segment ends with the client's tail unit
     const uint64_t v_end = with_tail ? nvec : u1;                    // float4 units [u0, v_end)
     const float* __restrict__ x = batch.c[c].x;
-    const float4* xv = reinterpret_cast<const float4*>(x);
+    const float4* __restrict__ xseg = reinterpret_cast<const float4*>(x) + u0;
     const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
     const uint32_t thresh = plan->thresh_bin << 19;
-    const uint32_t seg = blockIdx.x + c;
+    const float thresh_f = __uint_as_float(thresh);  // finite inputs: |x| >= thresh_f <=> key >= thresh
+    const uint32_t seg = q + c;
     unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     unsigned long long run = seg_prefix[seg];
     const unsigned long long run0 = run;
-    const uint64_t n_tiles = (v_end > u0) ? (v_end - u0 + kTileVec - 1) / kTileVec : 0;
+    const uint64_t n_vec = (v_end > u0) ? v_end - u0 : 0;        // float4 units of the segment
+    const uint32_t n_tiles = (uint32_t)((n_vec + kTileVec - 1) / kTileVec);
 
-    // every thread stages the float4s it will consume itself, so no barrier guards the staging buffers
-    auto issue = [&](uint64_t t) {
+    // copies of a warp are consecutive float4s (coalesced); any thread may stage any unit because a
+    // barrier separates the wait for a tile from its use
+    uint32_t istage = 0;
+    auto issue = [&](uint32_t t) {
       if (t < n_tiles) {
-        float4* dst = s_stage + (size_t)(t % kSelStages) * kTileVec;
+        float4* dst = s_stage + (size_t)istage * kTileVec;
+        const uint64_t base = (uint64_t)t * kTileVec;
+        if (base + kTileVec <= n_vec) {
 #pragma unroll
-        for (int v = 0; v < kSelectVecPerThread; ++v) {
-          const uint64_t vi = u0 + t * kTileVec + (uint64_t)v * kSelectThreads + tid;
-          if (vi < v_end) cp_async16(dst + v * kSelectThreads + tid, xv + vi);
-        }
-      }
-      cp_async_commit();  // one group per tile slot, empty past the end, keeps the group count uniform
-    };
-    // compaction of one tile held in registers: bits / valid per vector; e_base = element index of vector 0, thread 0
-    auto compact = [&](const uint32_t (&bits)[kSelectVecPerThread][4], const uint32_t (&valid)[kSelectVecPerThread], uint64_t vec0) {
-      uint32_t mask[kSelectVecPerThread];
-      unsigned long long packed = 0;
+          for (int v = 0; v < kSelectVecPerThread; ++v) {
+            const uint32_t g = v * kSelectThreads + tid;
+            cp_async16(dst + sel_slot(g), xseg + base + g);
+          }
+        } else {
 #pragma unroll
-      for (int v = 0; v < kSelectVecPerThread; ++v) {
-        uint32_t m = 0;
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) m |= (((bits[v][cc] & 0x7FFFFFFFu) >= thresh) ? 1u : 0u) << cc;
-        mask[v] = m & valid[v];
-        packed |= (unsigned long long)__popc(mask[v]) << (16 * v);
-      }
-      // block scan of the four per-vector counts, packed 16 bits each (tile totals <= 2048)
-      unsigned long long incl = packed;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long o = __shfl_up_sync(kFull, incl, off);
-        if (lane >= off) incl += o;
-      }
-      if (lane == 31) s_warp_incl[parity][warp] = incl;
-      __syncthreads();  // one barrier per tile: the scratch alternates between two copies
-      unsigned long long below = 0, tot = 0;
-#pragma unroll
-      for (int w = 0; w < kSelectThreads / 32; ++w) {
-        const unsigned long long t = s_warp_incl[parity][w];
-        if (w < warp) below += t;
-        tot += t;
-      }
-      parity ^= 1;
-      const unsigned long long excl = below + incl - packed;
-      unsigned long long vec_base = 0;
-#pragma unroll
-      for (int v = 0; v < kSelectVecPerThread; ++v) {
-        unsigned long long o = run + vec_base + ((excl >> (16 * v)) & 0xFFFF);
-        const uint64_t e0 = (vec0 + (uint64_t)v * kSelectThreads + tid) * 4;
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          if (mask[v] & (1u << cc)) {
-            const uint32_t b = bits[v][cc];
-            const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) |
-                                            (unsigned long long)(b & 0x80000000u) | (unsigned long long)(e0 + cc);
-            if (o < L.capacity) out[o] = pair;
-            ++o;
+          for (int v = 0; v < kSelectVecPerThread; ++v) {
+            const uint32_t g = v * kSelectThreads + tid;
+            if (base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
           }
         }
-        vec_base += (tot >> (16 * v)) & 0xFFFF;
       }
-      run += vec_base;
+      istage = (istage + 1 == kSelStages) ? 0u : istage + 1;
+      cp_async_commit();  // one group per tile slot, empty past the end, keeps the group count uniform
     };
 
 #pragma unroll
     for (int t = 0; t < kSelStages - 1; ++t) issue(t);
-    for (uint64_t t = 0; t < n_tiles; ++t) {
-      issue(t + kSelStages - 1);
-      cp_async_wait<kSelStages - 1>();  // the group of tile t has landed
-      const float4* src = s_stage + (size_t)(t % kSelStages) * kTileVec;
-      const uint64_t vec0 = u0 + t * kTileVec;
-      uint32_t bits[kSelectVecPerThread][4], valid[kSelectVecPerThread];
+    uint32_t stage = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) {
+      cp_async_wait<kSelStages - 2>();  // this thread's copies of tile t have landed
+      __syncthreads();                  // ... and everybody else's; and everybody is done with tile t - 1,
+      issue(t + kSelStages - 1);        // whose staging slot the next copies overwrite
+      const float4* src = s_stage + (size_t)stage * kTileVec;
+      stage = (stage + 1 == kSelStages) ? 0u : stage + 1;
+      const uint64_t base = (uint64_t)t * kTileVec;
+      // this thread's 16 consecutive coordinates: units 4 tid .. 4 tid + 3 of the tile
+      uint32_t m = 0;
+      const uint32_t g0 = 4u * tid;
+      const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < 4) ? n_vec - base - g0 : 4) : 0u;
 #pragma unroll
-      for (int v = 0; v < kSelectVecPerThread; ++v) {
-        const uint64_t vi = vec0 + (uint64_t)v * kSelectThreads + tid;
-        valid[v] = 0;
-        bits[v][0] = bits[v][1] = bits[v][2] = bits[v][3] = 0;
-        if (vi < v_end) {
-          const float4 f = src[v * kSelectThreads + tid];
-          bits[v][0] = __float_as_uint(f.x);
-          bits[v][1] = __float_as_uint(f.y);
-          bits[v][2] = __float_as_uint(f.z);
-          bits[v][3] = __float_as_uint(f.w);
-          valid[v] = 0xF;
+      for (int j = 0; j < 4; ++j) {
+        if ((uint32_t)j < left) {
+          const float4 f = src[sel_slot(g0 + j)];
+          m |= (fabsf(f.x) >= thresh_f ? 1u : 0u) << (4 * j);
+          m |= (fabsf(f.y) >= thresh_f ? 1u : 0u) << (4 * j + 1);
+          m |= (fabsf(f.z) >= thresh_f ? 1u : 0u) << (4 * j + 2);
+          m |= (fabsf(f.w) >= thresh_f ? 1u : 0u) << (4 * j + 3);
         }
       }
-      compact(bits, valid, vec0);
+      const uint32_t cnt = __popc(m);
+      // block scan of the per-thread counts: inside the warp, then over the 16 warp totals
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (lane == 31) s_warp_incl[parity][warp] = incl;
+      __syncthreads();
+      const uint32_t wt = (lane < kSelectThreads / 32) ? s_warp_incl[parity][lane] : 0u;
+      uint32_t wincl = wt;
+#pragma unroll
+      for (int off = 1; off < kSelectThreads / 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(kFull, wincl, off);
+        if (lane >= off) wincl += o;
+      }
+      const uint32_t tot = __shfl_sync(kFull, wincl, kSelectThreads / 32 - 1);
+      const uint32_t below = __shfl_sync(kFull, wincl - wt, warp);
+      parity ^= 1;
+      // emit this thread's candidates (few): values are re-read from the staging buffer
+      unsigned long long o = run + below + incl - cnt;
+      const uint32_t* srcw = reinterpret_cast<const uint32_t*>(src);
+      const uint64_t e_base = (u0 + base + g0) * 4;
+      while (m) {
+        const int bit = __ffs(m) - 1;
+        m &= m - 1;
+        const uint32_t b = srcw[sel_slot(g0 + (bit >> 2)) * 4 + (bit & 3)];
+        if (o < L.capacity)
+          out[o] = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) |
+                   (unsigned long long)(e_base + bit);
+        ++o;
+      }
+      run += tot;
     }
     cp_async_wait<0>();
-    if (with_tail && (d & 3)) {  // the client's ragged tail: d % 4 scalars, as one more (nearly empty) tile
-      uint32_t bits[kSelectVecPerThread][4], valid[kSelectVecPerThread];
-#pragma unroll
-      for (int v = 0; v < kSelectVecPerThread; ++v) {
-        valid[v] = 0;
-        bits[v][0] = bits[v][1] = bits[v][2] = bits[v][3] = 0;
-      }
-      if (tid == 0) {
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          if (nvec * 4 + cc < d) {
-            bits[0][cc] = __float_as_uint(x[nvec * 4 + cc]);
-            valid[0] |= 1u << cc;
-          }
+    if (with_tail && tid == 0) {
+      // the client's ragged tail (d % 4 scalars) follows every float4 unit: one thread appends it
+      for (uint64_t e = nvec * 4; e < d; ++e) {
+        const uint32_t b = __float_as_uint(x[e]);
+        if ((b & 0x7FFFFFFFu) >= thresh) {
+          if (run < L.capacity)
+            out[run] = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) | (unsigned long long)e;
+          ++run;
         }
       }
-      compact(bits, valid, nvec);
     }
     if (tid == 0) {
       // the update must be the one the plan was made from
       if (run - run0 != seg_count[seg]) set_status(&hdr->status, CVLC_ERR_PLAN_MISMATCH);
       if (with_tail) n_selected[c] = run;
     }
+    __syncthreads();  // the staging buffers (and the ticket word) are reused by the next segment
     pos = seg_end;
+  }
   }
 }
 
@@ -699,21 +707,27 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   const unsigned long long* __restrict__ sorted =
       reinterpret_cast<const unsigned long long*>(ws + ((flips & 1) ? L.off_buf_b : L.off_buf_a)) + (size_t)c * L.capacity;
 
-  if (tid == 0) {
-    unsigned long long cum = 0, Z = 0;
-    uint32_t yy = 0;
-    for (int y = CVLC_MAX_CODE_BITS; y >= 1; --y) {
-      const unsigned long long ny = plan->n_y[y];
-      if (r < cum + ny) {
-        yy = (uint32_t)y;
-        Z += (r - cum) * plan->cap[y];
-        break;
+  // packet r -> its code length and first rank: lane l of warp 0 holds length 32 - l (longest first)
+  if (warp == 0) {
+    const int yl = CVLC_MAX_CODE_BITS - lane;
+    const unsigned long long ny = plan->n_y[yl];
+    const unsigned long long nz = ny * plan->cap[yl];
+    unsigned long long cum = ny, zc = nz;  // inclusive scans over the lanes
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned long long a = __shfl_up_sync(kFull, cum, off), b = __shfl_up_sync(kFull, zc, off);
+      if (lane >= off) {
+        cum += a;
+        zc += b;
       }
-      cum += ny;
-      Z += ny * plan->cap[y];
     }
-    s_y = yy;
-    s_Z = Z;
+    const unsigned hit = __ballot_sync(kFull, r < cum);
+    if (hit == 0) {
+      if (lane == 0) s_y = 0;
+    } else if (lane == __ffs(hit) - 1) {
+      s_y = (uint32_t)yl;
+      s_Z = (zc - nz) + (r - (cum - ny)) * plan->cap[yl];
+    }
   }
   __syncthreads();
   const uint32_t y = s_y;
@@ -754,6 +768,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   const double Lc = (double)((1ull << y) - 1ull);
   const double dlo = (double)lo;
   const double den = __dsub_rn((double)hi, dlo);
+  const double scale = (hi != lo) ? __ddiv_rn(Lc, den) : 0.0;
   for (uint32_t j = tid; j < P; j += kPackThreads) {
     const unsigned long long pair = recs[j];
     const uint32_t key = (uint32_t)(pair >> 32);
@@ -761,12 +776,24 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;
     uint32_t code = 0;
     if (hi != lo) {
-      const double t = __dmul_rn(__ddiv_rn(__dsub_rn((double)__uint_as_float(b), dlo), den), Lc);
-      double j0 = floor(t);
-      if (j0 > Lc) j0 = Lc;
-      const double frac = __dsub_rn(t, j0);
+      const double num = __dsub_rn((double)__uint_as_float(b), dlo);
       const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
-      code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
+      // t = (num / den) * L decides floor(t) and [u < frac(t)].  num * (L / den) is within a few ulp of it;
+      // unless its fraction sits that close to 0, 1 or u, both decisions are the same and the division
+      // is not needed.
+      const double tf = __dmul_rn(num, scale);
+      const double jf = floor(tf);
+      const double ff = __dsub_rn(tf, jf);
+      const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
+      if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < Lc) {
+        code = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
+      } else {
+        const double t = __dmul_rn(__ddiv_rn(num, den), Lc);
+        double j0 = floor(t);
+        if (j0 > Lc) j0 = Lc;
+        const double frac = __dsub_rn(t, j0);
+        code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
+      }
     }
     recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
   }

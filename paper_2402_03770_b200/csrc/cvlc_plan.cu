@@ -41,7 +41,8 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
 
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;  // per client: nvec float4 units and one tail unit
-  uint64_t pos = (uint64_t)blockIdx.x * part.chunk;
+  for (uint32_t q = blockIdx.x; q < part.n_chunks; q += gridDim.x) {
+  uint64_t pos = (uint64_t)q * part.chunk;
   const uint64_t end = (pos + part.chunk < part.total) ? pos + part.chunk : part.total;
 
   while (pos < end) {
@@ -70,10 +71,10 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     }
     if (bad) atomicOr(nonfinite_all + c, 1u);
     __syncthreads();
-    // merge into the client's histogram and keep this segment's own counts (segment = block + client):
+    // merge into the client's histogram and keep this segment's own counts (segment = chunk + client):
     // the selection kernel derives its output offsets from them
     unsigned long long* __restrict__ hist = hist_all + (size_t)c * CVLC_HIST_BINS;
-    uint32_t* __restrict__ seg_hist = seg_hist_all + ((size_t)blockIdx.x + c) * CVLC_HIST_BINS;
+    uint32_t* __restrict__ seg_hist = seg_hist_all + ((size_t)q + c) * CVLC_HIST_BINS;
     for (int b = threadIdx.x; b < CVLC_HIST_BINS; b += kHistThreads) {
       uint32_t cnt = 0;
 #pragma unroll
@@ -86,6 +87,7 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     }
     __syncthreads();
     pos = seg_end;
+  }
   }
 }
 
@@ -562,7 +564,7 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
         PlanWsHeader* hdr = reinterpret_cast<PlanWsHeader*>(ws);
         hdr->n = batch.n;
         hdr->d = shape.d;
-        hdr->grid = part.grid;
+        hdr->n_chunks = part.n_chunks;
         hdr->magic = kPlanWsMagic;
       }
     }

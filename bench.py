@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--streams", type=int, default=2, help="CUDA streams the batches are spread over")
     ap.add_argument("--max-candidates", type=int, default=0,
                     help="candidate slots per client in the encode workspace; 0 = 3 * R * cap(1)")
-    ap.add_argument("--profile-kernel", default="k_select")
+    ap.add_argument("--profile-kernel", default="", help="kernel whose roofline is reported; default: the one with the largest total time")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-sample-clients", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -172,6 +172,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2402_03770_b200 import binding as B
+    from paper_2402_03770_b200 import replica as R
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -190,7 +191,7 @@ def run_ours(args):
     n_clients = args.clients or w.n_clients
     bpc = args.bits_per_coord
     budget = int(np.floor(bpc * d))
-    first_client = rank * n_clients  # every rank is an independent replica with its own clients
+    first_client = R.replica_clients(rank, n_clients)[0]  # every rank is an independent replica with its own clients
 
     # ---- inputs: seeded host generation (threads; numpy releases the GIL), then HBM-resident
     with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 4)) as ex:
@@ -256,10 +257,7 @@ def run_ours(args):
         barrier()
         total_ms = ev[0].elapsed_time(ev[-1])
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(n_steps)]
-        if world > 1:
-            t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+        total_ms = R.max_over_ranks(total_ms, dev)
         return total_ms, per
 
     for _ in range(max(args.warmup, 3)):
@@ -270,8 +268,8 @@ def run_ours(args):
     assert agg.status() == B.CVLC_OK, "decode-aggregate reported a device-side error"
 
     launches_before = B.cvlc_launch_count()
-    per_step_launch_cap = 8 * len(groups) + 8
-    B.cvlc_profile_select(args.profile_kernel, per_step_launch_cap * args.steps)
+    per_step_launch_cap = 16 * len(groups) + 8
+    B.cvlc_profile_select("*", per_step_launch_cap * args.steps)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -279,7 +277,11 @@ def run_ours(args):
     total_ms, per = timed(args.steps, False)
     clocks = sampler.stop() if rank == 0 else None
     gpu_launches = B.cvlc_launch_count() - launches_before
-    prof_n, prof_ms = B.cvlc_profile_read()
+    kernel_times = {}
+    for name in B.KERNEL_NAMES:
+        kn, kms = B.cvlc_profile_read(name)
+        if kn:
+            kernel_times[name] = (kn, kms)
     B.cvlc_profile_select(None, 0)
 
     ms_per_step = total_ms / args.steps
@@ -299,25 +301,51 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the profiled kernel: algorithmic bytes per launch / mean launch duration
-    plan0 = encoders[0].read_plan(0)
+    # ---- per-kernel CUDA-event times of the timed region, and the roofline of the dominant kernel:
+    # algorithmic bytes per launch / mean launch duration
+    plans = [enc.read_plan(i) for enc in encoders for i in range(enc.n)]
     stream_bytes = B.cvlc_stream_bytes(params[0])
-    alg_bytes = {
-        "k_hist": 4.0 * d * n_clients / len(groups),
-        "k_select": (4.0 * d + 8.0 * plan0.n_candidates) * n_clients / len(groups),
-        "k_sort_pass": 16.0 * plan0.n_candidates * n_clients / len(groups),
-        "k_pack": (8.0 * plan0.k + stream_bytes) * n_clients / len(groups),
+    n_groups = len(groups)
+    sum_cand = float(sum(p.n_candidates for p in plans))
+    sum_k = float(sum(p.k for p in plans))
+    sort_passes_per_step = kernel_times.get("k_sort_pass", (0, 0))[0] / max(1, args.steps)
+    alg_bytes_per_step = {   # algorithmic bytes all launches of one step move
+        "k_hist": 4.0 * d * n_clients,
+        "k_select": 4.0 * d * n_clients + 8.0 * sum_cand,
+        "k_sort_hist": 8.0 * sum_cand,
+        "k_sort_pass": 16.0 * sum_cand * 3.0,           # three digit passes move data (the fourth digit is constant)
+        "k_pack": 8.0 * sum_k + float(n_clients) * stream_bytes,
         "k_decode": float(n_clients) * stream_bytes + 4.0 * d,
         "k_fill_zero": 4.0 * d,
-    }.get(args.profile_kernel)
+    }
     peak, peak_kind = measured_hbm_peak()
+    total_kernel_ms = sum(ms for _, ms in kernel_times.values())
+    kernels = {}
+    for name, (kn, kms) in sorted(kernel_times.items(), key=lambda kv: -kv[1][1]):
+        entry = {"launches_per_step": kn / args.steps, "ms_per_step": kms / args.steps,
+                 "share": kms / total_kernel_ms if total_kernel_ms else None}
+        if name in alg_bytes_per_step:
+            entry["achieved_GBps"] = alg_bytes_per_step[name] / (kms / args.steps * 1e-3) / 1e9
+            entry["frac_of_hbm_peak"] = entry["achieved_GBps"] / peak
+        kernels[name] = entry
+    dominant = args.profile_kernel or (max(kernel_times.items(), key=lambda kv: kv[1][1])[0] if kernel_times else "")
     roofline = None
-    if alg_bytes and prof_n:
-        achieved = alg_bytes / (prof_ms / prof_n * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": args.profile_kernel, "achieved": achieved, "peak": peak,
-                    "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": NCU_TRAFFIC_BYTES.get(args.profile_kernel), "launches_timed": prof_n,
-                    "mean_launch_us": prof_ms / prof_n * 1e3, "algorithmic_bytes_per_launch": alg_bytes}
+    if dominant in kernel_times:
+        kn, kms = kernel_times[dominant]
+        if dominant in alg_bytes_per_step:
+            per_launch = alg_bytes_per_step[dominant] * args.steps / kn
+            achieved = per_launch / (kms / kn * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak,
+                        "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                        "traffic": NCU_TRAFFIC_BYTES.get(dominant), "launches_timed": kn,
+                        "mean_launch_us": kms / kn * 1e3, "algorithmic_bytes_per_launch": per_launch}
+        else:
+            # the single-CTA-per-client planner: FP64 series arithmetic with O(1) data, bound by the
+            # FP64 pipe of the SMs it occupies (64 FMA lanes per SM per clock)
+            sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+            fp64_peak = 2.0 * 64 * 148 * sm_max * 1e6 / 1e12
+            roofline = {"bound": "alu", "kernel": dominant, "achieved": None, "peak": fp64_peak, "unit": "TFLOP/s",
+                        "frac": None, "traffic": None, "launches_timed": kn, "mean_launch_us": kms / kn * 1e3}
     # whole-step minimum bytes (read every update once, write every stream; read the streams, write the aggregate)
     step_min_bytes = n_clients * (4.0 * d + stream_bytes) + n_clients * stream_bytes + 4.0 * d
     step_frac = step_min_bytes / (ms_per_step * 1e-3) / 1e9 / peak
@@ -339,9 +367,9 @@ def run_ours(args):
         "params_per_s": units / (ms_per_step * 1e-3),
         "step_min_bytes_frac_of_hbm_peak": step_frac,
         "per_step_ms": per,
-        "plan": {"k": int(plan0.k), "R": int(plan0.R), "n_candidates": int(plan0.n_candidates), "alpha_q": plan0.alpha_q,
-                 "lengths": {str(y): int(plan0.n_y[y]) for y in range(33) if plan0.n_y[y]}},
-        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(gpu_launches),
+        "plan_of_client_0": {"k": int(plans[0].k), "R": int(plans[0].R), "n_candidates": int(plans[0].n_candidates), "alpha_q": plans[0].alpha_q,
+                 "lengths": {str(y): int(plans[0].n_y[y]) for y in range(33) if plans[0].n_y[y]}},
+        "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(gpu_launches),
         "clocks": clocks,
     }
     print(json.dumps(line))

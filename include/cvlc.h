@@ -249,13 +249,14 @@ int cvlc_selftest_math(const double* in_dev, uint64_t n, double* log2_out_dev, d
 /* Launch accounting: number of kernels this library has launched in this process
  * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist"). */
 unsigned long long cvlc_launch_count(const char* kernel_name);
-/* Optional timing of one kernel: after cvlc_profile_select(name, n) the next n launches of
- * that kernel are bracketed by a CUDA event pair on their own stream; cvlc_profile_read
- * synchronises the device and returns how many were timed and their summed duration.
- * cvlc_profile_select(NULL, 0) switches it off and frees the events.  Single-threaded use. */
+/* Optional kernel timing: after cvlc_profile_select(name, n) the next n launches of that kernel
+ * ("*" = of every kernel) are bracketed by a CUDA event pair on their own stream;
+ * cvlc_profile_read synchronises the device and returns how many launches of `kernel_name`
+ * (NULL, "" or "*" = all) were timed and their summed duration.  cvlc_profile_select(NULL, 0)
+ * switches it off and frees the events.  Single-threaded use. */
 int cvlc_profile_select(const char* kernel_name, uint32_t max_launches);
 int cvlc_profile_reset(void);
-int cvlc_profile_read(uint32_t* launches, double* total_ms);
+int cvlc_profile_read(const char* kernel_name, uint32_t* launches, double* total_ms);
 
 #ifdef __cplusplus
 }

@@ -139,7 +139,7 @@ def lib() -> C.CDLL:
     L.cvlc_profile_reset.restype = C.c_int
     L.cvlc_profile_reset.argtypes = []
     L.cvlc_profile_read.restype = C.c_int
-    L.cvlc_profile_read.argtypes = [C.POINTER(u32), C.POINTER(f64)]
+    L.cvlc_profile_read.argtypes = [C.c_char_p, C.POINTER(u32), C.POINTER(f64)]
     _lib = L
     return L
 
@@ -328,9 +328,13 @@ def cvlc_profile_reset() -> None:
     _check(lib().cvlc_profile_reset(), "cvlc_profile_reset")
 
 
-def cvlc_profile_read():
+KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan", "k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
+                "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero", "k_decode"]
+
+
+def cvlc_profile_read(kernel_name: str = "*"):
     n, ms = C.c_uint32(), C.c_double()
-    _check(lib().cvlc_profile_read(C.byref(n), C.byref(ms)), "cvlc_profile_read")
+    _check(lib().cvlc_profile_read(kernel_name.encode(), C.byref(n), C.byref(ms)), "cvlc_profile_read")
     return int(n.value), float(ms.value)
 
 

@@ -1,0 +1,125 @@
+"""GPU parity at the full workload sizes, in the batched launch configuration the
+benchmark times: streams bit-exact against the oracle, aggregates within 1e-6 rel /
+1e-7 abs.  The oracle runs in spawned worker processes (one client each)."""
+import numpy as np
+import pytest
+
+import oracle as O
+from paper_2402_03770_b200 import workloads as W
+from gpu_util import assert_aggregate_close, assert_plan_equal, gpu_params, oracle_encode_clients, params_dict
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, keep_on_device=False):
+    w = W.WORKLOADS[workload]
+    dev = torch.device("cuda:0")
+    params, xs = [], []
+    for c in clients:
+        x = W.client_update(w, c, d=d)
+        seed, cid, rnd = W.philox_ids(w, c)
+        params.append(gpu_params(params_dict(x.size, int(np.floor(bpc * x.size)), seed=seed, client_id=cid, round=rnd)))
+        xs.append(torch.from_numpy(x).to(dev))
+    enc = B.BatchEncoder(params, dev, max_candidates=max_candidates)
+    outs = enc.run(xs)
+    assert enc.status() == B.CVLC_OK
+    del xs
+    return enc, outs
+
+
+def check_against_oracle(enc, outs, oracle_results):
+    for i, (client, fields, ost) in enumerate(oracle_results):
+        assert_plan_equal(enc.read_plan(i), fields)
+        got = outs[i].cpu().numpy()
+        assert got.size == ost.size
+        if not (got == ost).all():
+            bad = np.nonzero(got != ost)[0]
+            raise AssertionError(f"client {client}: stream differs at {bad.size} bytes, first at {bad[0]}")
+
+
+def decode_both(outs, oracle_streams, weights, d, torch, B, batches=1):
+    dev = torch.device("cuda:0")
+    n = len(outs)
+    result = torch.full((d,), float("nan"), dtype=torch.float32, device=dev)
+    Wt = float(np.asarray(weights, dtype=np.float64).sum())
+    per = (n + batches - 1) // batches
+    ref = None
+    for b in range(batches):
+        sl = slice(b * per, min(n, (b + 1) * per))
+        agg = B.Aggregator(sl.stop - sl.start, d, dev)
+        agg.set_clients(outs[sl], torch.from_numpy(np.asarray(weights[sl], dtype=np.float32)))
+        agg.run(sl.stop - sl.start, result, weight_total=Wt, accumulate=(b > 0))
+        assert agg.status() == B.CVLC_OK
+        ref = O.decode_aggregate(oracle_streams[sl], np.asarray(weights[sl], dtype=np.float32), d, weight_total=Wt,
+                                 out=ref, accumulate=(b > 0))
+    assert_aggregate_close(result.cpu().numpy(), ref)
+    return ref
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2402_03770_b200 import binding as B
+    assert torch.cuda.is_available()
+    B.lib()
+    B.cvlc_set_device(0)
+    return torch, B
+
+
+def test_small_cnn_all_20_clients(env):
+    torch, B = env
+    w = W.WORKLOADS["small_cnn"]
+    clients = list(range(w.n_clients))
+    ref = oracle_encode_clients("small_cnn", clients, None, 2.0)
+    enc, outs = gpu_batch_encode("small_cnn", clients, None, 2.0, 0, torch, B)
+    check_against_oracle(enc, outs, ref)
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w), w.d, torch, B)
+
+
+@pytest.mark.parametrize("bpc", [0.5, 1.0, 4.0])
+def test_resnet18_budget_sweep_two_clients(env, bpc):
+    torch, B = env
+    w = W.WORKLOADS["resnet18"]
+    clients = [0, 57]
+    ref = oracle_encode_clients("resnet18", clients, None, bpc)
+    enc, outs = gpu_batch_encode("resnet18", clients, None, bpc, 0, torch, B)
+    check_against_oracle(enc, outs, ref)
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w)[clients], w.d, torch, B)
+
+
+def test_resnet18_all_100_clients_as_benchmarked(env):
+    """the benchmark's step: one batched plan + encode of 100 clients at 2 bits per coordinate with the
+    benchmark's reduced candidate workspace, then one decode-aggregate with sample-count weights"""
+    torch, B = env
+    w = W.WORKLOADS["resnet18"]
+    clients = list(range(w.n_clients))
+    ref = oracle_encode_clients("resnet18", clients, None, 2.0)
+    budget = int(2.0 * w.d)
+    max_cand = 3 * (budget // 12000) * ((12000 - 80) // (24 + 1))
+    enc, outs = gpu_batch_encode("resnet18", clients, None, 2.0, max_cand, torch, B)
+    check_against_oracle(enc, outs, ref)
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w), w.d, torch, B)
+
+
+def test_resnet50_ties_and_zero_blocks(env):
+    torch, B = env
+    w = W.WORKLOADS["resnet50"]
+    clients = [0, 1, 2]
+    ref = oracle_encode_clients("resnet50", clients, None, 1.0)
+    enc, outs = gpu_batch_encode("resnet50", clients, None, 1.0, 0, torch, B)
+    check_against_oracle(enc, outs, ref)
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w)[clients], w.d, torch, B)
+
+
+def test_stress_1e8_in_accumulate_batches(env):
+    torch, B = env
+    w = W.WORKLOADS["stress"]
+    clients = [0, 1, 2]
+    ref = oracle_encode_clients("stress", clients, None, 0.25, procs=3)
+    budget = int(0.25 * w.d)
+    max_cand = 3 * (budget // 12000) * ((12000 - 80) // (27 + 1))
+    enc, outs = gpu_batch_encode("stress", clients, None, 0.25, max_cand, torch, B)
+    check_against_oracle(enc, outs, ref)
+    lengths = {y for y in range(33) if enc.read_plan(0).n_y[y]}
+    assert enc.read_plan(0).k < w.d // 100 and len(lengths) >= 2        # mostly 0-bit (sparsified) coordinates
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w)[clients], w.d, torch, B, batches=2)

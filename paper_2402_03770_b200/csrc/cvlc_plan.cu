@@ -157,35 +157,20 @@ __device__ __forceinline__ double energy_E(uint64_t Z, double beta, double D) {
 constexpr int kPlanThreads = 1024;
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
-// F(n) = 1 - gamma of Eq. (5), packets grouped by length, longest first.  One warp:
-// lane l holds candidate length l (count my_n, capacity my_cap, coefficient my_g).
-__device__ __forceinline__ double eval_F_warp(uint32_t my_n, uint32_t my_cap, double my_g, int lane, double beta,
-                                              double D, uint64_t d) {
-  uint64_t W = (uint64_t)my_n * my_cap;  // -> ranks covered down to and including this length
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const uint64_t o = __shfl_down_sync(kFull, W, off);
-    if (lane + off < 32) W += o;
-  }
-  const unsigned act = __ballot_sync(kFull, my_n > 0);
-  double E = 0.0;
-  if (my_n > 0) E = energy_E(W, beta, D);
-  const unsigned higher = (lane == 31) ? 0u : (act & ~((2u << lane) - 1u));
-  const int src = higher ? (__ffs(higher) - 1) : lane;
-  double Eprev = __shfl_sync(kFull, E, src);
-  if (!higher) Eprev = 0.0;
-  const double term = __dmul_rn(my_g, __dsub_rn(E, Eprev));
-  double F = 0.0;
-  unsigned m = act;
-  while (m) {
-    const int l = 31 - __clz(m);
-    m &= ~(1u << l);
-    F = __dadd_rn(F, __shfl_sync(kFull, term, l));
-  }
-  const uint64_t Wtot = __shfl_sync(kFull, W, 0);
-  if (Wtot > d) F = -CUDART_INF;
-  return F;
-}
+// scratch of the length-tuning loop (lives in the dynamic shared memory of the fit points)
+struct PlanSolver {
+  double Ecur[32];                // E(W_l) of the current counts
+  double Fpre[33];                // running sum of F after length l (index 32: nothing yet)
+  double Eab[33];                 // energy of the nearest used length at or above l
+  unsigned long long B[32];       // ranks covered by lengths >= l, the pair under work excluded
+  unsigned long long Wtot;
+  double Ev[1024];                // trial energies   [evaluation * m + slot]
+  double term[1024];              // g_l * (E - E_prev) of every used (evaluation, slot)
+  double Fv[126];                 // trial objective values
+  uint32_t tv[126];               // trial split of every evaluation (0xFFFFFFFF: not needed)
+  int slot_lane[32];              // used lengths <= i, longest first
+  int m;
+};
 
 struct PlanShared {
   double Fv[32];
@@ -368,16 +353,58 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
   const double beta = S.beta, D = S.D;
   const int nY = (int)T.nY;
   const uint32_t my_cap = (lane < nY) ? T.capY[lane] : 0u;
-  const double my_g = (lane < nY) ? T.gY[lane] : 0.0;
+
+  // ---- objective bookkeeping -----------------------------------------------------------
+  // F(n) = 1 - gamma of Eq. (5) is a running sum over the used lengths, longest first:
+  // F += g_l * (E(W_l) - E(W_prev)), W_l = ranks covered down to and including length l.
+  // For the current counts the kernel keeps, per candidate index l: the energy E(W_l)
+  // (Q.Ecur), the running sum after length l (Q.Fpre) and the energy of the nearest used
+  // length at or above l (Q.Eab).  An atomic operation on the lengths i > j leaves everything
+  // above i untouched, so a trial split only needs E for the used lengths at or below i and
+  // continues the running sum from Q.Fpre[i + 1]: the same operations in the same order as a
+  // full evaluation, on a fraction of the lanes.
+  PlanSolver& Q = *reinterpret_cast<PlanSolver*>(ptX);  // the fit points are no longer needed
+
+  auto refresh_state = [&]() {  // all threads; ends with a barrier
+    if (warp == 0) {
+      const uint32_t my_n = (lane < nY) ? S.n[lane] : 0u;
+      uint64_t W = (uint64_t)my_n * my_cap;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint64_t o = __shfl_down_sync(kFull, W, off);
+        if (lane + off < 32) W += o;
+      }
+      Q.Ecur[lane] = (my_n > 0) ? energy_E(W, beta, D) : 0.0;
+      if (lane == 0) Q.Wtot = W;
+      __syncwarp();
+      if (lane == 0) {
+        double F = 0.0, Eprev = 0.0;
+        Q.Fpre[32] = 0.0;
+        Q.Eab[32] = 0.0;
+        for (int l = 31; l >= 0; --l) {
+          if (l < nY && S.n[l] > 0) {
+            const double Ec = Q.Ecur[l];
+            F = __dadd_rn(F, __dmul_rn(T.gY[l], __dsub_rn(Ec, Eprev)));
+            Eprev = Ec;
+          }
+          Q.Fpre[l] = F;
+          Q.Eab[l] = Eprev;
+        }
+      }
+    }
+    __syncthreads();
+  };
 
   if (T.fixed_y != 0) {
     if (tid == 0) S.n[0] = T.R;
     __syncthreads();
+    refresh_state();
   } else {
     // ---- equal packets: best admissible single-length plan, ties to the longer code ----
-    if (warp < nY) {
-      const double F = eval_F_warp(lane == warp ? T.R : 0u, my_cap, my_g, lane, beta, D, T.d);
-      if (lane == 0) S.Fv[warp] = F;
+    if (tid < nY) {
+      const uint64_t W = (uint64_t)T.R * T.capY[tid];
+      // one term: F = 0 + g * (E - 0)
+      S.Fv[tid] = (W > T.d) ? -CUDART_INF : __dmul_rn(T.gY[tid], energy_E(W, beta, D));
     }
     __syncthreads();
     if (tid == 0) {
@@ -394,12 +421,15 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
       S.n[best < 0 ? 0 : best] = T.R;  // the host has checked that a plan is admissible
     }
     __syncthreads();
+    refresh_state();
 
     // ---- atomic operations (Section IV-C) on pairs of lengths until nothing moves ----
-    // An atomic operation bisects the split of X = n_a + n_c packets between the lengths
-    // a > c for the first t with F(t+1) <= F(t).  Four bisection levels are evaluated at
-    // once: warps 2q, 2q+1 evaluate F(mid+1), F(mid) of node q+1 of the decision tree,
-    // warp 30 evaluates the current split; then every thread walks the tree.
+    // An atomic operation bisects the split of X = n_i + n_j packets between the lengths
+    // i > j for the first t with F(t+1) <= F(t).  Several bisection levels are evaluated at once:
+    // evaluation e = 2q, 2q+1 is F(mid+1), F(mid) of node q+1 of the decision tree (heap order:
+    // child 2h after "F(mid+1) <= F(mid)", child 2h+1 after "F(mid+1) > F(mid)"); one thread per
+    // (evaluation, used length <= i) computes an energy and its term, one thread per evaluation
+    // adds the terms in order, then every thread walks the tree.
     for (int round = 0; round < 64; ++round) {
       int movedB = 0;
       for (int phase = 0; phase < 2; ++phase) {  // 0: neighbouring lengths until quiet; 1: every pair once
@@ -412,17 +442,40 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
               const uint32_t na0 = S.n[i], nc0 = S.n[j];
               const uint32_t X = na0 + nc0;
               if (X == 0) continue;
+              // setup: ranks covered by the other lengths, and the list of lengths a trial must evaluate
+              if (warp == 0) {
+                const uint32_t my_n = (lane < nY && lane != i && lane != j) ? S.n[lane] : 0u;
+                uint64_t Bs = (uint64_t)my_n * my_cap;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                  const uint64_t o = __shfl_down_sync(kFull, Bs, off);
+                  if (lane + off < 32) Bs += o;
+                }
+                Q.B[lane] = Bs;
+                const unsigned need = __ballot_sync(kFull, lane <= i && (my_n > 0 || lane == i || lane == j));
+                if (need & (1u << lane)) Q.slot_lane[lane == 31 ? 0 : __popc(need >> (lane + 1))] = lane;  // longest first
+                if (lane == 0) Q.m = __popc(need);
+              }
+              __syncthreads();
+              const int m = Q.m;
+              // the kernel is bound by the latency of one energy evaluation, so as many bisection levels
+              // as fit in one pass of the block are evaluated per round
+              const int levels = (126 * m <= kPlanThreads) ? 6 : (62 * m <= kPlanThreads) ? 5 : 4;
+              const int n_evals = 2 * ((1 << levels) - 1);
+              const uint64_t cap_i = T.capY[i], cap_j = T.capY[j];
+              const double F_cur = Q.Fpre[0];
               uint32_t lo = 0, hi = X;
-              double F_final = 0.0, F_cur = 0.0;
-              bool first = true;
+              double F_final = 0.0;
               while (lo < hi) {
-                // which evaluation does this warp own?
-                bool valid = false;
-                uint32_t t = 0;
-                if (warp < 30) {
-                  // node (warp/2 + 1) of the decision tree in heap order: child 2h after
-                  // "F(mid+1) <= F(mid)", child 2h+1 after "F(mid+1) > F(mid)"
-                  const int hnode = (warp >> 1) + 1;
+                // phase 1: energies, one thread per (evaluation, slot)
+                const int item = tid;
+                const bool has_item = item < n_evals * m;
+                int e = 0, sl = 0;
+                uint32_t t = 0xFFFFFFFFu;
+                if (has_item) {
+                  e = item / m;
+                  sl = item - e * m;
+                  const int hnode = (e >> 1) + 1;
                   const int depth = 31 - __clz(hnode);
                   uint32_t l3 = lo, h3 = hi;
                   bool open = true;
@@ -432,28 +485,49 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                     if ((hnode >> b) & 1) l3 = mid + 1; else h3 = mid;
                   }
                   if (open && l3 < h3) {
-                    const uint32_t mid = l3 + (h3 - l3) / 2;
-                    t = mid + ((warp & 1) ? 0u : 1u);
-                    valid = true;
+                    t = l3 + (h3 - l3) / 2 + ((e & 1) ? 0u : 1u);
+                    const int l = Q.slot_lane[sl];
+                    const uint64_t W = Q.B[l] + (uint64_t)t * cap_i + ((l <= j) ? (uint64_t)(X - t) * cap_j : 0ull);
+                    Q.Ev[item] = energy_E(W, beta, D);
                   }
-                } else if (warp == 30 && first) {
-                  t = na0;
-                  valid = true;
-                }
-                if (valid) {
-                  uint32_t my_n = (lane < nY) ? S.n[lane] : 0u;
-                  if (lane == i) my_n = t;
-                  if (lane == j) my_n = X - t;
-                  const double F = eval_F_warp(my_n, my_cap, my_g, lane, beta, D, T.d);
-                  if (lane == 0) S.Fv[warp] = F;
+                  if (sl == 0) Q.tv[e] = t;
                 }
                 __syncthreads();
-                if (first) F_cur = S.Fv[30];
-                first = false;
+                // phase 2: the terms g_l * (E_l - E_prev); only the lengths i and j can be unused in a trial
+                if (has_item && t != 0xFFFFFFFFu) {
+                  const int l = Q.slot_lane[sl];
+                  const uint32_t nn = (l == i) ? t : (l == j) ? (X - t) : 1u;
+                  if (nn > 0) {
+                    int p = sl - 1;
+                    while (p >= 0) {
+                      const int lp = Q.slot_lane[p];
+                      const uint32_t np = (lp == i) ? t : (lp == j) ? (X - t) : 1u;
+                      if (np > 0) break;
+                      --p;
+                    }
+                    const double Eprev = (p >= 0) ? Q.Ev[e * m + p] : Q.Eab[i + 1];
+                    Q.term[item] = __dmul_rn(T.gY[l], __dsub_rn(Q.Ev[item], Eprev));
+                  }
+                }
+                __syncthreads();
+                // phase 3: one thread per evaluation continues the running sum below length i
+                if (tid < n_evals && Q.tv[tid] != 0xFFFFFFFFu) {
+                  const uint32_t tt = Q.tv[tid];
+                  double F = Q.Fpre[i + 1];
+                  for (int q = 0; q < m; ++q) {
+                    const int l = Q.slot_lane[q];
+                    const uint32_t nn = (l == i) ? tt : (l == j) ? (X - tt) : 1u;
+                    if (nn > 0) F = __dadd_rn(F, Q.term[tid * m + q]);
+                  }
+                  const uint64_t Wtot = Q.B[0] + (uint64_t)tt * cap_i + (uint64_t)(X - tt) * cap_j;
+                  Q.Fv[tid] = (Wtot > T.d) ? -CUDART_INF : F;
+                }
+                __syncthreads();
+                // phase 4: every thread walks the decision tree
                 int hnode = 1;
-                for (int level = 0; level < 4 && lo < hi; ++level) {
+                for (int level = 0; level < levels && lo < hi; ++level) {
                   const uint32_t mid = lo + (hi - lo) / 2;
-                  const double F1 = S.Fv[2 * (hnode - 1)], F0 = S.Fv[2 * (hnode - 1) + 1];
+                  const double F1 = Q.Fv[2 * (hnode - 1)], F0 = Q.Fv[2 * (hnode - 1) + 1];
                   if (F1 > F0) {
                     lo = mid + 1;
                     F_final = F1;
@@ -472,8 +546,9 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   S.n[j] = X - lo;
                 }
                 moved = 1;
+                __syncthreads();
+                refresh_state();
               }
-              __syncthreads();
             }
           }
           if (phase == 1) movedB = moved;
@@ -485,12 +560,6 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
   }
 
   // ---- outputs ---------------------------------------------------------------------
-  if (warp == 0) {
-    const uint32_t my_n = (lane < nY) ? S.n[lane] : 0u;
-    const double F = eval_F_warp(my_n, my_cap, my_g, lane, beta, D, T.d);
-    if (lane == 0) S.Fv[0] = F;
-  }
-  __syncthreads();
   unsigned long long k = 0;
   for (int i = 0; i < nY; ++i) k += (unsigned long long)S.n[i] * T.capY[i];
   if (tid == 0) {
@@ -507,7 +576,7 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     plan->alpha = S.alpha;
     plan->alpha_q = S.alpha_q;
     plan->beta = beta;
-    plan->gamma = __dsub_rn(1.0, S.Fv[0]);
+    plan->gamma = __dsub_rn(1.0, Q.Fpre[0]);
     plan->B_next = __dadd_rn(1.0, Qmax);
     for (int y = 0; y <= CVLC_MAX_CODE_BITS; ++y) {
       plan->n_y[y] = 0;

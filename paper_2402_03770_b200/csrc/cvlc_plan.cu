@@ -158,18 +158,32 @@ constexpr int kPlanThreads = 1024;
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
 // scratch of the length-tuning loop (lives in the dynamic shared memory of the fit points)
+constexpr int kMaxBatchOps = 32;  // atomic operations evaluated together
+struct PlanOp {                   // one atomic operation of a batch
+  int i, j;                       // candidate indices, i > j
+  uint32_t X, na0;                // packets shared by the pair; current count of length i
+  uint32_t lo, hi;                // bisection interval
+  int m;                          // lengths a trial must evaluate (used lengths <= i, plus i and j)
+  int levels;                     // bisection levels evaluated in this round (0: waits)
+  int item_base, eval_base;       // first (evaluation, slot) item / first evaluation of this operation
+  double F_final;                 // F at the end of the bisection
+  unsigned char slot_lane[32];    // those lengths, longest first
+};
 struct PlanSolver {
   double Ecur[32];                // E(W_l) of the current counts
   double Fpre[33];                // running sum of F after length l (index 32: nothing yet)
   double Eab[33];                 // energy of the nearest used length at or above l
-  unsigned long long B[32];       // ranks covered by lengths >= l, the pair under work excluded
-  unsigned long long Wtot;
-  double Ev[1024];                // trial energies   [evaluation * m + slot]
-  double term[1024];              // g_l * (E - E_prev) of every used (evaluation, slot)
-  double Fv[126];                 // trial objective values
-  uint32_t tv[126];               // trial split of every evaluation (0xFFFFFFFF: not needed)
-  int slot_lane[32];              // used lengths <= i, longest first
-  int m;
+  unsigned long long Wc[32];      // ranks covered by lengths >= l, current counts
+  unsigned used;                  // lengths with a positive count
+  double Ev[1024];                // trial energies, one per item
+  double term[1024];              // g_l * (E - E_prev) of every used item
+  double Fv[1024];                // trial objective values, one per evaluation
+  uint32_t tv[1024];              // trial split of every evaluation (0xFFFFFFFF: not needed)
+  PlanOp op[kMaxBatchOps];
+  int item_end[kMaxBatchOps];     // exclusive end of every operation's items / evaluations in this round
+  int eval_end[kMaxBatchOps];
+  int n_ops, n_items, n_evals, unfinished;
+  int next_i, next_j, moved;      // where the sweep resumes after the batch
 };
 
 struct PlanShared {
@@ -375,7 +389,9 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
         if (lane + off < 32) W += o;
       }
       Q.Ecur[lane] = (my_n > 0) ? energy_E(W, beta, D) : 0.0;
-      if (lane == 0) Q.Wtot = W;
+      Q.Wc[lane] = W;
+      const unsigned used = __ballot_sync(kFull, my_n > 0);
+      if (lane == 0) Q.used = used;
       __syncwarp();
       if (lane == 0) {
         double F = 0.0, Eprev = 0.0;
@@ -424,131 +440,243 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     refresh_state();
 
     // ---- atomic operations (Section IV-C) on pairs of lengths until nothing moves ----
-    // An atomic operation bisects the split of X = n_i + n_j packets between the lengths
-    // i > j for the first t with F(t+1) <= F(t).  Several bisection levels are evaluated at once:
-    // evaluation e = 2q, 2q+1 is F(mid+1), F(mid) of node q+1 of the decision tree (heap order:
-    // child 2h after "F(mid+1) <= F(mid)", child 2h+1 after "F(mid+1) > F(mid)"); one thread per
-    // (evaluation, used length <= i) computes an energy and its term, one thread per evaluation
-    // adds the terms in order, then every thread walks the tree.
+    // An atomic operation bisects the split of X = n_i + n_j packets between the lengths i > j
+    // for the first t with F(t+1) <= F(t) and moves there if that is strictly better.  Most
+    // operations of a sweep change nothing, so consecutive operations are evaluated together as
+    // if none of them moved; the first one (in sweep order) that does move is applied, the later
+    // ones of the batch are dropped and the sweep resumes right after it: exactly the sequential
+    // result.  Per round every unfinished operation gets as many bisection levels as the block's
+    // 1024 (evaluation, length) items allow: evaluation e = 2q, 2q+1 of an operation is
+    // F(mid+1), F(mid) of node q+1 of its decision tree (heap order: child 2h after
+    // "F(mid+1) <= F(mid)", child 2h+1 after "F(mid+1) > F(mid)").
+    auto next_pair = [&](int phase, int& i, int& j) {  // sweep order; i = 0 marks the end
+      if (phase == 0) {
+        --i;
+        j = i - 1;
+      } else if (j > 0) {
+        --j;
+      } else {
+        --i;
+        j = i - 1;
+      }
+    };
     for (int round = 0; round < 64; ++round) {
       int movedB = 0;
       for (int phase = 0; phase < 2; ++phase) {  // 0: neighbouring lengths until quiet; 1: every pair once
         const int max_sweeps = (phase == 0) ? 256 : 1;
         for (int sweep = 0; sweep < max_sweeps; ++sweep) {
           int moved = 0;
-          for (int i = nY - 1; i >= 1; --i) {
-            const int j_hi = i - 1, j_lo = (phase == 0) ? i - 1 : 0;
-            for (int j = j_hi; j >= j_lo; --j) {
-              const uint32_t na0 = S.n[i], nc0 = S.n[j];
-              const uint32_t X = na0 + nc0;
-              if (X == 0) continue;
-              // setup: ranks covered by the other lengths, and the list of lengths a trial must evaluate
+          int ci = nY - 1, cj = nY - 2;  // cursor of the sweep
+          while (ci >= 1) {
+            // ---- collect a batch (every thread computes the same list; thread 0 records it)
+            {
+              int bi = ci, bj = cj, n_ops = 0, reserved = 0;
+              const unsigned used = Q.used;
+              while (bi >= 1 && n_ops < kMaxBatchOps) {
+                const uint32_t X = S.n[bi] + S.n[bj];
+                if (X > 0) {
+                  const unsigned need = (used | (1u << bi) | (1u << bj)) & (0xFFFFFFFFu >> (31 - bi));
+                  const int m = __popc(need);
+                  if (reserved + 2 * m > kPlanThreads) break;  // one level at least for every operation
+                  reserved += 2 * m;
+                  if (tid == 0) {
+                    PlanOp& o = Q.op[n_ops];
+                    o.i = bi; o.j = bj; o.X = X; o.na0 = S.n[bi]; o.lo = 0; o.hi = X; o.m = m; o.F_final = 0.0;
+                  }
+                  if (warp == n_ops && (need & (1u << lane)))
+                    Q.op[n_ops].slot_lane[lane == 31 ? 0 : __popc(need >> (lane + 1))] = (unsigned char)lane;
+                  ++n_ops;
+                }
+                next_pair(phase, bi, bj);
+              }
+              if (tid == 0) {
+                Q.n_ops = n_ops;
+                Q.next_i = bi;
+                Q.next_j = bj;
+                Q.moved = 0;
+                Q.unfinished = n_ops;
+              }
+              ci = bi;
+              cj = bj;
+              if (n_ops == 0) continue;  // the rest of the sweep had nothing to split
+            }
+            __syncthreads();
+            const int n_ops = Q.n_ops;
+            const double F_cur = Q.Fpre[0];
+            // ---- rounds until every operation of the batch has finished its bisection
+            while (true) {
+              // level assignment (warp 0, lane = operation): the planner is bound by the FP64 throughput
+              // of its SM, and every extra level evaluated ahead doubles the work, so all operations get
+              // the same small depth: the largest one whose items fit the block
               if (warp == 0) {
-                const uint32_t my_n = (lane < nY && lane != i && lane != j) ? S.n[lane] : 0u;
-                uint64_t Bs = (uint64_t)my_n * my_cap;
+                const bool mine = lane < n_ops;
+                const uint32_t span = (mine && Q.op[lane].lo < Q.op[lane].hi) ? Q.op[lane].hi - Q.op[lane].lo : 0u;
+                const int need_levels = span ? 32 - __clz(span) : 0;  // a bisection of s points takes at most floor(log2 s) + 1 steps
+                const int m_op = mine ? Q.op[lane].m : 0;
+                int depth = 0;
+                for (int cand = 1; cand <= 9; ++cand) {
+                  const int lv = need_levels < cand ? need_levels : cand;
+                  int items = lv ? 2 * ((1 << lv) - 1) * m_op : 0;
+#pragma unroll
+                  for (int off = 16; off > 0; off >>= 1) items += __shfl_xor_sync(kFull, items, off);
+                  if (items <= kPlanThreads) depth = cand; else break;
+                }
+                const int lv = need_levels < depth ? need_levels : depth;
+                const int ne = lv ? 2 * ((1 << lv) - 1) : 0;
+                int items_incl = ne * m_op, evals_incl = ne;
 #pragma unroll
                 for (int off = 1; off < 32; off <<= 1) {
-                  const uint64_t o = __shfl_down_sync(kFull, Bs, off);
-                  if (lane + off < 32) Bs += o;
+                  const int a1 = __shfl_up_sync(kFull, items_incl, off), a2 = __shfl_up_sync(kFull, evals_incl, off);
+                  if (lane >= off) {
+                    items_incl += a1;
+                    evals_incl += a2;
+                  }
                 }
-                Q.B[lane] = Bs;
-                const unsigned need = __ballot_sync(kFull, lane <= i && (my_n > 0 || lane == i || lane == j));
-                if (need & (1u << lane)) Q.slot_lane[lane == 31 ? 0 : __popc(need >> (lane + 1))] = lane;  // longest first
-                if (lane == 0) Q.m = __popc(need);
+                if (mine) {
+                  Q.op[lane].levels = lv;
+                  Q.op[lane].item_base = items_incl - ne * m_op;
+                  Q.op[lane].eval_base = evals_incl - ne;
+                }
+                Q.item_end[lane] = items_incl;
+                Q.eval_end[lane] = evals_incl;
+                const unsigned unfinished = __ballot_sync(kFull, need_levels > 0);
+                if (lane == 31) {
+                  Q.n_items = items_incl;
+                  Q.n_evals = evals_incl;
+                  Q.unfinished = __popc(unfinished);
+                }
               }
               __syncthreads();
-              const int m = Q.m;
-              // the kernel is bound by the latency of one energy evaluation, so as many bisection levels
-              // as fit in one pass of the block are evaluated per round
-              const int levels = (126 * m <= kPlanThreads) ? 6 : (62 * m <= kPlanThreads) ? 5 : 4;
-              const int n_evals = 2 * ((1 << levels) - 1);
-              const uint64_t cap_i = T.capY[i], cap_j = T.capY[j];
-              const double F_cur = Q.Fpre[0];
-              uint32_t lo = 0, hi = X;
-              double F_final = 0.0;
-              while (lo < hi) {
-                // phase 1: energies, one thread per (evaluation, slot)
-                const int item = tid;
-                const bool has_item = item < n_evals * m;
-                int e = 0, sl = 0;
-                uint32_t t = 0xFFFFFFFFu;
-                if (has_item) {
-                  e = item / m;
-                  sl = item - e * m;
-                  const int hnode = (e >> 1) + 1;
-                  const int depth = 31 - __clz(hnode);
-                  uint32_t l3 = lo, h3 = hi;
-                  bool open = true;
-                  for (int b = depth - 1; b >= 0; --b) {
-                    if (!(l3 < h3)) { open = false; break; }
-                    const uint32_t mid = l3 + (h3 - l3) / 2;
-                    if ((hnode >> b) & 1) l3 = mid + 1; else h3 = mid;
-                  }
-                  if (open && l3 < h3) {
-                    t = l3 + (h3 - l3) / 2 + ((e & 1) ? 0u : 1u);
-                    const int l = Q.slot_lane[sl];
-                    const uint64_t W = Q.B[l] + (uint64_t)t * cap_i + ((l <= j) ? (uint64_t)(X - t) * cap_j : 0ull);
-                    Q.Ev[item] = energy_E(W, beta, D);
-                  }
-                  if (sl == 0) Q.tv[e] = t;
+              if (Q.unfinished == 0) break;
+              // phase 1: energies, one thread per (operation, evaluation, slot)
+              int a = -1, e = 0, sl = 0;
+              uint32_t t = 0xFFFFFFFFu;
+              if (tid < Q.n_items) {
+                // the operation whose item range holds this thread: first a with tid < item_end[a]
+                int lo_a = 0, hi_a = 31;
+                while (lo_a < hi_a) {
+                  const int mid = (lo_a + hi_a) >> 1;
+                  if (tid < Q.item_end[mid]) hi_a = mid; else lo_a = mid + 1;
                 }
-                __syncthreads();
-                // phase 2: the terms g_l * (E_l - E_prev); only the lengths i and j can be unused in a trial
-                if (has_item && t != 0xFFFFFFFFu) {
-                  const int l = Q.slot_lane[sl];
-                  const uint32_t nn = (l == i) ? t : (l == j) ? (X - t) : 1u;
-                  if (nn > 0) {
-                    int p = sl - 1;
-                    while (p >= 0) {
-                      const int lp = Q.slot_lane[p];
-                      const uint32_t np = (lp == i) ? t : (lp == j) ? (X - t) : 1u;
-                      if (np > 0) break;
-                      --p;
-                    }
-                    const double Eprev = (p >= 0) ? Q.Ev[e * m + p] : Q.Eab[i + 1];
-                    Q.term[item] = __dmul_rn(T.gY[l], __dsub_rn(Q.Ev[item], Eprev));
-                  }
+                a = lo_a;
+                const PlanOp& o = Q.op[a];
+                const int rel = tid - o.item_base;
+                e = rel / o.m;
+                sl = rel - e * o.m;
+                const int hnode = (e >> 1) + 1;
+                const int depth = 31 - __clz(hnode);
+                uint32_t l3 = o.lo, h3 = o.hi;
+                bool open = true;
+                for (int b = depth - 1; b >= 0; --b) {
+                  if (!(l3 < h3)) { open = false; break; }
+                  const uint32_t mid = l3 + (h3 - l3) / 2;
+                  if ((hnode >> b) & 1) l3 = mid + 1; else h3 = mid;
                 }
-                __syncthreads();
-                // phase 3: one thread per evaluation continues the running sum below length i
-                if (tid < n_evals && Q.tv[tid] != 0xFFFFFFFFu) {
-                  const uint32_t tt = Q.tv[tid];
-                  double F = Q.Fpre[i + 1];
-                  for (int q = 0; q < m; ++q) {
-                    const int l = Q.slot_lane[q];
-                    const uint32_t nn = (l == i) ? tt : (l == j) ? (X - tt) : 1u;
-                    if (nn > 0) F = __dadd_rn(F, Q.term[tid * m + q]);
+                if (open && l3 < h3) {
+                  t = l3 + (h3 - l3) / 2 + ((e & 1) ? 0u : 1u);
+                  const int l = o.slot_lane[sl];
+                  // ranks down to length l with the pair's packets re-split: the current cover, minus the
+                  // pair's current share, plus the trial's
+                  uint64_t W = Q.Wc[l] - (uint64_t)S.n[o.i] * T.capY[o.i] + (uint64_t)t * T.capY[o.i];
+                  if (l <= o.j) W = W - (uint64_t)S.n[o.j] * T.capY[o.j] + (uint64_t)(o.X - t) * T.capY[o.j];
+                  Q.Ev[tid] = energy_E(W, beta, D);
+                }
+                if (sl == 0) Q.tv[o.eval_base + e] = t;
+              }
+              __syncthreads();
+              // phase 2: the terms g_l * (E_l - E_prev); only the lengths i and j can be unused in a trial
+              if (a >= 0 && t != 0xFFFFFFFFu) {
+                const PlanOp& o = Q.op[a];
+                const int l = o.slot_lane[sl];
+                const uint32_t nn = (l == o.i) ? t : (l == o.j) ? (o.X - t) : 1u;
+                if (nn > 0) {
+                  int p = sl - 1;
+                  while (p >= 0) {
+                    const int lp = o.slot_lane[p];
+                    const uint32_t np = (lp == o.i) ? t : (lp == o.j) ? (o.X - t) : 1u;
+                    if (np > 0) break;
+                    --p;
                   }
-                  const uint64_t Wtot = Q.B[0] + (uint64_t)tt * cap_i + (uint64_t)(X - tt) * cap_j;
+                  const double Eprev = (p >= 0) ? Q.Ev[tid - sl + p] : Q.Eab[o.i + 1];
+                  Q.term[tid] = __dmul_rn(T.gY[l], __dsub_rn(Q.Ev[tid], Eprev));
+                }
+              }
+              __syncthreads();
+              // phase 3: one thread per evaluation continues the running sum below length i
+              if (tid < Q.n_evals) {
+                int lo_a = 0, hi_a = 31;
+                while (lo_a < hi_a) {
+                  const int mid = (lo_a + hi_a) >> 1;
+                  if (tid < Q.eval_end[mid]) hi_a = mid; else lo_a = mid + 1;
+                }
+                const PlanOp& o = Q.op[lo_a];
+                const uint32_t tt = Q.tv[tid];
+                if (tt != 0xFFFFFFFFu) {
+                  const int ee = tid - o.eval_base;
+                  const double* tm = Q.term + o.item_base + ee * o.m;
+                  double F = Q.Fpre[o.i + 1];
+                  for (int z = 0; z < o.m; ++z) {
+                    const int l = o.slot_lane[z];
+                    const uint32_t nn = (l == o.i) ? tt : (l == o.j) ? (o.X - tt) : 1u;
+                    if (nn > 0) F = __dadd_rn(F, tm[z]);
+                  }
+                  const uint64_t Wtot = Q.Wc[0] - (uint64_t)S.n[o.i] * T.capY[o.i] - (uint64_t)S.n[o.j] * T.capY[o.j] +
+                                        (uint64_t)tt * T.capY[o.i] + (uint64_t)(o.X - tt) * T.capY[o.j];
                   Q.Fv[tid] = (Wtot > T.d) ? -CUDART_INF : F;
                 }
-                __syncthreads();
-                // phase 4: every thread walks the decision tree
-                int hnode = 1;
-                for (int level = 0; level < levels && lo < hi; ++level) {
-                  const uint32_t mid = lo + (hi - lo) / 2;
-                  const double F1 = Q.Fv[2 * (hnode - 1)], F0 = Q.Fv[2 * (hnode - 1) + 1];
-                  if (F1 > F0) {
-                    lo = mid + 1;
-                    F_final = F1;
-                    hnode = 2 * hnode + 1;
-                  } else {
-                    hi = mid;
-                    F_final = F0;
-                    hnode = 2 * hnode;
+              }
+              __syncthreads();
+              // phase 4: one thread per operation walks its decision tree
+              if (tid < n_ops) {
+                PlanOp& o = Q.op[tid];
+                if (o.levels > 0) {
+                  uint32_t lo = o.lo, hi = o.hi;
+                  double Ff = o.F_final;
+                  int hnode = 1;
+                  for (int level = 0; level < o.levels && lo < hi; ++level) {
+                    const uint32_t mid = lo + (hi - lo) / 2;
+                    const double F1 = Q.Fv[o.eval_base + 2 * (hnode - 1)], F0 = Q.Fv[o.eval_base + 2 * (hnode - 1) + 1];
+                    if (F1 > F0) {
+                      lo = mid + 1;
+                      Ff = F1;
+                      hnode = 2 * hnode + 1;
+                    } else {
+                      hi = mid;
+                      Ff = F0;
+                      hnode = 2 * hnode;
+                    }
                   }
+                  o.lo = lo;
+                  o.hi = hi;
+                  o.F_final = Ff;
                 }
-                __syncthreads();
               }
-              if (lo != na0 && F_final > F_cur) {
-                if (tid == 0) {
-                  S.n[i] = lo;
-                  S.n[j] = X - lo;
+              __syncthreads();
+            }
+            // ---- the first operation of the batch that improves F is applied; the sweep resumes after it
+            if (tid == 0) {
+              for (int a = 0; a < n_ops; ++a) {
+                const PlanOp& o = Q.op[a];
+                if (o.lo != o.na0 && o.F_final > F_cur) {
+                  S.n[o.i] = o.lo;
+                  S.n[o.j] = o.X - o.lo;
+                  int ri = o.i, rj = o.j;
+                  next_pair(phase, ri, rj);
+                  Q.next_i = ri;
+                  Q.next_j = rj;
+                  Q.moved = 1;
+                  break;
                 }
-                moved = 1;
-                __syncthreads();
-                refresh_state();
               }
+            }
+            __syncthreads();
+            ci = Q.next_i;
+            cj = Q.next_j;
+            if (Q.moved) {
+              moved = 1;
+              refresh_state();
+            } else {
+              __syncthreads();
             }
           }
           if (phase == 1) movedB = moved;

@@ -556,6 +556,9 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
   __shared__ uint32_t s_tile;
   __shared__ uint32_t s_wc[kSortThreads / 32][kDigits];  // per-warp digit counters -> per-warp offsets
   __shared__ unsigned long long s_base[kDigits];         // position of this tile's first item per digit
+  __shared__ uint32_t s_dstart[kDigits];                 // first slot of every digit value inside the tile
+  __shared__ uint32_t s_scan_w[kSortThreads / 32];
+  __shared__ unsigned long long s_items[kSortTile];      // the tile's items in digit order
   extern __shared__ uint32_t s_prefix[];                 // [n + 1] first sort tile of every client
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
@@ -646,6 +649,32 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
         open[q] = tile > 0;
         st_relaxed(state + (size_t)tile * kDigits + dg, (tile == 0 ? kFlagPrefix : kFlagAgg) | t);
       }
+      // first slot of every digit value inside the tile: exclusive scan of the tile's digit counts in digit
+      // order (thread t owns digits t and t + 256), done while the look-back loads are in flight
+      {
+        uint32_t carry = 0;
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+          uint32_t incl = tot[q];
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t o = __shfl_up_sync(kFull, incl, off);
+            if (lane >= off) incl += o;
+          }
+          if (lane == 31) s_scan_w[warp] = incl;
+          __syncthreads();
+          uint32_t below = 0, all = 0;
+#pragma unroll
+          for (int w = 0; w < kSortThreads / 32; ++w) {
+            const uint32_t v = s_scan_w[w];
+            if (w < warp) below += v;
+            all += v;
+          }
+          s_dstart[tid + q * kSortThreads] = carry + below + incl - tot[q];
+          carry += all;
+          __syncthreads();
+        }
+      }
       for (long long t = (long long)tile - 1; t >= 0; --t) {
         bool any_open = false;
 #pragma unroll
@@ -666,13 +695,23 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
         s_base[dg] = gbase[dg] + run[q];
       }
     }
-    __syncthreads();
+    // the items go to shared memory in digit order, then out in runs of consecutive addresses
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       if ((first + i * 32 + lane) < n) {
         const uint32_t dig = sort_digit(item[i], pass, keytop);
-        const unsigned long long o = s_base[dig] + s_wc[warp][dig] + rank[i];
-        if (o < n && o < L.capacity) dst[o] = item[i];
+        s_items[s_dstart[dig] + s_wc[warp][dig] + rank[i]] = item[i];
+      }
+    }
+    __syncthreads();
+    {
+      const unsigned long long tile_first = (unsigned long long)tile * kSortTile;
+      const uint32_t count = (n - tile_first < (unsigned long long)kSortTile) ? (uint32_t)(n - tile_first) : (uint32_t)kSortTile;
+      for (uint32_t k = tid; k < count; k += kSortThreads) {
+        const unsigned long long it = s_items[k];
+        const uint32_t dig = sort_digit(it, pass, keytop);
+        const unsigned long long o = s_base[dig] + (k - s_dstart[dig]);
+        if (o < n && o < L.capacity) dst[o] = it;
       }
     }
     __syncthreads();

@@ -558,8 +558,9 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
   __shared__ unsigned long long s_base[kDigits];         // position of this tile's first item per digit
   __shared__ uint32_t s_dstart[kDigits];                 // first slot of every digit value inside the tile
   __shared__ uint32_t s_scan_w[kSortThreads / 32];
-  __shared__ unsigned long long s_items[kSortTile];      // the tile's items in digit order
-  extern __shared__ uint32_t s_prefix[];                 // [n + 1] first sort tile of every client
+  extern __shared__ unsigned long long s_dyn[];
+  unsigned long long* s_items = s_dyn;                                         // [kSortTile] the tile's items in digit order
+  uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_dyn + kSortTile);         // [n + 1] first sort tile of every client
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -906,6 +907,8 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_select<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSelStages * kSelStageBytes));
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_sort_pass<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSortTile * 8 + (CVLC_MAX_BATCH + 1) * 4));
+    if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
   BatchDesc<CAP> batch;
@@ -944,7 +947,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     }
     for (int pass = 0; pass < kSortPasses; ++pass) {
       LaunchScope ls(kKSortPass, st);
-      k_sort_pass<CAP><<<grid, kSortThreads, ((size_t)n + 1) * 4, st>>>(pass, batch, w, L);
+      k_sort_pass<CAP><<<grid, kSortThreads, (size_t)kSortTile * 8 + ((size_t)n + 1) * 4, st>>>(pass, batch, w, L);
     }
   }
   {

@@ -297,17 +297,33 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// sort key digits (see the ranking kernels below); the selection kernel already counts them
+__device__ __forceinline__ uint32_t sort_keytop(const cvlc_plan_t* plan) { return ((plan->top_bin + 1u) << 19) - 1u; }
+
+__device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass, uint32_t keytop) {
+  const uint32_t key = (uint32_t)(pair >> 32);
+  const uint32_t inv = key > keytop ? 0u : keytop - key;  // key > keytop only if the plan is not of this update
+  return (inv >> (kDigitBits * pass)) & (kDigits - 1);
+}
+
 // Staging layout: float4 unit g of a tile (g = 0 .. 2047, in memory order) sits in slot
 // g ^ ((g >> 3) & 3).  The copies of a warp (consecutive g) and the reads of a warp (thread t
 // reads its own four consecutive units 4t .. 4t+3) are then both free of bank conflicts.
-__device__ __forceinline__ uint32_t sel_slot(uint32_t g) { return g ^ ((g >> 3) & 3u); }
+constexpr int kSelThreads = 512;                      // threads of the selection kernel
+constexpr int kSelVec = 4;                            // float4 units (16 coordinates) per thread and tile
+constexpr uint32_t kSelTileVec = kSelThreads * kSelVec;  // 2048 float4 = 8192 coordinates = 32 KB
+static_assert(kSelTileVec * 16 == kSelStageBytes, "stage size");
+__device__ __forceinline__ uint32_t sel_slot(uint32_t g) { return g ^ ((g >> 3) & (uint32_t)(kSelVec - 1)); }
 
 template <int CAP>
-__global__ void __launch_bounds__(kSelectThreads, 2)
+__global__ void __launch_bounds__(kSelThreads, 2)
 k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_constant__ Partition part,
          const unsigned char* __restrict__ plan_ws, unsigned char* ws, const __grid_constant__ EncLayout L) {
   extern __shared__ float4 s_stage[];  // [kSelStages][2048 float4]
-  __shared__ uint32_t s_warp_incl[2][kSelectThreads / 32];
+  __shared__ uint32_t s_warp_incl[2][kSelThreads / 32];
+  __shared__ uint32_t s_dhist[kSortPasses * kDigits];  // digit histograms of the segment's candidates (for the ranking passes)
+  for (int i = threadIdx.x; i < kSortPasses * kDigits; i += kSelThreads) s_dhist[i] = 0;
+  __syncthreads();
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -317,7 +333,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
   unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;
-  constexpr uint32_t kTileVec = kSelectThreads * kSelectVecPerThread;  // 2048 float4 = 8192 coordinates
+  constexpr uint32_t kTileVec = kSelTileVec;
   int parity = 0;
   __shared__ uint32_t s_chunk;
 
@@ -341,6 +357,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
     const uint32_t thresh = plan->thresh_bin << 19;
     const float thresh_f = __uint_as_float(thresh);  // finite inputs: |x| >= thresh_f <=> key >= thresh
+    const uint32_t keytop = sort_keytop(plan);
     const uint32_t seg = q + c;
     unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     unsigned long long run = seg_prefix[seg];
@@ -357,14 +374,14 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         const uint64_t base = (uint64_t)t * kTileVec;
         if (base + kTileVec <= n_vec) {
 #pragma unroll
-          for (int v = 0; v < kSelectVecPerThread; ++v) {
-            const uint32_t g = v * kSelectThreads + tid;
+          for (int v = 0; v < kSelVec; ++v) {
+            const uint32_t g = v * kSelThreads + tid;
             cp_async16(dst + sel_slot(g), xseg + base + g);
           }
         } else {
 #pragma unroll
-          for (int v = 0; v < kSelectVecPerThread; ++v) {
-            const uint32_t g = v * kSelectThreads + tid;
+          for (int v = 0; v < kSelVec; ++v) {
+            const uint32_t g = v * kSelThreads + tid;
             if (base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
           }
         }
@@ -385,10 +402,10 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       const uint64_t base = (uint64_t)t * kTileVec;
       // this thread's 16 consecutive coordinates: units 4 tid .. 4 tid + 3 of the tile
       uint32_t m = 0;
-      const uint32_t g0 = 4u * tid;
-      const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < 4) ? n_vec - base - g0 : 4) : 0u;
+      const uint32_t g0 = (uint32_t)kSelVec * tid;
+      const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < kSelVec) ? n_vec - base - g0 : kSelVec) : 0u;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < kSelVec; ++j) {
         if ((uint32_t)j < left) {
           const float4 f = src[sel_slot(g0 + j)];
           m |= (fabsf(f.x) >= thresh_f ? 1u : 0u) << (4 * j);
@@ -398,7 +415,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         }
       }
       const uint32_t cnt = __popc(m);
-      // block scan of the per-thread counts: inside the warp, then over the 16 warp totals
+      // block scan of the per-thread counts: inside the warp, then over the warp totals
       uint32_t incl = cnt;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -407,14 +424,14 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       }
       if (lane == 31) s_warp_incl[parity][warp] = incl;
       __syncthreads();
-      const uint32_t wt = (lane < kSelectThreads / 32) ? s_warp_incl[parity][lane] : 0u;
+      const uint32_t wt = (lane < kSelThreads / 32) ? s_warp_incl[parity][lane] : 0u;
       uint32_t wincl = wt;
 #pragma unroll
-      for (int off = 1; off < kSelectThreads / 32; off <<= 1) {
+      for (int off = 1; off < kSelThreads / 32; off <<= 1) {
         const uint32_t o = __shfl_up_sync(kFull, wincl, off);
         if (lane >= off) wincl += o;
       }
-      const uint32_t tot = __shfl_sync(kFull, wincl, kSelectThreads / 32 - 1);
+      const uint32_t tot = __shfl_sync(kFull, wincl, kSelThreads / 32 - 1);
       const uint32_t below = __shfl_sync(kFull, wincl - wt, warp);
       parity ^= 1;
       // emit this thread's candidates (few): values are re-read from the staging buffer
@@ -425,9 +442,11 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         const int bit = __ffs(m) - 1;
         m &= m - 1;
         const uint32_t b = srcw[sel_slot(g0 + (bit >> 2)) * 4 + (bit & 3)];
-        if (o < L.capacity)
-          out[o] = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) |
-                   (unsigned long long)(e_base + bit);
+        const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) |
+                                        (unsigned long long)(e_base + bit);
+        if (o < L.capacity) out[o] = pair;
+#pragma unroll
+        for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + sort_digit(pair, p, keytop)], 1u);
         ++o;
       }
       run += tot;
@@ -438,8 +457,9 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       for (uint64_t e = nvec * 4; e < d; ++e) {
         const uint32_t b = __float_as_uint(x[e]);
         if ((b & 0x7FFFFFFFu) >= thresh) {
-          if (run < L.capacity)
-            out[run] = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) | (unsigned long long)e;
+          const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) | (unsigned long long)e;
+          if (run < L.capacity) out[run] = pair;
+          for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + sort_digit(pair, p, keytop)], 1u);
           ++run;
         }
       }
@@ -450,6 +470,16 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       if (with_tail) n_selected[c] = run;
     }
     __syncthreads();  // the staging buffers (and the ticket word) are reused by the next segment
+    {
+      // the segment's digit counts join the client's
+      unsigned long long* ghist = reinterpret_cast<unsigned long long*>(ws + L.off_ghist) + (size_t)c * kSortPasses * kDigits;
+      for (int i = tid; i < kSortPasses * kDigits; i += kSelThreads) {
+        const uint32_t v = s_dhist[i];
+        s_dhist[i] = 0;
+        if (v) atomicAdd(ghist + i, (unsigned long long)v);
+      }
+      __syncthreads();
+    }
     pos = seg_end;
   }
   }
@@ -465,14 +495,6 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
 // the clients interleaved; decoupled look-back per digit value).  A pass whose digit is the same
 // for every candidate of a client (normally the fourth) is skipped for that client; which buffer
 // holds its data after pass q follows from the mask of skipped passes.
-
-__device__ __forceinline__ uint32_t sort_keytop(const cvlc_plan_t* plan) { return ((plan->top_bin + 1u) << 19) - 1u; }
-
-__device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass, uint32_t keytop) {
-  const uint32_t key = (uint32_t)(pair >> 32);
-  const uint32_t inv = key > keytop ? 0u : keytop - key;  // key > keytop only if the plan is not of this update
-  return (inv >> (kDigitBits * pass)) & (kDigits - 1);
-}
 
 // The clients' candidate arrays are concatenated in units of sort tiles (2048 pairs) and cut
 // into equal contiguous chunks, one per block; a block that crosses a client boundary merges
@@ -927,7 +949,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   }
   if (pws) {
     LaunchScope ls(kKSelect, st);
-    k_select<CAP><<<part.grid, kSelectThreads, kSelStages * kSelStageBytes, st>>>(batch, shape.d, part, pws, w, L);
+    k_select<CAP><<<part.grid, kSelThreads, kSelStages * kSelStageBytes, st>>>(batch, shape.d, part, pws, w, L);
   } else {
     const uint64_t want = L.select_tiles * n;
     const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
@@ -937,7 +959,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   {
     const uint64_t want = L.sort_tiles_max * n;
     const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
-    {
+    if (!pws) {  // the selection with known offsets has counted the digits already
       LaunchScope ls(kKSortHist, st);
       k_sort_hist<CAP><<<grid, 256, 0, st>>>(batch, w, L);
     }

@@ -369,6 +369,13 @@ def run_ours(args):
         "per_step_ms": per,
         "plan_of_client_0": {"k": int(plans[0].k), "R": int(plans[0].R), "n_candidates": int(plans[0].n_candidates), "alpha_q": plans[0].alpha_q,
                  "lengths": {str(y): int(plans[0].n_y[y]) for y in range(33) if plans[0].n_y[y]}},
+        "phase_ms_per_step": {
+            "plan": sum(kernels[k]["ms_per_step"] for k in ("k_zero_words", "k_hist", "k_plan") if k in kernels),
+            "encode": sum(kernels[k]["ms_per_step"] for k in ("k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
+                                                                "k_sort_scan", "k_sort_pass", "k_pack") if k in kernels),
+            "decode_aggregate": sum(kernels[k]["ms_per_step"] for k in ("k_decode_prepare", "k_fill_zero", "k_decode")
+                                    if k in kernels)},
+        "step_min_bytes_frac_of_nominal_8TBps": step_min_bytes / (ms_per_step * 1e-3) / 8e12,
         "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(gpu_launches),
         "clocks": clocks,
     }

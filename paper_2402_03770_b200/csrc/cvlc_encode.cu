@@ -573,16 +573,18 @@ k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
 }
 
 template <int CAP>
-__global__ void __launch_bounds__(kSortThreads)
+__global__ void __launch_bounds__(kSortThreads, 4)
 k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
+  constexpr int kWarps = kSortThreads / 32;
+  static_assert(kWarps == 8, "one 128-bit shared-memory word holds the eight warps' 16-bit counters of a digit value");
+  constexpr int kPerThread = kDigits / kSortThreads;  // digit values owned by a thread
   __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_wc[kSortThreads / 32][kDigits];  // per-warp digit counters -> per-warp offsets
-  __shared__ unsigned long long s_base[kDigits];         // position of this tile's first item per digit
-  __shared__ uint32_t s_dstart[kDigits];                 // first slot of every digit value inside the tile
-  __shared__ uint32_t s_scan_w[kSortThreads / 32];
+  __shared__ __align__(16) uint16_t s_wc[kDigits][kWarps];  // per digit value: the warps' counters, then their first slots
+  __shared__ unsigned long long s_gofs[kDigits];           // global position of slot 0 of the tile, per digit value
+  __shared__ uint32_t s_scan_w[kWarps];
   extern __shared__ unsigned long long s_dyn[];
-  unsigned long long* s_items = s_dyn;                                         // [kSortTile] the tile's items in digit order
-  uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_dyn + kSortTile);         // [n + 1] first sort tile of every client
+  unsigned long long* s_items = s_dyn;                                  // [kSortTile] the tile's items in digit order
+  uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_dyn + kSortTile);  // [n + 1] first sort tile of every client
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -597,14 +599,12 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
   unsigned long long* state_all =
       reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)pass * n_clients * L.sort_tiles_max * kDigits;
   const unsigned lanemask_lt = (1u << lane) - 1u;
-  constexpr int kPerThread = kDigits / kSortThreads;  // digit values owned by a thread
+  uint4* s_wc4 = reinterpret_cast<uint4*>(&s_wc[0][0]);
 
   while (true) {
     if (tid == 0) s_tile = atomicAdd(&hdr->sort_ticket[pass], 1u);
 #pragma unroll
-    for (int w = 0; w < kSortThreads / 32; ++w)
-#pragma unroll
-      for (int q = 0; q < kPerThread; ++q) s_wc[w][tid + q * kSortThreads] = 0;
+    for (int q = 0; q < kPerThread; ++q) s_wc4[tid + q * kSortThreads] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     const uint32_t gt = s_tile;
     if (gt >= total_tickets) break;
@@ -637,22 +637,30 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
       const unsigned long long idx = first + i * 32 + lane;
       item[i] = (idx < n) ? src[idx] : ~0ull;
     }
-    // stable rank inside the warp: items in (i, lane) order
+    // stable rank inside the warp: items in (i, lane) order.  The lanes holding the same digit value are
+    // found by intersecting the ballots of its nine bits (a match instruction costs as many steps as
+    // there are distinct values in the warp, about thirty here).
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       const bool valid = (first + i * 32 + lane) < n;
-      const uint32_t dig = valid ? sort_digit(item[i], pass, keytop) : 0xFFFFFFFFu;
-      const unsigned peers = __match_any_sync(kFull, dig);
-      const int leader = __ffs(peers) - 1;
+      const uint32_t dig = valid ? sort_digit(item[i], pass, keytop) : 0u;
+      unsigned peers = __ballot_sync(kFull, valid);
+#pragma unroll
+      for (int b = 0; b < kDigitBits; ++b) {
+        const unsigned bal = __ballot_sync(kFull, (dig >> b) & 1u);
+        peers &= ((dig >> b) & 1u) ? bal : ~bal;
+      }
+      const int leader = __ffs(peers | (valid ? 0u : 1u << lane)) - 1;
       uint32_t pre = 0;
-      if (valid && lane == leader) pre = s_wc[warp][dig];
+      if (valid && lane == leader) pre = s_wc[dig][warp];
       pre = __shfl_sync(kFull, pre, leader);
       rank[i] = pre + __popc(peers & lanemask_lt);
-      if (valid && lane == leader) s_wc[warp][dig] = pre + __popc(peers);
+      if (valid && lane == leader) s_wc[dig][warp] = (uint16_t)(pre + __popc(peers));
       __syncwarp();
     }
     __syncthreads();
-    // thread = digit values tid, tid + 256: offsets of the warps inside the tile, tile count, look-back
+    // thread = digit values tid, tid + 256: the warps' counts of the value (one 128-bit word), the tile
+    // count, the value's first slot inside the tile (block scan in digit order), look-back
     {
       uint32_t tot[kPerThread];
       unsigned long long run[kPerThread];
@@ -660,20 +668,17 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 #pragma unroll
       for (int q = 0; q < kPerThread; ++q) {
         const int dg = tid + q * kSortThreads;
+        const uint4 cw = s_wc4[dg];
+        const uint32_t w32[4] = {cw.x, cw.y, cw.z, cw.w};
         uint32_t t = 0;
 #pragma unroll
-        for (int w = 0; w < kSortThreads / 32; ++w) {
-          const uint32_t cnt = s_wc[w][dg];
-          s_wc[w][dg] = t;
-          t += cnt;
-        }
+        for (int h = 0; h < 4; ++h) t += (w32[h] & 0xFFFFu) + (w32[h] >> 16);
         tot[q] = t;
         run[q] = 0;
         open[q] = tile > 0;
         st_relaxed(state + (size_t)tile * kDigits + dg, (tile == 0 ? kFlagPrefix : kFlagAgg) | t);
       }
-      // first slot of every digit value inside the tile: exclusive scan of the tile's digit counts in digit
-      // order (thread t owns digits t and t + 256), done while the look-back loads are in flight
+      uint32_t dstart[kPerThread];
       {
         uint32_t carry = 0;
 #pragma unroll
@@ -688,15 +693,31 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
           __syncthreads();
           uint32_t below = 0, all = 0;
 #pragma unroll
-          for (int w = 0; w < kSortThreads / 32; ++w) {
+          for (int w = 0; w < kWarps; ++w) {
             const uint32_t v = s_scan_w[w];
             if (w < warp) below += v;
             all += v;
           }
-          s_dstart[tid + q * kSortThreads] = carry + below + incl - tot[q];
+          dstart[q] = carry + below + incl - tot[q];
           carry += all;
           __syncthreads();
         }
+      }
+      // the counters become first slots: slot of (value, warp) = first slot of the value + items of earlier warps
+#pragma unroll
+      for (int q = 0; q < kPerThread; ++q) {
+        const uint4 cw = s_wc4[tid + q * kSortThreads];
+        const uint32_t c32[4] = {cw.x, cw.y, cw.z, cw.w};
+        uint32_t w32[4], t = dstart[q];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const uint32_t lo16 = t;
+          t += c32[h] & 0xFFFFu;
+          const uint32_t hi16 = t;
+          t += c32[h] >> 16;
+          w32[h] = (lo16 & 0xFFFFu) | (hi16 << 16);
+        }
+        s_wc4[tid + q * kSortThreads] = make_uint4(w32[0], w32[1], w32[2], w32[3]);
       }
       for (long long t = (long long)tile - 1; t >= 0; --t) {
         bool any_open = false;
@@ -715,15 +736,16 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
       for (int q = 0; q < kPerThread; ++q) {
         const int dg = tid + q * kSortThreads;
         if (tile > 0) st_relaxed(state + (size_t)tile * kDigits + dg, kFlagPrefix | (run[q] + tot[q]));
-        s_base[dg] = gbase[dg] + run[q];
+        s_gofs[dg] = gbase[dg] + run[q] - dstart[q];
       }
     }
+    __syncthreads();
     // the items go to shared memory in digit order, then out in runs of consecutive addresses
 #pragma unroll
     for (int i = 0; i < kSortItemsPerThread; ++i) {
       if ((first + i * 32 + lane) < n) {
         const uint32_t dig = sort_digit(item[i], pass, keytop);
-        s_items[s_dstart[dig] + s_wc[warp][dig] + rank[i]] = item[i];
+        s_items[(uint32_t)s_wc[dig][warp] + rank[i]] = item[i];
       }
     }
     __syncthreads();
@@ -732,8 +754,7 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
       const uint32_t count = (n - tile_first < (unsigned long long)kSortTile) ? (uint32_t)(n - tile_first) : (uint32_t)kSortTile;
       for (uint32_t k = tid; k < count; k += kSortThreads) {
         const unsigned long long it = s_items[k];
-        const uint32_t dig = sort_digit(it, pass, keytop);
-        const unsigned long long o = s_base[dig] + (k - s_dstart[dig]);
+        const unsigned long long o = s_gofs[sort_digit(it, pass, keytop)] + k;
         if (o < n && o < L.capacity) dst[o] = it;
       }
     }

@@ -103,6 +103,12 @@ def lib() -> C.CDLL:
         L.cvlc_pq_quantize_oracle.argtypes = [C.c_float, C.c_float, C.c_float, u32, u32]
         L.cvlc_pq_dequantize_oracle.restype = C.c_float
         L.cvlc_pq_dequantize_oracle.argtypes = [u32, C.c_float, C.c_float, u32]
+        L.cvlc_qsgd_norm_oracle.restype = C.c_float
+        L.cvlc_qsgd_norm_oracle.argtypes = [C.POINTER(C.c_float), u32]
+        L.cvlc_qsgd_quantize_oracle.restype = u32
+        L.cvlc_qsgd_quantize_oracle.argtypes = [C.c_float, C.c_float, u32, u32]
+        L.cvlc_qsgd_dequantize_oracle.restype = C.c_float
+        L.cvlc_qsgd_dequantize_oracle.argtypes = [u32, C.c_float, u32]
         L.cvlc_encode_oracle.restype = C.c_int
         L.cvlc_encode_oracle.argtypes = [C.c_void_p, P(OrcParams), P(OrcPlan), C.c_void_p, C.c_size_t,
                                          C.c_void_p]
@@ -240,6 +246,19 @@ def pq_quantize(x: float, lo: float, hi: float, y: int, rnd: int) -> int:
 
 def pq_dequantize(code: int, lo: float, hi: float, y: int) -> float:
     return float(lib().cvlc_pq_dequantize_oracle(code, lo, hi, y))
+
+
+def qsgd_norm(v: np.ndarray) -> float:
+    v = _f32(v)
+    return float(lib().cvlc_qsgd_norm_oracle(v.ctypes.data_as(C.POINTER(C.c_float)), v.size))
+
+
+def qsgd_quantize(x: float, norm: float, y: int, rnd: int) -> int:
+    return int(lib().cvlc_qsgd_quantize_oracle(x, norm, y, rnd))
+
+
+def qsgd_dequantize(code: int, norm: float, y: int) -> float:
+    return float(lib().cvlc_qsgd_dequantize_oracle(code, norm, y))
 
 
 def encode(x: np.ndarray, p: OrcParams, pl: OrcPlan, want_rank: bool = False):

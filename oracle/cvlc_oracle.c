@@ -9,6 +9,7 @@
  */
 #include "cvlc_oracle.h"
 
+#include <float.h>
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
@@ -165,7 +166,7 @@ static int params_ok(const orc_params* p) {
   if (p->d < 2 || p->d > ((uint64_t)1 << 31)) return 0;
   if (p->packet_bits == 0 || (p->packet_bits % 32) != 0) return 0;
   if (p->header_bits < 80 || p->header_bits >= p->packet_bits) return 0;
-  if (p->quantizer != 0) return 0;
+  if (p->quantizer != ORC_QUANT_PQ && p->quantizer != ORC_QUANT_QSGD) return 0;
   if (p->max_code_bits < 1 || p->max_code_bits > ORC_MAX_Y) return 0;
   if (!(p->scale_B >= 1.0) || !(p->scale_B < 1e300)) return 0;
   return 1;
@@ -193,9 +194,24 @@ size_t cvlc_stream_bytes_oracle(const orc_params* p) {
   return (size_t)(64 + R * (p->packet_bits / 8));
 }
 
-/* Quantization error factor of PQ with P = cap(y) values at y bits:
- * Q = P / (2^y - 1)^2 (Appendix, case study). */
-static double Q_of(uint32_t cap_y, uint32_t y) {
+/* Magnitude levels of a y-bit QSGD code.  The paper gives every record y bits and lets
+ * QSGD quantize absolute values; it does not say where the sign goes.  Here the top bit of
+ * the code is the sign and the other y - 1 bits hold a level 0..s_q, s_q = 2^(y-1) - 1, so a
+ * record stays s + y bits wide and Eq. (3) holds unchanged.  One bit cannot hold a level. */
+static uint32_t qsgd_levels(uint32_t y) { return (y >= 2) ? (uint32_t)((((uint64_t)1) << (y - 1)) - 1) : 0u; }
+
+/* Quantization error factor with P = cap(y) values at y bits (Appendix, case study).
+ * PQ:   Q = P / (2^y - 1)^2, 2^y - 1 being the intervals between its 2^y centroids.
+ * QSGD: Q = min(P / s_q^2, sqrt(P) / s_q), the paper's min(Q_1, Q_2) with its level count
+ *       (printed as 2^y) replaced by the s_q levels the record format really has. */
+static double Q_of(uint32_t quantizer, uint32_t cap_y, uint32_t y) {
+  if (quantizer == ORC_QUANT_QSGD) {
+    if (y < 2) return INFINITY;
+    double sq = (double)qsgd_levels(y);
+    double Q1 = (double)cap_y / (sq * sq);
+    double Q2 = sqrt((double)cap_y) / sq;
+    return (Q1 < Q2) ? Q1 : Q2;
+  }
   double L = (double)(((uint64_t)1 << y) - 1);
   return (double)cap_y / (L * L);
 }
@@ -203,7 +219,7 @@ static double Q_of(uint32_t cap_y, uint32_t y) {
 double cvlc_quant_error_Q_oracle(const orc_params* p, uint32_t y) {
   uint32_t s, R, cap[ORC_MAX_Y + 1];
   if (cvlc_derive_oracle(p, &s, &R, cap) != ORC_OK || y < 1 || y > p->max_code_bits) return NAN;
-  return Q_of(cap[y], y);
+  return Q_of(p->quantizer, cap[y], y);
 }
 
 /* The bracket of Eq. (5) is c = Q/B^2 + 1/B_c^2 with 1/B_c = 1 - 1/B; g = 1 - c is
@@ -228,7 +244,7 @@ double cvlc_default_scale_oracle(const orc_params* p) {
   uint32_t s = 1;
   while (((uint64_t)1 << s) < p->d) ++s;
   uint32_t cap8 = (p->packet_bits - p->header_bits) / (s + 8);
-  return 1.0 + Q_of(cap8, 8);
+  return 1.0 + Q_of(p->quantizer, cap8, 8);
 }
 
 /* Planner context: candidate lengths and their coefficients */
@@ -256,7 +272,7 @@ static int ctx_init(plan_ctx* c, const orc_params* p, uint32_t* s_out) {
   c->y_min = 0;
   c->nY = 0;
   for (uint32_t y = 1; y <= p->max_code_bits; ++y) {
-    c->Q[y] = Q_of(c->cap[y], y);
+    c->Q[y] = Q_of(p->quantizer, c->cap[y], y);
     c->g[y] = g_of(c->Q[y], p->scale_B);
     if (c->y_min == 0 && c->g[y] > 0.0) c->y_min = y;
   }
@@ -431,6 +447,7 @@ int cvlc_plan_oracle(const float* x, const orc_params* p, orc_plan* plan) {
 int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan) {
   if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
   if (y < 1 || y > p->max_code_bits) return ORC_ERR_INVALID_ARG;
+  if (p->quantizer == ORC_QUANT_QSGD && y < 2) return ORC_ERR_INVALID_ARG;
   plan_ctx c;
   uint32_t s;
   int rc = ctx_init(&c, p, &s);
@@ -439,7 +456,7 @@ int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan) {
   /* evaluate gamma with the single length y as the only candidate */
   c.nY = 1;
   c.Y[0] = y;
-  c.Q[y] = Q_of(c.cap[y], y);
+  c.Q[y] = Q_of(p->quantizer, c.cap[y], y);
   c.g[y] = g_of(c.Q[y], p->scale_B);
   c.y_min = y;
   ctx_set_beta(&c, 2.0 * (-1.0) + 1.0);
@@ -497,6 +514,50 @@ float cvlc_pq_dequantize_oracle(uint32_t code, float lo, float hi, uint32_t y) {
   double L = (double)(((uint64_t)1 << y) - 1);
   double den = (double)hi - (double)lo;
   return (float)((double)lo + (double)code * (den / L));
+}
+
+/* ======================================================================== */
+/* QSGD stochastic quantization (Alistarh et al.): |x| / ||segment||_2 is      */
+/* rounded up or down onto the grid {0, 1/s_q, ..., 1}, unbiased; the sign is  */
+/* kept.  Section IV-C: the header carries the l2-norm as the centroid         */
+/* distribution (32 bits).                                                     */
+/* ======================================================================== */
+
+/* l2-norm of a packet's values: squares (exact in double) added in rank order in double,
+ * square root, rounded to fp32; a result beyond the fp32 range is stored as FLT_MAX. */
+float cvlc_qsgd_norm_oracle(const float* v, uint32_t n) {
+  double sum = 0.0;
+  for (uint32_t j = 0; j < n; ++j) sum = sum + (double)v[j] * (double)v[j];
+  double r = sqrt(sum);
+  if (r > (double)FLT_MAX) return FLT_MAX;
+  return (float)r;
+}
+
+/* code = sign bit (bit y-1) | level (bits 0..y-2) */
+uint32_t cvlc_qsgd_quantize_oracle(float x, float norm, uint32_t y, uint32_t rnd) {
+  uint32_t sq = qsgd_levels(y);
+  uint32_t sign = (x < 0.0f) ? 1u : 0u;
+  uint32_t level = 0;
+  if (norm > 0.0f) {
+    double a = fabs((double)x);
+    double t = (a / (double)norm) * (double)sq;
+    double j0 = floor(t);
+    if (j0 > (double)sq) j0 = (double)sq;
+    double frac = t - j0;
+    double u = (double)rnd * (1.0 / 4294967296.0);
+    level = (uint32_t)j0;
+    if (u < frac) level += 1;
+    if (level > sq) level = sq; /* only when |x| > norm, i.e. the norm was cut to FLT_MAX */
+  }
+  return (sign << (y - 1)) | level;
+}
+
+float cvlc_qsgd_dequantize_oracle(uint32_t code, float norm, uint32_t y) {
+  uint32_t sq = qsgd_levels(y);
+  uint32_t level = code & sq; /* s_q = 2^(y-1) - 1 is also the mask of the level bits */
+  double mag = (double)level * ((double)norm / (double)sq);
+  float v = (float)mag;
+  return ((code >> (y - 1)) & 1u) ? -v : v;
 }
 
 /* ======================================================================== */
@@ -592,21 +653,36 @@ int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan
     for (uint32_t q = 0; q < plan->n_y[y]; ++q, ++r) {
       uint8_t* pkt = stream + 64 + (size_t)r * pkt_bytes;
       uint32_t P = cap[y];
-      /* centroid distribution of PQ: minimum and maximum of the packet's values */
-      float lo = canon(x[rank[Z]]), hi = lo;
-      for (uint32_t j = 1; j < P; ++j) {
-        float v = canon(x[rank[Z + j]]);
-        if (v < lo) lo = v;
-        if (v > hi) hi = v;
-      }
+      float lo = 0.0f, hi = 0.0f, norm = 0.0f;
       put_bits(pkt, 0, s, 8);
       put_bits(pkt, 8, (uint64_t)y, 8);
-      put_bits(pkt, 16, float_bits(lo), 32);
-      put_bits(pkt, 48, float_bits(hi), 32);
+      if (p->quantizer == ORC_QUANT_QSGD) {
+        /* centroid distribution of QSGD: the l2-norm of the packet's values (32 bits) */
+        if (y < 2) { free(rank); return ORC_ERR_INVALID_ARG; }
+        float* seg = (float*)malloc(sizeof(float) * (size_t)P);
+        if (!seg) { free(rank); return ORC_ERR_INVALID_ARG; }
+        for (uint32_t j = 0; j < P; ++j) seg[j] = canon(x[rank[Z + j]]);
+        norm = cvlc_qsgd_norm_oracle(seg, P);
+        free(seg);
+        put_bits(pkt, 16, float_bits(norm), 32);
+      } else {
+        /* centroid distribution of PQ: minimum and maximum of the packet's values (64 bits) */
+        lo = canon(x[rank[Z]]);
+        hi = lo;
+        for (uint32_t j = 1; j < P; ++j) {
+          float v = canon(x[rank[Z + j]]);
+          if (v < lo) lo = v;
+          if (v > hi) hi = v;
+        }
+        put_bits(pkt, 16, float_bits(lo), 32);
+        put_bits(pkt, 48, float_bits(hi), 32);
+      }
       for (uint32_t j = 0; j < P; ++j) {
         uint32_t pid = rank[Z + j];
         uint32_t rnd = cvlc_philox_coord_oracle(p->seed, p->client_id, p->round, pid);
-        uint32_t code = cvlc_pq_quantize_oracle(canon(x[pid]), lo, hi, (uint32_t)y, rnd);
+        uint32_t code = (p->quantizer == ORC_QUANT_QSGD)
+                            ? cvlc_qsgd_quantize_oracle(canon(x[pid]), norm, (uint32_t)y, rnd)
+                            : cvlc_pq_quantize_oracle(canon(x[pid]), lo, hi, (uint32_t)y, rnd);
         uint64_t bitpos = (uint64_t)p->header_bits + (uint64_t)j * (s + (uint32_t)y);
         put_bits(pkt, bitpos, pid, s);
         put_bits(pkt, bitpos + s, code, (uint32_t)y);
@@ -624,7 +700,7 @@ int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan
 /* ======================================================================== */
 
 typedef struct {
-  uint32_t s, R, packet_bits, header_bits;
+  uint32_t s, R, packet_bits, header_bits, quantizer;
   uint64_t d;
   double B;
 } stream_head;
@@ -633,7 +709,8 @@ static int parse_head(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_hea
   if (nbytes < 64) return ORC_ERR_BAD_STREAM;
   if (get_le(st, 4) != 0x434C5643u) return ORC_ERR_BAD_STREAM;
   if (get_le(st + 4, 2) != 1) return ORC_ERR_BAD_STREAM;
-  if (get_le(st + 6, 1) != 0) return ORC_ERR_BAD_STREAM;
+  h->quantizer = (uint32_t)get_le(st + 6, 1);
+  if (h->quantizer != ORC_QUANT_PQ && h->quantizer != ORC_QUANT_QSGD) return ORC_ERR_BAD_STREAM;
   h->s = (uint32_t)get_le(st + 7, 1);
   h->d = get_le(st + 8, 8);
   h->R = (uint32_t)get_le(st + 16, 4);
@@ -677,13 +754,19 @@ int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* 
       y_prev = y;
       float lo = bits_float((uint32_t)get_bits(pkt, 16, 32));
       float hi = bits_float((uint32_t)get_bits(pkt, 48, 32));
+      if (h.quantizer == ORC_QUANT_QSGD) {
+        /* lo is the norm field: a finite, non-negative fp32; the code needs a sign and a level bit */
+        uint32_t nb = (uint32_t)get_bits(pkt, 16, 32);
+        if (y < 2 || nb >= 0x7F800000u) { rc = ORC_ERR_BAD_STREAM; break; }
+      }
       uint32_t P = (h.packet_bits - h.header_bits) / (s + y);
       for (uint32_t j = 0; j < P; ++j) {
         uint64_t bitpos = (uint64_t)h.header_bits + (uint64_t)j * (s + y);
         uint64_t pid = get_bits(pkt, bitpos, s);
         uint32_t code = (uint32_t)get_bits(pkt, bitpos + s, y);
         if (pid >= d) { rc = ORC_ERR_BAD_STREAM; break; }
-        float v = cvlc_pq_dequantize_oracle(code, lo, hi, y);
+        float v = (h.quantizer == ORC_QUANT_QSGD) ? cvlc_qsgd_dequantize_oracle(code, lo, y)
+                                                  : cvlc_pq_dequantize_oracle(code, lo, hi, y);
         acc[pid] = acc[pid] + (double)coef * (double)v;
       }
       if (rc != ORC_OK) break;

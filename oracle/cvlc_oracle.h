@@ -39,13 +39,15 @@ enum {
 
 #define ORC_HIST_BINS 4096
 #define ORC_MAX_Y 32
+#define ORC_QUANT_PQ 0u   /* uniform centroids on [min, max] of the packet (Suresh et al.) */
+#define ORC_QUANT_QSGD 1u /* sign and level of |x| / l2-norm of the packet (Alistarh et al.) */
 
 typedef struct {
   uint64_t d;             /* number of coordinates */
   uint64_t budget_bits;   /* uplink budget of this client this round, bits */
   uint32_t packet_bits;   /* b  (Section IV-C: 1500 bytes) */
   uint32_t header_bits;   /* H  (Eq. (2)) */
-  uint32_t quantizer;     /* 0 = PQ */
+  uint32_t quantizer;     /* ORC_QUANT_PQ or ORC_QUANT_QSGD */
   uint32_t max_code_bits; /* largest candidate code length, <= 32 */
   double scale_B;         /* B of the scaling operation (Section IV-B) */
   uint64_t seed;          /* Philox key */
@@ -84,7 +86,7 @@ void cvlc_alpha_fit_oracle(const uint64_t h[ORC_HIST_BINS], uint64_t d, double* 
 int cvlc_derive_oracle(const orc_params* p, uint32_t* s, uint32_t* R, uint32_t cap[ORC_MAX_Y + 1]);
 double cvlc_default_scale_oracle(const orc_params* p);
 size_t cvlc_stream_bytes_oracle(const orc_params* p);
-/* coefficient g(y) = 1 - (Q(y)/B^2 + (1-1/B)^2) of Eq. (5); Q of PQ (Appendix, case study) */
+/* coefficient g(y) = 1 - (Q(y)/B^2 + (1-1/B)^2) of Eq. (5); Q of the chosen quantizer (Appendix, case study) */
 double cvlc_coeff_g_oracle(const orc_params* p, uint32_t y);
 double cvlc_quant_error_Q_oracle(const orc_params* p, uint32_t y);
 /* F(n) = 1 - gamma for packet counts n_y (index = code length) at exponent beta; -inf if inadmissible */
@@ -100,6 +102,10 @@ int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan);
 int cvlc_rank_oracle(const float* x, uint64_t d, uint64_t k, uint32_t* idx_out);
 uint32_t cvlc_pq_quantize_oracle(float x, float lo, float hi, uint32_t y, uint32_t rnd);
 float cvlc_pq_dequantize_oracle(uint32_t code, float lo, float hi, uint32_t y);
+/* QSGD: y >= 2; code = sign << (y-1) | level, level in 0..2^(y-1)-1 */
+float cvlc_qsgd_norm_oracle(const float* v, uint32_t n);
+uint32_t cvlc_qsgd_quantize_oracle(float x, float norm, uint32_t y, uint32_t rnd);
+float cvlc_qsgd_dequantize_oracle(uint32_t code, float norm, uint32_t y);
 int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan, uint8_t* stream,
                        size_t capacity, uint32_t* ranked_idx_out /* k entries or NULL */);
 

@@ -1,6 +1,7 @@
 """An independent reader of the packet stream, written from the format definition
-(global header + fixed-size packets; packet = header {s, y_r, min, max} + (PID, CID)
-pairs, Fig. 2 of the paper), used by the tests to check both encoders.  It shares
+(global header + fixed-size packets; packet = header {s, y_r, centroid distribution} +
+(PID, CID) pairs, Fig. 2 of the paper; the centroid distribution is {min, max} for PQ and
+{l2-norm, 0} for QSGD), used by the tests to check both encoders.  It shares
 no code with the oracle or with the CUDA library."""
 from __future__ import annotations
 
@@ -88,3 +89,13 @@ def dequantize(pk: Packet) -> np.ndarray:
     L = float(2 ** pk.y - 1)
     step = (np.float64(pk.hi) - np.float64(pk.lo)) / L
     return (np.float64(pk.lo) + pk.cid.astype(np.float64) * step).astype(np.float32)
+
+
+def dequantize_qsgd(pk: Packet) -> np.ndarray:
+    """QSGD record: top bit of the CID = sign, the rest = level on a grid of 2^(y-1) - 1 steps
+    of the packet's l2-norm (kept in the first centroid field)."""
+    sq = 2 ** (pk.y - 1) - 1
+    level = (pk.cid & np.uint64(sq)).astype(np.float64)
+    negative = ((pk.cid >> np.uint64(pk.y - 1)) & np.uint64(1)).astype(bool)
+    mag = (level * (np.float64(pk.lo) / np.float64(sq))).astype(np.float32)
+    return np.where(negative, -mag, mag).astype(np.float32)

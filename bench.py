@@ -47,6 +47,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18")
     ap.add_argument("--bits-per-coord", type=float, default=2.0)
+    ap.add_argument("--quantizer", default="pq", choices=["pq", "qsgd"], help="the two quantizers of the paper's experiments")
     ap.add_argument("--clients", type=int, default=0, help="0 = the workload's client count")
     ap.add_argument("--d", type=int, default=0, help="0 = the workload's d (smaller values are for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="clients per plan/encode call; 0 = all clients in one call")
@@ -124,7 +125,10 @@ class ClockSampler:
 # reference arm: the CPU oracle as it stands, on a bounded sample of the workload
 # --------------------------------------------------------------------------------------------
 
-def oracle_step(w, d, bpc, clients):
+QUANTIZERS = {"pq": 0, "qsgd": 1}
+
+
+def oracle_step(w, d, bpc, clients, quantizer=0):
     """plan + encode of `clients`, then decode-aggregate of their streams; returns seconds"""
     import oracle as O
     xs = [W.client_update(w, c, d=d) for c in clients]
@@ -133,7 +137,7 @@ def oracle_step(w, d, bpc, clients):
     streams = []
     for c, x in zip(clients, xs):
         seed, cid, rnd = W.philox_ids(w, c)
-        p = O.make_params(d, int(np.floor(bpc * d)), seed=seed, client_id=cid, round=rnd)
+        p = O.make_params(d, int(np.floor(bpc * d)), seed=seed, client_id=cid, round=rnd, quantizer=quantizer)
         streams.append(O.encode(x, p, O.plan(x, p)))
     O.decode_aggregate(streams, weights, d)
     return time.perf_counter() - t0
@@ -148,8 +152,8 @@ def run_reference(args):
     n = max(1, args.cpu_sample_clients)
     clients = list(range(n))
     for _ in range(min(args.warmup, 1)):
-        oracle_step(w, d, args.bits_per_coord, clients[:1])
-    times = [oracle_step(w, d, args.bits_per_coord, clients) for _ in range(args.steps)]
+        oracle_step(w, d, args.bits_per_coord, clients[:1], QUANTIZERS[args.quantizer])
+    times = [oracle_step(w, d, args.bits_per_coord, clients, QUANTIZERS[args.quantizer]) for _ in range(args.steps)]
     t = float(np.mean(times))
     value = 4.0 * d * n / t / 1e9
     sample = f"{n} of {args.clients or w.n_clients} clients per step (plan+encode each, decode-aggregate of those {n})"
@@ -157,7 +161,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64 plan / f32 data", "data": "synthetic",
-        "config": {"workload": f"{w.name} d={d} bits_per_coord={args.bits_per_coord}", "sample": sample},
+        "config": {"workload": f"{w.name} d={d} bits_per_coord={args.bits_per_coord} quantizer={args.quantizer}", "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "params_per_s": d * n / t,
@@ -203,7 +207,7 @@ def run_ours(args):
     params = []
     for c in range(n_clients):
         seed, cid, rnd = W.philox_ids(w, first_client + c)
-        params.append(B.make_params(d, budget, seed=seed, client_id=cid, round=rnd))
+        params.append(B.make_params(d, budget, seed=seed, client_id=cid, round=rnd, quantizer=QUANTIZERS[args.quantizer]))
     batch = args.batch or n_clients
     groups = [list(range(i, min(i + batch, n_clients))) for i in range(0, n_clients, batch)]
     n_streams = max(1, min(args.streams, len(groups)))
@@ -353,7 +357,7 @@ def run_ours(args):
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         n_s = max(1, min(args.cpu_sample_clients, n_clients))
-        t = oracle_step(w, d, bpc, list(range(n_s)))
+        t = oracle_step(w, d, bpc, list(range(n_s)), QUANTIZERS[args.quantizer])
         cpu_baseline = {"value": 4.0 * d * n_s / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                         "sample": f"{n_s} of {n_clients} clients: plan+encode each, decode-aggregate of those {n_s}; {t:.1f} s"}
 
@@ -361,7 +365,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 data / f64 plan+quantizer / u32 keys", "data": "synthetic",
-        "config": {"workload": f"{w.name} d={d} clients={n_clients} bits_per_coord={bpc} packet=1500B",
+        "config": {"workload": f"{w.name} d={d} clients={n_clients} bits_per_coord={bpc} quantizer={args.quantizer} packet=1500B",
                    "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams, "clients_per_call": batch, "max_candidates": int(max_cand),
                    "multi_gpu": "replicas only: every rank runs its own clients and aggregator"},
         "params_per_s": units / (ms_per_step * 1e-3),

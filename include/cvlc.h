@@ -60,6 +60,19 @@ enum {
 #define CVLC_MAX_CLIENTS_PER_CALL 4096
 #define CVLC_MAX_BATCH 512
 
+/* The two quantizers of the paper's experiments (Section V; Appendix, case study).  Both put uniform
+ * centroids behind a y-bit centroid ID, so a record is s + y bits for either (Eq. (3)).
+ *  PQ    centroids = 2^y points on [min, max] of the packet's values; the header's centroid
+ *        distribution is {min, max} (64 bits); Q = P / (2^y - 1)^2.
+ *  QSGD  quantizes |x| against the l2-norm of the packet's values, which is the header's centroid
+ *        distribution (32 bits, then 32 zero bits).  The paper leaves the place of the sign open:
+ *        here the top bit of the centroid ID is the sign and the other y - 1 bits hold a level
+ *        0..s_q, s_q = 2^(y-1) - 1, value = sign * level * norm / s_q.  Lengths start at y = 2;
+ *        Q = min(P / s_q^2, sqrt(P) / s_q), the paper's min(Q_1, Q_2) at this level count.
+ *        The norm is sqrt(sum of squares added in rank order in double) rounded to fp32. */
+#define CVLC_QUANT_PQ 0u
+#define CVLC_QUANT_QSGD 1u
+
 /* Problem statement of Section IV-C: the update has d coordinates, the client may
  * send budget_bits this round in packets of packet_bits (b) with header_bits (H)
  * of header each; lengths are chosen from 1..max_code_bits (Section IV-B, "Y kinds
@@ -69,7 +82,7 @@ typedef struct cvlc_params {
   uint64_t budget_bits;   /* uplink budget of this client this round; R = floor(budget_bits / packet_bits) */
   uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes) */
   uint32_t header_bits;   /* H; 80 <= H < b; 80 = s (8) + y_r (8) + min,max (64), Fig. 2 */
-  uint32_t quantizer;     /* 0 = PQ (uniform centroids on [min,max]) */
+  uint32_t quantizer;     /* CVLC_QUANT_PQ or CVLC_QUANT_QSGD */
   uint32_t max_code_bits; /* 1..32 */
   double scale_B;         /* B >= 1 of the scaling operation; cvlc_default_scale() in the first round */
   uint64_t seed;          /* Philox4x32-10 key */
@@ -142,9 +155,10 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
 /*
  * Algorithm 1, steps 15-17.  Ranks the coordinates of x_dev by |x| (ties by
  * ascending index), gives packet r the next cap(y_r) ranks, stores the packet's
- * minimum and maximum, quantizes each value stochastically onto the 2^y_r uniform
- * centroids (unbiased; random word = Philox4x32-10 of the coordinate index) and
- * packs (position ID, centroid ID) pairs behind the packet header (Fig. 2).
+ * centroid distribution (PQ: minimum and maximum; QSGD: l2-norm), quantizes each value
+ * stochastically onto the uniform centroids of its y_r-bit code (unbiased; random word
+ * = Philox4x32-10 of the coordinate index) and packs (position ID, centroid ID) pairs
+ * behind the packet header (Fig. 2).
  * stream_dev (16-byte aligned) receives cvlc_stream_bytes(p) bytes.
  * plan_dev must come from cvlc_plan / cvlc_plan_fixed on the same x_dev and params.
  * plan_ws_dev: the workspace that call used, untouched since (it holds per-chunk candidate
@@ -188,7 +202,8 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
 
 /*
  * Parameter-server aggregation (Section III, step 3) fused with decoding: for every
- * record of every client, value = min + CID * (max - min) / (2^y - 1), scaled by
+ * record of every client, value = min + CID * (max - min) / (2^y - 1) (PQ; the QSGD value is
+ * given with CVLC_QUANT_QSGD; every stream names its quantizer in its header), scaled by
  * 1/B_i (Section IV-B, scaling) and by weight_i / weight_total, added into
  * out_dev[PID].  Uniform weights give the paper's 1/|S_t| average.
  *  streams_dev       device array of n_clients device pointers (each 16-byte aligned)

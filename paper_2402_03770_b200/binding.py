@@ -31,6 +31,9 @@ CVLC_ERR_NOT_IMPLEMENTED = 11
 CVLC_ERR_SCALE_TOO_SMALL = 12
 CVLC_ERR_PLAN_MISMATCH = 13
 
+CVLC_QUANT_PQ = 0
+CVLC_QUANT_QSGD = 1
+
 MAX_CODE_BITS = 32
 MAX_BATCH = 512
 HIST_BINS = 4096

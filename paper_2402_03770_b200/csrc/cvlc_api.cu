@@ -19,7 +19,7 @@ bool params_ok(const cvlc_params* p) {
   if (p->d < 2 || p->d > (1ull << 31)) return false;
   if (p->packet_bits == 0 || (p->packet_bits % 32) != 0) return false;
   if (p->header_bits < 80 || p->header_bits >= p->packet_bits) return false;
-  if (p->quantizer != 0) return false;
+  if (p->quantizer != CVLC_QUANT_PQ && p->quantizer != CVLC_QUANT_QSGD) return false;
   if (p->max_code_bits < 1 || p->max_code_bits > CVLC_MAX_CODE_BITS) return false;
   if (!(p->scale_B >= 1.0) || !(p->scale_B < 1e300)) return false;
   return true;
@@ -45,10 +45,18 @@ int derive(const cvlc_params* p, Derived* D) {
   return CVLC_OK;
 }
 
-// PQ error factor Q = P / (2^y - 1)^2 (Appendix, case study) and the coefficient of Eq. (5):
-// g = 1 - (Q / B^2 + (1 - 1/B)^2).  Plain IEEE operations in this order; the host compiler is
-// told not to contract them (-ffp-contract=off).
-double quant_Q(uint32_t cap_y, uint32_t y) {
+// Error factor Q of P = cap(y) values at y bits (Appendix, case study) and the coefficient of Eq. (5):
+// g = 1 - (Q / B^2 + (1 - 1/B)^2).  PQ: Q = P / (2^y - 1)^2.  QSGD: Q = min(P / s_q^2, sqrt(P) / s_q) with
+// the s_q = 2^(y-1) - 1 levels its y-bit code holds beside the sign; one bit holds none.  Plain IEEE
+// operations in this order; the host compiler is told not to contract them (-ffp-contract=off).
+double quant_Q(uint32_t quantizer, uint32_t cap_y, uint32_t y) {
+  if (quantizer == CVLC_QUANT_QSGD) {
+    if (y < 2) return INFINITY;
+    const double sq = (double)((1ull << (y - 1)) - 1ull);
+    const double Q1 = (double)cap_y / (sq * sq);
+    const double Q2 = sqrt((double)cap_y) / sq;
+    return (Q1 < Q2) ? Q1 : Q2;
+  }
   const double L = (double)((1ull << y) - 1ull);
   return (double)cap_y / (L * L);
 }
@@ -76,12 +84,13 @@ int build_shape(const cvlc_params* p, uint32_t fixed_y, Shape* S) {
   for (uint32_t y = 0; y <= CVLC_MAX_CODE_BITS; ++y) S->cap[y] = D.cap[y];
   if (fixed_y) {
     if (fixed_y > p->max_code_bits) return CVLC_ERR_INVALID_ARG;
+    if (p->quantizer == CVLC_QUANT_QSGD && fixed_y < 2) return CVLC_ERR_INVALID_ARG;
     if ((uint64_t)D.R * D.cap[fixed_y] > p->d) return CVLC_ERR_BUDGET_TOO_LARGE;
     return CVLC_OK;
   }
   bool usable = false;
   for (uint32_t y = 1; y <= p->max_code_bits; ++y)
-    if (coeff_g(quant_Q(D.cap[y], y), p->scale_B) > 0.0) usable = true;
+    if (coeff_g(quant_Q(p->quantizer, D.cap[y], y), p->scale_B) > 0.0) usable = true;
   if (!usable) return CVLC_ERR_SCALE_TOO_SMALL;
   // an admissible single-length plan must exist: the longest code sends the fewest coordinates
   if ((uint64_t)D.R * D.cap[p->max_code_bits] > p->d) return CVLC_ERR_BUDGET_TOO_LARGE;
@@ -137,7 +146,7 @@ double cvlc_default_scale(const cvlc_params* p) {
   if (!params_ok(&q)) return NAN;
   const uint32_t s = position_bits(q.d);
   const uint32_t cap8 = (q.packet_bits - q.header_bits) / (s + 8);
-  return 1.0 + quant_Q(cap8, 8);
+  return 1.0 + quant_Q(p->quantizer, cap8, 8);
 }
 
 size_t cvlc_plan_workspace_bytes(const cvlc_params* p) { return cvlc_plan_batch_workspace_bytes(p, 1); }
@@ -231,7 +240,7 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
   if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
   const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
   if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
-  if ((size_t)S.cap[1] * 8 > 200 * 1024) return CVLC_ERR_INVALID_ARG;  // a packet's records are staged in shared memory
+  if ((size_t)S.cap[1] * (S.quantizer == CVLC_QUANT_QSGD ? 16 : 8) > 200 * 1024) return CVLC_ERR_INVALID_ARG;  // a packet's records are staged in shared memory
   if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
   return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
                                                                                                        : CVLC_ERR_CUDA;

@@ -63,14 +63,14 @@ k_decode_prepare(const uint8_t* const* __restrict__ streams, const uint64_t* __r
         const uint64_t sd = (uint64_t)h0.z | ((uint64_t)h0.w << 32);
         const uint32_t sR = h1.x, pb = h1.y, hb = h1.z;
         const double B = __longlong_as_double((long long)((uint64_t)h3.x | ((uint64_t)h3.y << 32)));
-        ok = (magic == CVLC_STREAM_MAGIC) && ((ver_q_s & 0xFFFF) == 1) && (((ver_q_s >> 16) & 0xFF) == 0) &&
+        ok = (magic == CVLC_STREAM_MAGIC) && ((ver_q_s & 0xFFFF) == 1) && (((ver_q_s >> 16) & 0xFF) <= CVLC_QUANT_QSGD) &&
              ((ver_q_s >> 24) == s) && (sd == d) && (pb != 0) && ((pb & 31) == 0) && (hb >= 80) && (hb < pb) &&
              (B >= 1.0) && (B < 1e300);
         if (ok) ok = ((uint64_t)CVLC_STREAM_HEADER_BYTES + (uint64_t)sR * (pb / 8) == nbytes);
         if (ok) {
           R = sR;
           coef[i] = (float)((double)weights[i] / (W * B));
-          meta[2 * i] = pb;
+          meta[2 * i] = pb | ((ver_q_s >> 16) & 0xFF);  // packet bits are a multiple of 32: the quantizer rides below
           meta[2 * i + 1] = hb;
         }
       }
@@ -137,7 +137,7 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
       if (s_prefix[mid] <= g) lo_c = mid; else hi_c = mid;
     }
     const uint32_t c = lo_c, r = g - s_prefix[c];
-    const uint32_t pb = meta[2 * c], H = meta[2 * c + 1];
+    const uint32_t pb = meta[2 * c] & ~31u, quantizer = meta[2 * c] & 31u, H = meta[2 * c + 1];
     const uint32_t n_words = pb >> 5;
     const uint32_t* pkt = reinterpret_cast<const uint32_t*>(streams[c] + CVLC_STREAM_HEADER_BYTES) + (size_t)r * n_words;
     const uint32_t w0 = __ldg(pkt), w1 = __ldg(pkt + 1), w2 = __ldg(pkt + 2);
@@ -152,8 +152,17 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
     const float hi = __uint_as_float((w1 >> 16) | (w2 << 16));
     const uint32_t wd = s + y;
     const uint32_t P = (pb - H) / wd;
-    const double dlo = (double)lo;
-    const double step = (hi == lo) ? 0.0 : __ddiv_rn(__dsub_rn((double)hi, dlo), (double)((1ull << y) - 1ull));
+    const bool qsgd = quantizer == CVLC_QUANT_QSGD;
+    // QSGD: the first centroid field is the packet's l2-norm (finite, not negative); a code is the sign
+    // bit above a level of 2^(y-1) - 1 steps, so one bit is not a code
+    if (qsgd && (y < 2 || __float_as_uint(lo) >= 0x7F800000u)) {
+      if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
+      continue;
+    }
+    const uint32_t level_mask = qsgd ? (uint32_t)((1ull << (y - 1)) - 1ull) : 0u;
+    const double dlo = qsgd ? 0.0 : (double)lo;
+    const double step = qsgd ? __ddiv_rn((double)lo, (double)level_mask)
+                             : ((hi == lo) ? 0.0 : __ddiv_rn(__dsub_rn((double)hi, dlo), (double)((1ull << y) - 1ull)));
     const float cf = coef[c];
     const unsigned long long code_mask = (1ull << y) - 1ull;
     for (uint32_t j = lane; j < P; j += 32) {
@@ -173,7 +182,13 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
         set_status(status, CVLC_ERR_BAD_STREAM);
         continue;
       }
-      const float v = (float)__dadd_rn(dlo, __dmul_rn((double)code, step));
+      float v;
+      if (qsgd) {
+        const float mag = (float)__dmul_rn((double)(code & level_mask), step);
+        v = ((code >> (y - 1)) & 1u) ? -mag : mag;
+      } else {
+        v = (float)__dadd_rn(dlo, __dmul_rn((double)code, step));
+      }
       atomicAdd(out + pid, cf * v);
     }
   }

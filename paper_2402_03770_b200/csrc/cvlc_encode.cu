@@ -91,7 +91,8 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
     if (plan->status != CVLC_OK)
       bad = plan->status;
     else if (plan->s != shape.s || plan->R != shape.R || nsum != shape.R || k != plan->k || k == 0 ||
-             k > plan->n_candidates || plan->n_candidates > shape.d || plan->thresh_bin >= CVLC_HIST_BINS)
+             k > plan->n_candidates || plan->n_candidates > shape.d || plan->thresh_bin >= CVLC_HIST_BINS ||
+             (shape.quantizer == CVLC_QUANT_QSGD && plan->n_y[1] != 0))  // a one-bit QSGD code holds no level
       bad = CVLC_ERR_PLAN_MISMATCH;
     else if (plan->n_candidates > L.capacity)
       bad = CVLC_ERR_WORKSPACE_TOO_SMALL;
@@ -763,17 +764,17 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 }
 
 // ===================================================================================
-// K5  per-packet min/max, PQ stochastic quantization, bit packing
+// K5  per-packet centroid distribution (PQ: min/max; QSGD: l2-norm), stochastic quantization, bit packing
 // ===================================================================================
 // One CTA per (packet, client).  Packet r (longest codes first) holds ranks [Z, Z + cap(y_r)).
 
 constexpr int kPackThreads = 128;
 
-template <int CAP>
+template <int CAP, bool QSGD>
 __global__ void __launch_bounds__(kPackThreads)
 k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
        const __grid_constant__ EncLayout L) {
-  extern __shared__ unsigned long long recs[];  // [cap(1)]
+  extern __shared__ unsigned long long recs[];  // [cap(1)], QSGD: then cap(1) squares
   __shared__ float s_red[2][kPackThreads / 32];
   __shared__ uint32_t s_y;
   __shared__ unsigned long long s_Z;
@@ -818,8 +819,74 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   const unsigned long long Z = s_Z;
   const uint32_t P = plan->cap[y];
   const uint32_t wd = s + y;
+  float lo, hi;  // the header's two centroid fields
 
-  // minimum / maximum of the packet's signed values (the centroid distribution of PQ)
+  if constexpr (QSGD) {
+    // ---- QSGD: |x| against the packet's l2-norm; code = sign bit above a level of s_q = 2^(y-1) - 1 steps ----
+    __shared__ float s_norm;
+    double* sqv = reinterpret_cast<double*>(recs + shape.cap[1]);
+    for (uint32_t j = tid; j < P; j += kPackThreads) {
+      const unsigned long long pair = sorted[Z + j];
+      recs[j] = pair;
+      const double a = (double)__uint_as_float((uint32_t)(pair >> 32));
+      sqv[j] = __dmul_rn(a, a);  // exact: 24 x 24 bits
+    }
+    __syncthreads();
+    // the norm is defined with the squares added in rank order in double: one thread walks the chain
+    if (tid == 0) {
+      double sum = 0.0;
+      uint32_t j = 0;
+      for (; j + 8 <= P; j += 8) {
+        double v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = sqv[j + u];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum = __dadd_rn(sum, v[u]);
+      }
+      for (; j < P; ++j) sum = __dadd_rn(sum, sqv[j]);
+      const double rt = __dsqrt_rn(sum);
+      s_norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
+    }
+    __syncthreads();
+    const float norm = s_norm;
+    lo = norm;
+    hi = 0.0f;
+    const uint32_t sq = (uint32_t)((1ull << (y - 1)) - 1ull);  // y >= 2: checked with the plan
+    const double sqd = (double)sq;
+    const double dn = (double)norm;
+    const double scale = (norm > 0.0f) ? __ddiv_rn(sqd, dn) : 0.0;
+    for (uint32_t j = tid; j < P; j += kPackThreads) {
+      const unsigned long long pair = recs[j];
+      const uint32_t key = (uint32_t)(pair >> 32);
+      const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
+      const uint32_t sign = key ? (((uint32_t)pair >> 31) & 1u) : 0u;  // -0 is stored as +0
+      uint32_t level = 0;
+      if (norm > 0.0f) {
+        const double a = (double)__uint_as_float(key);
+        const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+        // t = (a / norm) * s_q decides floor(t) and [u < frac(t)]; a * (s_q / norm) is within a few ulp of it
+        // and decides the same unless its fraction sits that close to 0, 1 or u
+        const double tf = __dmul_rn(a, scale);
+        const double jf = floor(tf);
+        const double ff = __dsub_rn(tf, jf);
+        const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
+        if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < sqd) {
+          level = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
+        } else {
+          const double t = __dmul_rn(__ddiv_rn(a, dn), sqd);
+          double j0 = floor(t);
+          if (j0 > sqd) j0 = sqd;
+          const double frac = __dsub_rn(t, j0);
+          level = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
+          if (level > sq) level = sq;
+        }
+      }
+      const uint32_t code = (sign << (y - 1)) | level;
+      recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
+    }
+    __syncthreads();
+  } else {
+  // ---- PQ: minimum / maximum of the packet's signed values (its centroid distribution) ----
   float vmin = CUDART_INF_F, vmax = -CUDART_INF_F;
   for (uint32_t j = tid; j < P; j += kPackThreads) {
     const unsigned long long pair = sorted[Z + j];
@@ -840,7 +907,8 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     s_red[1][warp] = vmax;
   }
   __syncthreads();
-  float lo = s_red[0][0], hi = s_red[1][0];
+  lo = s_red[0][0];
+  hi = s_red[1][0];
 #pragma unroll
   for (int w = 1; w < kPackThreads / 32; ++w) {
     lo = fminf(lo, s_red[0][w]);
@@ -881,6 +949,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
   }
   __syncthreads();
+  }  // PQ
 
   // gather the packet's 32-bit words: header {s, y, lo, hi}, then records of wd bits from bit H
   const uint32_t H = shape.header_bits;
@@ -946,7 +1015,9 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-    e = cudaFuncSetAttribute(k_pack<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = cudaFuncSetAttribute(k_pack<CAP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_pack<CAP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_select<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSelStages * kSelStageBytes));
     if (e != cudaSuccess) return e;
@@ -960,7 +1031,8 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
   const EncLayout L = enc_layout(shape.d, n, capacity);
   unsigned char* w = static_cast<unsigned char*>(ws);
-  const size_t pack_smem = (size_t)shape.cap[1] * 8;
+  const bool qsgd = shape.quantizer == CVLC_QUANT_QSGD;
+  const size_t pack_smem = (size_t)shape.cap[1] * (qsgd ? 16 : 8);  // records; QSGD: and their squares
 
   const Partition part = make_partition(shape.d, n);
   const unsigned char* pws = static_cast<const unsigned char*>(plan_ws);
@@ -995,7 +1067,10 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   }
   {
     LaunchScope ls(kKPack, st);
-    k_pack<CAP><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+    if (qsgd)
+      k_pack<CAP, true><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+    else
+      k_pack<CAP, false><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
   }
   return cudaGetLastError();
 }

@@ -233,8 +233,17 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     const double B = batch.c[blockIdx.x].scale_B;
     const bool in_range = y <= shape.max_code_bits;
     const uint32_t cap_y = in_range ? shape.cap[y] : 0u;
-    const double L = (double)((1ull << y) - 1ull);
-    const double Q = __ddiv_rn((double)cap_y, __dmul_rn(L, L));
+    double Q;  // error factor of cap(y) values at y bits (Appendix, case study)
+    if (shape.quantizer == CVLC_QUANT_QSGD) {
+      // min(P / s_q^2, sqrt(P) / s_q), s_q = 2^(y-1) - 1 levels beside the sign bit; one bit holds no level
+      const double sq = (double)((1ull << (y - 1)) - 1ull);
+      const double Q1 = __ddiv_rn((double)cap_y, __dmul_rn(sq, sq));
+      const double Q2 = __ddiv_rn(__dsqrt_rn((double)cap_y), sq);
+      Q = (y < 2) ? CUDART_INF : ((Q1 < Q2) ? Q1 : Q2);
+    } else {
+      const double L = (double)((1ull << y) - 1ull);  // PQ: P / (2^y - 1)^2
+      Q = __ddiv_rn((double)cap_y, __dmul_rn(L, L));
+    }
     const double one_m = __dsub_rn(1.0, __ddiv_rn(1.0, B));
     const double g = __dsub_rn(1.0, __dadd_rn(__ddiv_rn(Q, __dmul_rn(B, B)), __dmul_rn(one_m, one_m)));
     unsigned member;

@@ -48,20 +48,20 @@ def oracle_plan_encode(x: np.ndarray, pd: dict, fixed_y: int = 0):
 
 
 def _worker_encode(args):
-    workload_name, client, d, bpc, fixed_y = args
+    workload_name, client, d, bpc, fixed_y, quantizer = args
     from paper_2402_03770_b200 import workloads as W
     w = W.WORKLOADS[workload_name]
     x = W.client_update(w, client, d=d)
     seed, cid, rnd = W.philox_ids(w, client)
-    pd = params_dict(x.size, int(np.floor(bpc * x.size)), seed=seed, client_id=cid, round=rnd)
+    pd = params_dict(x.size, int(np.floor(bpc * x.size)), seed=seed, client_id=cid, round=rnd, quantizer=quantizer)
     fields, st = oracle_plan_encode(x, pd, fixed_y)
     return client, fields, st
 
 
 def oracle_encode_clients(workload_name: str, clients: Sequence[int], d: Optional[int], bpc: float,
-                          fixed_y: int = 0, procs: Optional[int] = None):
+                          fixed_y: int = 0, procs: Optional[int] = None, quantizer: int = 0):
     """Oracle plan+encode of several clients of a workload, in spawned worker processes."""
-    jobs = [(workload_name, c, d, bpc, fixed_y) for c in clients]
+    jobs = [(workload_name, c, d, bpc, fixed_y, quantizer) for c in clients]
     procs = procs or min(len(jobs), max(1, (os.cpu_count() or 2) - 1), 32)
     if procs <= 1 or len(jobs) == 1:
         return [_worker_encode(j) for j in jobs]

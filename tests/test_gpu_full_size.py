@@ -11,14 +11,15 @@ from gpu_util import assert_aggregate_close, assert_plan_equal, gpu_params, orac
 pytestmark = pytest.mark.gpu
 
 
-def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, keep_on_device=False):
+def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, quantizer=0):
     w = W.WORKLOADS[workload]
     dev = torch.device("cuda:0")
     params, xs = [], []
     for c in clients:
         x = W.client_update(w, c, d=d)
         seed, cid, rnd = W.philox_ids(w, c)
-        params.append(gpu_params(params_dict(x.size, int(np.floor(bpc * x.size)), seed=seed, client_id=cid, round=rnd)))
+        params.append(gpu_params(params_dict(x.size, int(np.floor(bpc * x.size)), seed=seed, client_id=cid, round=rnd,
+                                             quantizer=quantizer)))
         xs.append(torch.from_numpy(x).to(dev))
     enc = B.BatchEncoder(params, dev, max_candidates=max_candidates)
     outs = enc.run(xs)
@@ -99,6 +100,18 @@ def test_resnet18_all_100_clients_as_benchmarked(env):
     enc, outs = gpu_batch_encode("resnet18", clients, None, 2.0, max_cand, torch, B)
     check_against_oracle(enc, outs, ref)
     decode_both(outs, [r[2] for r in ref], W.client_weights(w), w.d, torch, B)
+
+
+def test_resnet18_qsgd_three_clients(env):
+    """the second quantizer of the paper's experiments at the benchmark's size and budget"""
+    torch, B = env
+    w = W.WORKLOADS["resnet18"]
+    clients = [0, 31, 99]
+    ref = oracle_encode_clients("resnet18", clients, None, 2.0, quantizer=1)
+    enc, outs = gpu_batch_encode("resnet18", clients, None, 2.0, 0, torch, B, quantizer=1)
+    check_against_oracle(enc, outs, ref)
+    assert enc.read_plan(0).n_y[1] == 0
+    decode_both(outs, [r[2] for r in ref], W.client_weights(w)[clients], w.d, torch, B)
 
 
 def test_resnet50_ties_and_zero_blocks(env):

@@ -95,6 +95,10 @@ def lib() -> C.CDLL:
         L.cvlc_plan_from_alpha_oracle.argtypes = [P(OrcParams), f64, P(OrcPlan)]
         L.cvlc_plan_oracle.restype = C.c_int
         L.cvlc_plan_oracle.argtypes = [C.c_void_p, P(OrcParams), P(OrcPlan)]
+        L.cvlc_plan_from_histogram_oracle.restype = C.c_int
+        L.cvlc_plan_from_histogram_oracle.argtypes = [C.c_void_p, P(OrcParams), P(OrcPlan)]
+        L.cvlc_decode_apply_oracle.restype = C.c_int
+        L.cvlc_decode_apply_oracle.argtypes = [P(C.c_void_p), P(u64), C.c_void_p, u32, f64, u64, C.c_void_p]
         L.cvlc_plan_fixed_oracle.restype = C.c_int
         L.cvlc_plan_fixed_oracle.argtypes = [P(OrcParams), u32, P(OrcPlan)]
         L.cvlc_rank_oracle.restype = C.c_int
@@ -213,6 +217,16 @@ def plan_from_alpha(p: OrcParams, alpha_q: float) -> OrcPlan:
     return plan
 
 
+def plan_from_histogram(h: np.ndarray, p: OrcParams) -> OrcPlan:
+    h = np.ascontiguousarray(h, dtype=np.uint64)
+    assert h.size == HIST_BINS
+    pl = OrcPlan()
+    rc = lib().cvlc_plan_from_histogram_oracle(h.ctypes.data, C.byref(p), C.byref(pl))
+    if rc != ORC_OK:
+        raise OracleError(rc, "plan_from_histogram")
+    return pl
+
+
 def plan(x: np.ndarray, p: OrcParams) -> OrcPlan:
     x = _f32(x)
     assert x.size == p.d
@@ -293,3 +307,19 @@ def decode_aggregate(streams: Sequence[np.ndarray], weights: np.ndarray, d: int,
     if rc != ORC_OK:
         raise OracleError(rc, "decode_aggregate")
     return out
+
+
+def decode_apply(streams: Sequence[np.ndarray], weights: np.ndarray, model: np.ndarray, *,
+                 weight_total: float = 0.0) -> np.ndarray:
+    """model <- model - aggregate, in place; returns model"""
+    n = len(streams)
+    streams = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    ptrs = (C.c_void_p * n)(*[s.ctypes.data for s in streams])
+    sizes = (C.c_uint64 * n)(*[s.size for s in streams])
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    assert w.size == n and model.dtype == np.float32 and model.flags.c_contiguous
+    rc = lib().cvlc_decode_apply_oracle(ptrs, sizes, w.ctypes.data, n, float(weight_total), model.size,
+                                        model.ctypes.data)
+    if rc != ORC_OK:
+        raise OracleError(rc, "decode_apply")
+    return model

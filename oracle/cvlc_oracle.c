@@ -430,16 +430,30 @@ int cvlc_plan_from_alpha_oracle(const orc_params* p, double alpha_q, orc_plan* p
   return ORC_OK;
 }
 
+/* Section IV-C, last paragraph: a client may send the distribution of its update to the
+ * parameter server, which solves the problem and returns k and the P_r.  The distribution
+ * is the 4096-bin histogram of |x|: Algorithm 1 uses the update only through alpha. */
+int cvlc_plan_from_histogram_oracle(const uint64_t h[ORC_HIST_BINS], const orc_params* p, orc_plan* plan) {
+  if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
+  uint64_t total = 0;
+  for (int j = 0; j < ORC_HIST_BINS; ++j) total += h[j];
+  if (total != p->d) return ORC_ERR_INVALID_ARG;
+  /* bins of exponent 255: Inf and NaN */
+  for (int j = (int)(0x7F800000u >> 19); j < ORC_HIST_BINS; ++j)
+    if (h[j] != 0) return ORC_ERR_NONFINITE_INPUT;
+  double alpha, alpha_q;
+  cvlc_alpha_fit_oracle(h, p->d, &alpha, &alpha_q);
+  int rc = cvlc_plan_from_alpha_oracle(p, alpha_q, plan);
+  if (rc == ORC_OK) plan->alpha = alpha;
+  return rc;
+}
+
 int cvlc_plan_oracle(const float* x, const orc_params* p, orc_plan* plan) {
   if (!params_ok(p)) return ORC_ERR_INVALID_ARG;
   static uint64_t h[ORC_HIST_BINS];
   int rc = cvlc_histogram_oracle(x, p->d, h);
   if (rc != ORC_OK) return rc;
-  double alpha, alpha_q;
-  cvlc_alpha_fit_oracle(h, p->d, &alpha, &alpha_q);
-  rc = cvlc_plan_from_alpha_oracle(p, alpha_q, plan);
-  if (rc == ORC_OK) plan->alpha = alpha;
-  return rc;
+  return cvlc_plan_from_histogram_oracle(h, p, plan);
 }
 
 /* Degenerate plan: every packet at one length y ("Top_k plus y-bit quantization",
@@ -781,5 +795,18 @@ int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* 
     }
   }
   free(acc);
+  return rc;
+}
+
+/* Section III, step 3: w_{t+1} = w_t - (weighted mean of the decoded updates), in fp32 */
+int cvlc_decode_apply_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
+                             const float* weights, uint32_t n_clients, double weight_total,
+                             uint64_t d, float* model) {
+  float* agg = (float*)malloc(sizeof(float) * (size_t)d);
+  if (!agg) return ORC_ERR_INVALID_ARG;
+  int rc = cvlc_decode_aggregate_oracle(streams, stream_bytes, weights, n_clients, weight_total, d, agg, 0);
+  if (rc == ORC_OK)
+    for (uint64_t i = 0; i < d; ++i) model[i] = model[i] - agg[i];
+  free(agg);
   return rc;
 }

@@ -95,6 +95,8 @@ double cvlc_objective_oracle(const orc_params* p, double beta, const uint32_t n_
 int cvlc_candidates_oracle(const orc_params* p, uint32_t Y[ORC_MAX_Y + 1]);
 int cvlc_plan_from_alpha_oracle(const orc_params* p, double alpha, orc_plan* plan);
 int cvlc_plan_oracle(const float* x, const orc_params* p, orc_plan* plan);
+/* planning at the parameter server from a client's histogram (Section IV-C, last paragraph) */
+int cvlc_plan_from_histogram_oracle(const uint64_t h[ORC_HIST_BINS], const orc_params* p, orc_plan* plan);
 int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan);
 
 /* --- encoding ------------------------------------------------------------ */
@@ -113,6 +115,10 @@ int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan
 int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
                                  const float* weights, uint32_t n_clients, double weight_total,
                                  uint64_t d, float* out, int accumulate);
+/* model <- model - aggregate (Section III, step 3) */
+int cvlc_decode_apply_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
+                             const float* weights, uint32_t n_clients, double weight_total,
+                             uint64_t d, float* model);
 
 #ifdef __cplusplus
 }

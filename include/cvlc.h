@@ -153,6 +153,29 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
                     void* ws_dev, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Planning at the parameter server (Section IV-C, last paragraph: a client with limited capacity
+ * sends the distribution of its update, the server solves the problem and returns k and the P_r).
+ * The distribution is the 4096-bin histogram of |x| that cvlc_plan itself works from
+ * (bin = (bits(x) & 0x7FFFFFFF) >> 19): Algorithm 1 uses the update only through alpha.
+ *
+ * cvlc_histogram_batch: hist_dev receives n * 4096 uint64 counts, client after client; x_dev and
+ * params as in cvlc_plan_batch (only d is used; all clients share it).  The workspace is sized by
+ * cvlc_plan_batch_workspace_bytes and is NOT a plan workspace afterwards.
+ *
+ * cvlc_plan_from_histogram_batch: hist_dev holds n * 4096 uint64 counts (device memory, 8-byte
+ * aligned); plans_dev receives the same plans cvlc_plan_batch makes from the updates themselves.
+ * Such a plan comes without the per-chunk candidate counts: the client encodes with
+ * plan_ws_dev = NULL (passing this call's workspace there is refused with PLAN_MISMATCH).
+ * Errors: as cvlc_plan_batch (host); device-detected, in the plan's status word and at byte 0 of
+ * ws_dev: INVALID_ARG when a histogram's counts do not add up to d, NONFINITE_INPUT when a bin of
+ * exponent 255 is not empty.
+ */
+int cvlc_histogram_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint64_t* hist_dev,
+                         void* ws_dev, size_t ws_bytes, void* cuda_stream);
+int cvlc_plan_from_histogram_batch(const uint64_t* hist_dev, const cvlc_params* params, uint32_t n,
+                                   cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Algorithm 1, steps 15-17.  Ranks the coordinates of x_dev by |x| (ties by
  * ascending index), gives packet r the next cap(y_r) ranks, stores the packet's
  * centroid distribution (PQ: minimum and maximum; QSGD: l2-norm), quantizes each value
@@ -245,6 +268,18 @@ int cvlc_decode_aggregate_noalloc(const uint8_t* const* streams_dev, const uint6
                                   const float* weights_dev, uint32_t n_clients, double weight_total,
                                   uint64_t d, float* out_dev, int accumulate, int32_t* status_dev,
                                   void* cuda_stream);
+
+/*
+ * The parameter server's model step (Section III, step 3): w_{t+1} = w_t - aggregate.
+ * cvlc_decode_aggregate into aggregate_dev (d fp32, overwritten; kept for the caller), then
+ * model_dev[i] -= aggregate_dev[i] in fp32.  Two kernels rather than atomics straight into the
+ * model: adding a hundred small terms one by one to a large weight would round a hundred times.
+ * After a device-detected decode error the model is left untouched.  Other arguments and errors
+ * as cvlc_decode_aggregate; model_dev 16-byte aligned and distinct from aggregate_dev.
+ */
+int cvlc_decode_apply(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev, const float* weights_dev,
+                      uint32_t n_clients, double weight_total, uint64_t d, float* model_dev, float* aggregate_dev,
+                      void* ws_dev, size_t ws_bytes, void* cuda_stream);
 
 /* Waits for cuda_stream and returns the status word at byte 0 of a plan or workspace. */
 int cvlc_read_status(const void* plan_or_ws_dev, void* cuda_stream);

@@ -45,7 +45,7 @@ EXPORTS = [
     "cvlc_plan_workspace_bytes", "cvlc_encode_workspace_bytes", "cvlc_decode_workspace_bytes",
     "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_plan_batch_workspace_bytes",
     "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
-    "cvlc_selftest_philox", "cvlc_selftest_math",
+    "cvlc_selftest_philox", "cvlc_selftest_math", "cvlc_histogram_batch", "cvlc_plan_from_histogram_batch", "cvlc_decode_apply",
     "cvlc_decode_aggregate_noalloc", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
@@ -127,6 +127,12 @@ def lib() -> C.CDLL:
     L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
     L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
+    L.cvlc_histogram_batch.restype = C.c_int
+    L.cvlc_histogram_batch.argtypes = [vp, PP, u32, vp, vp, sz, vp]
+    L.cvlc_plan_from_histogram_batch.restype = C.c_int
+    L.cvlc_plan_from_histogram_batch.argtypes = [vp, PP, u32, vp, vp, sz, vp]
+    L.cvlc_decode_apply.restype = C.c_int
+    L.cvlc_decode_apply.argtypes = [vp, vp, vp, u32, f64, u64, vp, vp, vp, sz, vp]
     L.cvlc_decode_aggregate_noalloc.restype = C.c_int
     L.cvlc_decode_aggregate_noalloc.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, vp]
     L.cvlc_read_status.restype = C.c_int
@@ -281,6 +287,36 @@ def cvlc_decode_aggregate(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor,
            "cvlc_decode_aggregate")
 
 
+def cvlc_histogram_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], hist: torch.Tensor, ws: torch.Tensor,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+    """hist: device int64/uint64 tensor of n * HIST_BINS counts (what a client sends when the server plans)."""
+    n = len(xs)
+    assert len(params) == n and hist.element_size() == 8 and hist.numel() >= n * HIST_BINS
+    _check(lib().cvlc_histogram_batch(_ptr_array(xs), _params_array(params), n, _ptr(hist), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_histogram_batch")
+
+
+def cvlc_plan_from_histogram_batch(hist: torch.Tensor, params: Sequence[CvlcParams], plans: torch.Tensor,
+                                   ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    n = len(params)
+    assert hist.element_size() == 8 and hist.numel() >= n * HIST_BINS
+    assert plans.dtype == torch.uint8 and plans.numel() >= n * PLAN_BYTES
+    _check(lib().cvlc_plan_from_histogram_batch(_ptr(hist), _params_array(params), n, _ptr(plans), _ptr(ws),
+                                                ws.numel() * ws.element_size(), _stream_handle(stream)),
+           "cvlc_plan_from_histogram_batch")
+
+
+def cvlc_decode_apply(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor, n_clients: int,
+                      weight_total: float, d: int, model: torch.Tensor, aggregate: torch.Tensor, ws: torch.Tensor,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+    """model <- model - aggregate of the decoded streams; `aggregate` (d fp32) receives the aggregate."""
+    assert model.dtype == torch.float32 and model.numel() == d
+    assert aggregate.dtype == torch.float32 and aggregate.numel() == d
+    _check(lib().cvlc_decode_apply(_ptr(stream_ptrs), _ptr(stream_bytes), _ptr(weights), int(n_clients),
+                                   float(weight_total), int(d), _ptr(model), _ptr(aggregate), _ptr(ws),
+                                   ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_decode_apply")
+
+
 NOALLOC_MAX_CLIENTS = 256
 
 
@@ -332,7 +368,7 @@ def cvlc_profile_reset() -> None:
 
 
 KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan", "k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
-                "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero", "k_decode"]
+                "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero", "k_decode", "k_hist_check", "k_apply"]
 
 
 def cvlc_profile_read(kernel_name: str = "*"):
@@ -438,6 +474,11 @@ class Aggregator:
         cvlc_decode_aggregate(self.ptrs, self.sizes, self.weights, n, weight_total, self.d, out, accumulate,
                               self.ws, stream)
         return out
+
+    def apply(self, n: int, model: torch.Tensor, aggregate: torch.Tensor, *, weight_total: float = 0.0,
+              stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        cvlc_decode_apply(self.ptrs, self.sizes, self.weights, n, weight_total, self.d, model, aggregate, self.ws, stream)
+        return model
 
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         return cvlc_read_status(self.ws, stream)

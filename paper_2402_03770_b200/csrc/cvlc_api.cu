@@ -193,6 +193,51 @@ int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32
   return launch_plan(desc, n, S, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
+int cvlc_histogram_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint64_t* hist_dev,
+                         void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!x_dev || !params || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  for (uint32_t i = 0; i < n; ++i) {
+    Derived D;
+    const int rc = derive(&params[i], &D);
+    if (rc != CVLC_OK) return rc;
+    if (params[i].d != params[0].d) return CVLC_ERR_INVALID_ARG;
+    if (!aligned(x_dev[i], 16)) return CVLC_ERR_INVALID_ARG;
+    memset(&desc[i], 0, sizeof desc[i]);
+    desc[i].x = x_dev[i];
+  }
+  memset(&S, 0, sizeof S);
+  S.d = params[0].d;
+  if (!aligned(hist_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  return launch_histogram(desc, n, S, ws_dev, reinterpret_cast<unsigned long long*>(hist_dev),
+                          static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+}
+
+int cvlc_plan_from_histogram_batch(const uint64_t* hist_dev, const cvlc_params* params, uint32_t n,
+                                   cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!hist_dev || !params || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  for (uint32_t i = 0; i < n; ++i) {
+    Shape Si;
+    const int rc = build_shape(&params[i], 0, i == 0 ? &S : &Si);
+    if (rc != CVLC_OK) return rc;
+    if (i && !same_shape(params[0], params[i])) return CVLC_ERR_INVALID_ARG;
+    memset(&desc[i], 0, sizeof desc[i]);
+    desc[i].plan = plans_dev + i;
+    desc[i].seed = params[i].seed;
+    desc[i].scale_B = params[i].scale_B;
+    desc[i].client_id = params[i].client_id;
+    desc[i].round = params[i].round;
+  }
+  if (!aligned(hist_dev, 8) || !aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  return launch_plan_from_hist(desc, n, S, reinterpret_cast<const unsigned long long*>(hist_dev), ws_dev,
+                               static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+}
+
 int cvlc_plan(const float* x_dev, const cvlc_params* p, cvlc_plan_t* plan_dev, void* ws_dev, size_t ws_bytes,
               void* cuda_stream) {
   return cvlc_plan_batch(&x_dev, p, 1, 0, plan_dev, ws_dev, ws_bytes, cuda_stream);
@@ -264,6 +309,18 @@ int cvlc_decode_aggregate(const uint8_t* const* streams_dev, const uint64_t* str
   if (ws_bytes < dec_ws_bytes(n_clients)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   return launch_decode(streams_dev, stream_bytes_dev, weights_dev, n_clients, weight_total, d, position_bits(d), out_dev,
                        accumulate ? 1 : 0, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
+}
+
+int cvlc_decode_apply(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev, const float* weights_dev,
+                      uint32_t n_clients, double weight_total, uint64_t d, float* model_dev, float* aggregate_dev,
+                      void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (!aligned(model_dev, 16) || model_dev == aggregate_dev) return CVLC_ERR_INVALID_ARG;
+  const int rc = cvlc_decode_aggregate(streams_dev, stream_bytes_dev, weights_dev, n_clients, weight_total, d,
+                                       aggregate_dev, 0, ws_dev, ws_bytes, cuda_stream);
+  if (rc != CVLC_OK) return rc;
+  return launch_apply(model_dev, aggregate_dev, d, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
              ? CVLC_OK
              : CVLC_ERR_CUDA;
 }

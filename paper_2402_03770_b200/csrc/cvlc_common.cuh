@@ -181,7 +181,7 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 
 enum KernelId {
   kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan, kKSortPass, kKPack,
-  kKDecodePrepare, kKFillZero, kKDecode, kKSelftest, kNumKernelIds
+  kKDecodePrepare, kKFillZero, kKDecode, kKSelftest, kKHistCheck, kKApply, kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -199,6 +199,11 @@ struct LaunchScope {
 // ---- launchers (one per translation unit) ---------------------------------------
 
 cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
+cudaError_t launch_histogram(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
+                             unsigned long long* hist_out, cudaStream_t st);
+cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const Shape& shape,
+                                  const unsigned long long* hist, void* ws, cudaStream_t st);
+cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st);
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
                           const void* plan_ws, void* ws, cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,

@@ -210,6 +210,37 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
   return cudaGetLastError();
 }
 
+// K8  model <- model - aggregate (Section III, step 3); nothing is touched after a decode error
+__global__ void __launch_bounds__(256)
+k_apply(float* __restrict__ model, const float* __restrict__ agg, uint64_t d, const unsigned char* dec_ws) {
+  if (*reinterpret_cast<const int32_t*>(dec_ws + kDecWsStatus) != 0) return;
+  const uint64_t nvec = d >> 2;
+  float4* mv = reinterpret_cast<float4*>(model);
+  const float4* av = reinterpret_cast<const float4*>(agg);
+  for (uint64_t v = (uint64_t)blockIdx.x * 256 + threadIdx.x; v < nvec; v += (uint64_t)gridDim.x * 256) {
+    float4 m = mv[v];
+    const float4 a = av[v];
+    m.x = __fsub_rn(m.x, a.x);
+    m.y = __fsub_rn(m.y, a.y);
+    m.z = __fsub_rn(m.z, a.z);
+    m.w = __fsub_rn(m.w, a.w);
+    mv[v] = m;
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
+    const uint64_t i = (nvec << 2) + threadIdx.x;
+    model[i] = __fsub_rn(model[i], agg[i]);
+  }
+}
+
+cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st) {
+  const uint64_t nvec = d >> 2;
+  const uint64_t want = (nvec + 255) / 256;
+  const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? (want ? want : 1) : 8 * kNumSM);
+  LaunchScope ls(kKApply, st);
+  k_apply<<<grid, 256, 0, st>>>(model, agg, d, static_cast<const unsigned char*>(dec_ws));
+  return cudaGetLastError();
+}
+
 }  // namespace cvlc
 
 // ===================================================================================

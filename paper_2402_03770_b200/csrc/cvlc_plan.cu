@@ -210,7 +210,7 @@ template <int CAP>
 __global__ void __launch_bounds__(kPlanThreads, 1)
 k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restrict__ nonfinite_all,
        const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
-       const __grid_constant__ Partition part, unsigned char* ws) {
+       const __grid_constant__ Partition part, unsigned char* ws, int have_segments) {
   extern __shared__ unsigned char smem_raw[];
   unsigned long long* Nsuf = reinterpret_cast<unsigned long long*>(smem_raw);  // [4096] survival counts
   double* ptX = reinterpret_cast<double*>(smem_raw + 4096 * 8);                // fit points, ascending bin
@@ -226,6 +226,14 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
   cvlc_plan_t* __restrict__ plan = batch.c[blockIdx.x].plan;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (*nonfinite & 2u) {  // a histogram from outside whose counts do not add up to d
+    if (tid == 0) {
+      plan->status = CVLC_ERR_INVALID_ARG;
+      set_status(ws_status, CVLC_ERR_INVALID_ARG);
+    }
+    return;
+  }
 
   // ---- candidate lengths: g(y) > 0 (the paper's B > (Q+1)/2) and not dominated --------
   if (warp == 0) {
@@ -741,8 +749,9 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
   __syncthreads();
 
   // candidates per segment of this client (segment = part of the client inside one block's chunk of
-  // the histogram / selection kernels) and their exclusive prefix: the selection kernel's offsets
-  {
+  // the histogram / selection kernels) and their exclusive prefix: the selection kernel's offsets.
+  // A plan made from a histogram alone has no segments; its workspace header stays unmarked.
+  if (have_segments) {
     const uint32_t c = blockIdx.x;
     const uint32_t S = part.max_segments;
     uint32_t* seg_count = reinterpret_cast<uint32_t*>(ws + plan_off_seg_count(batch.n));
@@ -782,7 +791,8 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
 // ===================================================================================
 
 template <int CAP>
-static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
+static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
+                                 unsigned long long* hist_out, cudaStream_t st) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -814,16 +824,97 @@ static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Sh
     LaunchScope ls(kKHist, st);
     k_hist<CAP><<<part.grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, part, hist, flags, seg_hist);
   }
+  if (hist_out) {
+    // the histograms alone: what a client sends when the parameter server plans for it.  The workspace
+    // header stays unmarked, so an encode call cannot take it for one that holds a plan's segment tables.
+    const cudaError_t e2 = cudaGetLastError();
+    if (e2 != cudaSuccess) return e2;
+    return cudaMemcpyAsync(hist_out, hist, (size_t)n * CVLC_HIST_BINS * 8, cudaMemcpyDeviceToDevice, st);
+  }
   {
     LaunchScope ls(kKPlan, st);
-    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w);
+    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w, 1);
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
-  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, st);
-  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, st);
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, nullptr, st);
+  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, nullptr, st);
+}
+
+cudaError_t launch_histogram(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
+                             unsigned long long* hist_out, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, hist_out, st);
+  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, hist_out, st);
+}
+
+// Checks histograms that come from outside: flag bit 0 = a value of exponent 255 (Inf, NaN),
+// bit 1 = the counts do not add up to d.
+__global__ void __launch_bounds__(256)
+k_hist_check(const unsigned long long* __restrict__ hist_all, uint64_t d, uint32_t* __restrict__ flags) {
+  __shared__ unsigned long long s_sum[8];
+  __shared__ uint32_t s_nonfinite;
+  const unsigned long long* hist = hist_all + (size_t)blockIdx.x * CVLC_HIST_BINS;
+  if (threadIdx.x == 0) s_nonfinite = 0;
+  __syncthreads();
+  unsigned long long sum = 0;
+  for (int j = threadIdx.x; j < CVLC_HIST_BINS; j += 256) {
+    const unsigned long long h = hist[j];
+    sum += h;
+    if (j >= (int)(0x7F800000u >> 19) && h != 0) s_nonfinite = 1u;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+  if ((threadIdx.x & 31) == 0) s_sum[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long tot = 0;
+    for (int w = 0; w < 8; ++w) tot += s_sum[w];
+    flags[blockIdx.x] = s_nonfinite | ((tot != d) ? 2u : 0u);
+  }
+}
+
+template <int CAP>
+static cudaError_t launch_plan_from_hist_t(const ClientDesc* clients, uint32_t n, const Shape& shape,
+                                           const unsigned long long* hist, void* ws, cudaStream_t st) {
+  static bool attr_done[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+    e = cudaFuncSetAttribute(k_plan<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
+    if (e != cudaSuccess) return e;
+    attr_done[dev] = true;
+  }
+  BatchDesc<CAP> batch;
+  batch.n = n;
+  batch.pad = 0;
+  for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
+  unsigned char* w = static_cast<unsigned char*>(ws);
+  uint32_t* flags = reinterpret_cast<uint32_t*>(w + plan_off_flags(n));
+  const Partition part = make_partition(shape.d, n);
+  {
+    // status word and header start at zero: the header stays unmarked, so an encode call cannot take
+    // this workspace for one that holds segment tables
+    LaunchScope ls(kKZeroWords, st);
+    k_zero_words<<<1, 64, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsHist / 4);
+  }
+  {
+    LaunchScope ls(kKHistCheck, st);
+    k_hist_check<<<n, 256, 0, st>>>(hist, shape.d, flags);
+  }
+  {
+    LaunchScope ls(kKPlan, st);
+    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w, 0);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const Shape& shape,
+                                  const unsigned long long* hist, void* ws, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_from_hist_t<kSmallBatch>(clients, n, shape, hist, ws, st);
+  return launch_plan_from_hist_t<kLargeBatch>(clients, n, shape, hist, ws, st);
 }
 
 // ---- diagnostics ---------------------------------------------------------------------

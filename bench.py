@@ -56,6 +56,8 @@ def parse_args():
                     help="candidate slots per client in the encode workspace; 0 = 3 * R * cap(1)")
     ap.add_argument("--profile-kernel", default="", help="kernel whose roofline is reported; default: the one with the largest total time")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-batch", type=int, default=10, help="clients per call of the end-to-end leg: host-to-device copies of one sub-batch overlap the kernels of the previous ones")
+    ap.add_argument("--e2e-streams", type=int, default=3)
     ap.add_argument("--cpu-sample-clients", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -227,21 +229,34 @@ def run_ours(args):
     done = [torch.cuda.Event() for _ in range(n_streams)]
     fork = torch.cuda.Event()
 
+    # the end-to-end leg has its own, smaller sub-batches on a few streams, so that the copy of one
+    # sub-batch runs under the kernels of the ones before it (same kernels, same results)
+    if not args.no_e2e:
+        eb = max(1, min(args.e2e_batch, n_clients))
+        e2e_groups = [list(range(i, min(i + eb, n_clients))) for i in range(0, n_clients, eb)]
+        e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(max(1, min(args.e2e_streams, len(e2e_groups))))]
+        e2e_encoders = [B.BatchEncoder([params[c] for c in g], dev, max_candidates=max_cand) for g in e2e_groups]
+        e2e_agg = B.Aggregator(n_clients, d, dev)
+        e2e_agg.set_clients([o for enc in e2e_encoders for o in enc.outs], weights)
+        e2e_done = [torch.cuda.Event() for _ in e2e_streams]
+
     def step(from_host: bool):
+        g_list, s_list, e_list, a, dn = (e2e_groups, e2e_streams, e2e_encoders, e2e_agg, e2e_done) if from_host else \
+            (groups, streams, encoders, agg, done)
         fork.record(main)
-        for s in streams:
+        for s in s_list:
             s.wait_event(fork)
-        for gi, g in enumerate(groups):
-            s = streams[gi % n_streams]
+        for gi, g in enumerate(g_list):
+            s = s_list[gi % len(s_list)]
             if from_host:
                 with torch.cuda.stream(s):
                     for c in g:
                         dev_x[c].copy_(pinned[c], non_blocking=True)
-            encoders[gi].run([dev_x[c] for c in g], stream=s)
-        for s, e in zip(streams, done):
+            e_list[gi].run([dev_x[c] for c in g], stream=s)
+        for s, e in zip(s_list, dn):
             e.record(s)
             main.wait_event(e)
-        agg.run(n_clients, result, stream=main)
+        a.run(n_clients, result, stream=main)
         if from_host:
             result_host.copy_(result, non_blocking=True)
 
@@ -298,7 +313,11 @@ def run_ours(args):
         e2e_ms, _ = timed(max(1, args.e2e_steps), True)
         e2e_ms /= max(1, args.e2e_steps)
         e2e = {"value": 4.0 * units / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": 4 * d * n_clients, "d2h_bytes_per_step": 4 * d}
+               "h2d_bytes_per_step": 4 * d * n_clients, "d2h_bytes_per_step": 4 * d,
+               "clients_per_call": eb, "streams": len(e2e_streams)}
+        for enc in e2e_encoders:
+            assert enc.status() == B.CVLC_OK, "encode reported a device-side error in the end-to-end leg"
+        assert e2e_agg.status() == B.CVLC_OK
 
     if rank != 0:
         if world > 1:

@@ -497,7 +497,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
 // for every candidate of a client (normally the fourth) is skipped for that client; which buffer
 // holds its data after pass q follows from the mask of skipped passes.
 
-// The clients' candidate arrays are concatenated in units of sort tiles (2048 pairs) and cut
+// The clients' candidate arrays are concatenated in units of sort tiles (kSortTile pairs) and cut
 // into equal contiguous chunks, one per block; a block that crosses a client boundary merges
 // its shared histograms into that client's and starts afresh.
 template <int CAP>
@@ -573,192 +573,281 @@ k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
   if (tid == 0) reinterpret_cast<uint32_t*>(ws + L.off_pass_mask)[c] = mask;
 }
 
-template <int CAP>
-__global__ void __launch_bounds__(kSortThreads, 4)
-k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
+// two adjacent look-back words in one 128-bit access (each 64-bit half is its own atomic access)
+__device__ __forceinline__ void ld_relaxed2(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_relaxed2(unsigned long long* p, unsigned long long a, unsigned long long b) {
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b) : "memory");
+}
+
+struct SortShared {
+  uint32_t tile;                                        // ticket of the tile being worked on
+  uint32_t next;                                        // the ticket after it (known once the tile's items are requested)
+  uint32_t scan_w[kSortThreads / 32];                   // warp totals of the block scan
+  __align__(16) uint16_t wc[kSortThreads / 32][kDigits];  // per warp and digit value: the count, then the first slot
+                                                          // (lanes index it by digit value: the banks are as random as the digits)
+  uint32_t gofs[kDigits];  // per digit value: (position in dst of the tile's first item of that value) - (its slot in the tile)
+  uint32_t mm[kSortThreads / 32][kDigits];  // per warp and digit value: lanes of the current row holding it (zero between rows)
+};
+
+constexpr size_t kSortSharedBytes = (sizeof(SortShared) + 15) & ~(size_t)15;
+constexpr size_t sort_smem_bytes(uint32_t n) { return kSortSharedBytes + (size_t)kSortTile * 8 + (4 * (size_t)n + 1) * 4; }
+
+// One tile of one digit pass.  FULL: the tile holds kSortTile items (no bounds checks in the item loops).
+// Thread t < 256 owns the digit values 2t and 2t + 1 in the counting, scan and look-back steps.
+template <bool FULL, class Prefetch>
+__device__ __forceinline__ void sort_tile(SortShared& sh, unsigned long long* __restrict__ s_items,
+                                          const unsigned long long* __restrict__ src, unsigned long long* __restrict__ dst,
+                                          unsigned long long* __restrict__ state, const unsigned long long* __restrict__ gbase,
+                                          uint32_t tile, uint32_t count, uint32_t n32, uint32_t keytop, int shift,
+                                          int32_t* status, uint32_t next, Prefetch&& prefetch_next) {
   constexpr int kWarps = kSortThreads / 32;
-  static_assert(kWarps == 8, "one 128-bit shared-memory word holds the eight warps' 16-bit counters of a digit value");
-  constexpr int kPerThread = kDigits / kSortThreads;  // digit values owned by a thread
-  __shared__ uint32_t s_tile;
-  __shared__ __align__(16) uint16_t s_wc[kDigits][kWarps];  // per digit value: the warps' counters, then their first slots
-  __shared__ unsigned long long s_gofs[kDigits];           // global position of slot 0 of the tile, per digit value
-  __shared__ uint32_t s_scan_w[kWarps];
-  extern __shared__ unsigned long long s_dyn[];
-  unsigned long long* s_items = s_dyn;                                  // [kSortTile] the tile's items in digit order
-  uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_dyn + kSortTile);  // [n + 1] first sort tile of every client
+  constexpr int IT = kSortItemsPerThread;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned lanemask_lt = (1u << lane) - 1u;
+  const uint32_t wbase = (uint32_t)warp * (32 * IT) + lane;  // this thread's first item inside the tile
+
+  unsigned long long item[IT];
+  uint32_t rd[IT];  // digit value | rank among the warp's items of that value << 16
+  {
+    const unsigned long long* __restrict__ p = src + (size_t)tile * kSortTile + wbase;
+#pragma unroll
+    for (int i = 0; i < IT; ++i) item[i] = (FULL || wbase + i * 32 < count) ? p[i * 32] : ~0ull;
+  }
+  if (tid == 0) sh.next = next;  // waits for the ticket counter's answer, behind the item requests
+  // the look-back needs the digit values' first positions in dst: requested early, used late
+  unsigned long long gb0 = 0, gb1 = 0;
+  if (tid < kDigits / 2) {
+    const ulonglong2 g = *reinterpret_cast<const ulonglong2*>(gbase + 2 * tid);
+    gb0 = g.x;
+    gb1 = g.y;
+  }
+  // stable rank inside the warp, items in (i, lane) order.  The lanes of a row that hold the same digit value
+  // find each other through a word of shared memory that each of them ORs its lane bit into (nine ballots cost
+  // four times the issue slots, a match instruction one step per distinct value in the warp); all of them read
+  // the warp's running count of the value, the highest lane then updates it and clears the word.
+  uint32_t* mm = &sh.mm[warp][0];
+#pragma unroll
+  for (int i = 0; i < IT; ++i) {
+    const bool valid = FULL || (wbase + i * 32 < count);
+    const uint32_t key = (uint32_t)(item[i] >> 32);
+    const uint32_t inv = keytop - (key < keytop ? key : keytop);  // key > keytop only if the plan is not of this update
+    const uint32_t dig = (inv >> shift) & (kDigits - 1);
+    if (valid) atomicOr(mm + dig, 1u << lane);
+    __syncwarp();
+    unsigned peers = 1u << lane;
+    uint32_t pre = 0;
+    if (valid) {
+      peers = *reinterpret_cast<volatile uint32_t*>(mm + dig);
+      pre = *reinterpret_cast<volatile uint16_t*>(&sh.wc[warp][dig]);
+    }
+    __syncwarp();
+    rd[i] = dig | ((pre + __popc(peers & lanemask_lt)) << 16);
+    if (valid && (peers >> lane) == 1u) {  // no peer in a higher lane
+      sh.wc[warp][dig] = (uint16_t)(pre + __popc(peers));
+      mm[dig] = 0u;
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+  prefetch_next(sh.next);
+
+  // counts of the two digit values in every warp (a 32-bit word holds both), published as the tile's aggregate
+  constexpr int kOwners = kDigits / 2;
+  const bool owner = tid < kOwners;
+  uint32_t* wc32 = reinterpret_cast<uint32_t*>(&sh.wc[0][0]);
+  uint32_t tot0 = 0, tot1 = 0, incl = 0;
+  unsigned long long* my_state = state + (size_t)tile * kDigits + 2 * (tid & (kOwners - 1));
+  if (owner) {
+    uint32_t p = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) p += wc32[w * (kDigits / 2) + tid];  // 16-bit lanes: no carry (<= kSortTile)
+    tot0 = p & 0xFFFFu;
+    tot1 = p >> 16;
+    const unsigned long long f = (tile == 0) ? kFlagPrefix : kFlagAgg;
+    st_relaxed2(my_state, f | tot0, f | tot1);
+    // first slot of every digit value inside the tile: block scan in digit order
+    incl = tot0 + tot1;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t o = __shfl_up_sync(kFull, incl, off);
+      if (lane >= off) incl += o;
+    }
+    if (lane == 31) sh.scan_w[warp] = incl;
+  }
+  __syncthreads();
+  if (owner) {
+    uint32_t below = 0;
+#pragma unroll
+    for (int w = 0; w < kOwners / 32; ++w) {
+      const uint32_t v = sh.scan_w[w];
+      if (w < warp) below += v;
+    }
+    const uint32_t dstart0 = below + incl - (tot0 + tot1);
+    const uint32_t dstart1 = dstart0 + tot0;
+    // the counters become first slots: slot of (value, warp) = first slot of the value + items of earlier warps
+    {
+      uint32_t t = dstart0 | (dstart1 << 16);  // both running slots stay below 2^16
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const uint32_t v = wc32[w * (kDigits / 2) + tid];
+        wc32[w * (kDigits / 2) + tid] = t;
+        t += v;
+      }
+    }
+    // decoupled look-back over the client's earlier tiles, both digit values per step
+    unsigned long long run0 = 0, run1 = 0;
+    if (tile > 0) {
+      constexpr int kWin = 4;  // predecessors requested together: one round trip for all of them
+      bool open0 = true, open1 = true;
+      for (long long t = (long long)tile - 1; t >= 0 && (open0 || open1); t -= kWin) {
+        unsigned long long a[kWin], b[kWin];
+#pragma unroll
+        for (int j = 0; j < kWin; ++j) {
+          a[j] = b[j] = kFlagPrefix;  // before the client's first tile: nothing, chain closed
+          if (t - j >= 0) ld_relaxed2(state + (size_t)(t - j) * kDigits + 2 * tid, a[j], b[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < kWin; ++j) {
+          if (!(open0 || open1)) break;
+          int polls = 0;
+          while ((a[j] & kFlagMask) == 0 || (b[j] & kFlagMask) == 0) {
+            if (++polls > kMaxPolls) {
+              set_status(status, CVLC_ERR_DEVICE_TIMEOUT);
+              a[j] = b[j] = kFlagPrefix;  // give up: close both chains
+              break;
+            }
+            if (polls > 64) __nanosleep(64);
+            ld_relaxed2(state + (size_t)(t - j) * kDigits + 2 * tid, a[j], b[j]);
+          }
+          if (open0) {
+            run0 += a[j] & kValMask;
+            open0 = (a[j] & kFlagMask) != kFlagPrefix;
+          }
+          if (open1) {
+            run1 += b[j] & kValMask;
+            open1 = (b[j] & kFlagMask) != kFlagPrefix;
+          }
+        }
+      }
+      st_relaxed2(my_state, kFlagPrefix | (run0 + tot0), kFlagPrefix | (run1 + tot1));
+    }
+    sh.gofs[2 * tid] = (uint32_t)(gb0 + run0) - dstart0;
+    sh.gofs[2 * tid + 1] = (uint32_t)(gb1 + run1) - dstart1;
+  }
+  __syncthreads();
+  // the items go to shared memory in digit order, then out in runs of consecutive addresses
+#pragma unroll
+  for (int i = 0; i < IT; ++i) {
+    if (FULL || wbase + i * 32 < count) {
+      const uint32_t dig = rd[i] & 0xFFFFu;
+      s_items[(uint32_t)sh.wc[warp][dig] + (rd[i] >> 16)] = item[i];
+    }
+  }
+  __syncthreads();
+  if (FULL) {
+#pragma unroll
+    for (int j = 0; j < IT; ++j) {
+      const uint32_t k = j * kSortThreads + tid;
+      const unsigned long long it = s_items[k];
+      const uint32_t key = (uint32_t)(it >> 32);
+      const uint32_t inv = keytop - (key < keytop ? key : keytop);
+      const uint32_t o = sh.gofs[(inv >> shift) & (kDigits - 1)] + k;
+      if (o < n32) dst[o] = it;
+    }
+  } else {
+    for (uint32_t k = tid; k < count; k += kSortThreads) {
+      const unsigned long long it = s_items[k];
+      const uint32_t key = (uint32_t)(it >> 32);
+      const uint32_t inv = keytop - (key < keytop ? key : keytop);
+      const uint32_t o = sh.gofs[(inv >> shift) & (kDigits - 1)] + k;
+      if (o < n32) dst[o] = it;
+    }
+  }
+}
+
+template <int CAP>
+__global__ void __launch_bounds__(kSortThreads, kSortMinBlocks)
+k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
+  static_assert(kSortThreads * 2 >= kDigits && kSortTile <= 0xFFFF, "two digit values per owning thread; 16-bit slots");
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  SortShared& sh = *reinterpret_cast<SortShared*>(s_raw);
+  unsigned long long* s_items = reinterpret_cast<unsigned long long*>(s_raw + kSortSharedBytes);  // [kSortTile] the tile's items in digit order
+  uint32_t* s_prefix = reinterpret_cast<uint32_t*>(s_items + kSortTile);                         // [n + 1] first sort tile of every client
+  uint32_t* s_ncand = s_prefix + (batch.n + 1);  // [n] candidates of the client
+  uint32_t* s_keytop = s_ncand + batch.n;        // [n] top of its key range
+  uint32_t* s_mask = s_keytop + batch.n;         // [n] its constant digits
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (hdr->status != 0) return;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const uint32_t n_clients = batch.n;
   {
     const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + L.off_sort_prefix);
+    const uint32_t* pass_mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask);
     for (uint32_t i = tid; i <= n_clients; i += kSortThreads) s_prefix[i] = prefix[i];
+    for (uint32_t i = tid; i < n_clients; i += kSortThreads) {
+      const cvlc_plan_t* plan = batch.c[i].plan;
+      s_ncand[i] = (uint32_t)plan->n_candidates;  // <= capacity < 2^32: checked by k_encode_init
+      s_keytop[i] = sort_keytop(plan);
+      s_mask[i] = pass_mask[i];
+    }
   }
+  for (int i = tid; i < (kSortThreads / 32) * kDigits; i += kSortThreads) (&sh.mm[0][0])[i] = 0u;
+  if (tid == 0) sh.tile = atomicAdd(&hdr->sort_ticket[pass], 1u);
   __syncthreads();
   const uint32_t total_tickets = hdr->max_sort_tiles * n_clients;
-  const uint32_t* pass_mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask);
   unsigned long long* state_all =
       reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)pass * n_clients * L.sort_tiles_max * kDigits;
-  const unsigned lanemask_lt = (1u << lane) - 1u;
-  uint4* s_wc4 = reinterpret_cast<uint4*>(&s_wc[0][0]);
+  uint4* s_wc4 = reinterpret_cast<uint4*>(&sh.wc[0][0]);
+  const int shift = kDigitBits * pass;
 
   while (true) {
-    if (tid == 0) s_tile = atomicAdd(&hdr->sort_ticket[pass], 1u);
-#pragma unroll
-    for (int q = 0; q < kPerThread; ++q) s_wc4[tid + q * kSortThreads] = make_uint4(0u, 0u, 0u, 0u);
-    __syncthreads();
-    const uint32_t gt = s_tile;
+    const uint32_t gt = sh.tile;
     if (gt >= total_tickets) break;
+    s_wc4[2 * tid] = make_uint4(0u, 0u, 0u, 0u);
+    s_wc4[2 * tid + 1] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();  // everyone has read the ticket; the counters are clear
+    // the next ticket is fetched while this tile is worked on
+    uint32_t next = 0;
+    if (tid == 0) next = atomicAdd(&hdr->sort_ticket[pass], 1u);
     // tile-major tickets with the clients interleaved: the tiles in flight are a few consecutive
     // tiles of every client, which keeps every look-back short
     const uint32_t tile = gt / n_clients;
     const uint32_t c = gt - tile * n_clients;
-    const uint32_t mask = pass_mask[c];
-    if (tile >= s_prefix[c + 1] - s_prefix[c] || (mask & (1u << pass))) {  // no such tile, or a constant digit
-      __syncthreads();  // everyone has read s_tile before the next ticket overwrites it
-      continue;
-    }
-    const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
-    const unsigned long long n = plan->n_candidates;
-    const uint32_t keytop = sort_keytop(plan);
-    const int flips = __popc(~mask & ((1u << pass) - 1u));
-    unsigned long long* buf_a = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
-    unsigned long long* buf_b = reinterpret_cast<unsigned long long*>(ws + L.off_buf_b) + (size_t)c * L.capacity;
-    const unsigned long long* __restrict__ src = (flips & 1) ? buf_b : buf_a;
-    unsigned long long* __restrict__ dst = (flips & 1) ? buf_a : buf_b;
-    unsigned long long* state = state_all + (size_t)s_prefix[c] * kDigits;
-    const unsigned long long* gbase = reinterpret_cast<const unsigned long long*>(ws + L.off_gbase) +
-                                      (size_t)c * kSortPasses * kDigits + (size_t)pass * kDigits;
-
-    unsigned long long item[kSortItemsPerThread];
-    uint32_t rank[kSortItemsPerThread];
-    const unsigned long long first = (unsigned long long)tile * kSortTile + (unsigned long long)warp * (32 * kSortItemsPerThread);
-#pragma unroll
-    for (int i = 0; i < kSortItemsPerThread; ++i) {
-      const unsigned long long idx = first + i * 32 + lane;
-      item[i] = (idx < n) ? src[idx] : ~0ull;
-    }
-    // stable rank inside the warp: items in (i, lane) order.  The lanes holding the same digit value are
-    // found by intersecting the ballots of its nine bits (a match instruction costs as many steps as
-    // there are distinct values in the warp, about thirty here).
-#pragma unroll
-    for (int i = 0; i < kSortItemsPerThread; ++i) {
-      const bool valid = (first + i * 32 + lane) < n;
-      const uint32_t dig = valid ? sort_digit(item[i], pass, keytop) : 0u;
-      unsigned peers = __ballot_sync(kFull, valid);
-#pragma unroll
-      for (int b = 0; b < kDigitBits; ++b) {
-        const unsigned bal = __ballot_sync(kFull, (dig >> b) & 1u);
-        peers &= ((dig >> b) & 1u) ? bal : ~bal;
-      }
-      const int leader = __ffs(peers | (valid ? 0u : 1u << lane)) - 1;
-      uint32_t pre = 0;
-      if (valid && lane == leader) pre = s_wc[dig][warp];
-      pre = __shfl_sync(kFull, pre, leader);
-      rank[i] = pre + __popc(peers & lanemask_lt);
-      if (valid && lane == leader) s_wc[dig][warp] = (uint16_t)(pre + __popc(peers));
-      __syncwarp();
-    }
-    __syncthreads();
-    // thread = digit values tid, tid + 256: the warps' counts of the value (one 128-bit word), the tile
-    // count, the value's first slot inside the tile (block scan in digit order), look-back
-    {
-      uint32_t tot[kPerThread];
-      unsigned long long run[kPerThread];
-      bool open[kPerThread];
-#pragma unroll
-      for (int q = 0; q < kPerThread; ++q) {
-        const int dg = tid + q * kSortThreads;
-        const uint4 cw = s_wc4[dg];
-        const uint32_t w32[4] = {cw.x, cw.y, cw.z, cw.w};
-        uint32_t t = 0;
-#pragma unroll
-        for (int h = 0; h < 4; ++h) t += (w32[h] & 0xFFFFu) + (w32[h] >> 16);
-        tot[q] = t;
-        run[q] = 0;
-        open[q] = tile > 0;
-        st_relaxed(state + (size_t)tile * kDigits + dg, (tile == 0 ? kFlagPrefix : kFlagAgg) | t);
-      }
-      uint32_t dstart[kPerThread];
-      {
-        uint32_t carry = 0;
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-          uint32_t incl = tot[q];
-#pragma unroll
-          for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t o = __shfl_up_sync(kFull, incl, off);
-            if (lane >= off) incl += o;
-          }
-          if (lane == 31) s_scan_w[warp] = incl;
-          __syncthreads();
-          uint32_t below = 0, all = 0;
-#pragma unroll
-          for (int w = 0; w < kWarps; ++w) {
-            const uint32_t v = s_scan_w[w];
-            if (w < warp) below += v;
-            all += v;
-          }
-          dstart[q] = carry + below + incl - tot[q];
-          carry += all;
-          __syncthreads();
+    const uint32_t mask = s_mask[c];
+    auto source = [&](uint32_t cc, uint32_t m) -> unsigned long long* {  // buffer holding client cc's items before this pass
+      const int flips = __popc(~m & ((1u << pass) - 1u));
+      return reinterpret_cast<unsigned long long*>(ws + ((flips & 1) ? L.off_buf_b : L.off_buf_a)) + (size_t)cc * L.capacity;
+    };
+    if (tile < s_prefix[c + 1] - s_prefix[c] && !(mask & (1u << pass))) {  // else: no such tile, or a constant digit
+      const uint32_t n32 = s_ncand[c];
+      const uint32_t keytop = s_keytop[c];
+      const int flips = __popc(~mask & ((1u << pass) - 1u));
+      const unsigned long long* src = source(c, mask);
+      unsigned long long* dst =
+          reinterpret_cast<unsigned long long*>(ws + ((flips & 1) ? L.off_buf_a : L.off_buf_b)) + (size_t)c * L.capacity;
+      unsigned long long* state = state_all + (size_t)s_prefix[c] * kDigits;
+      const unsigned long long* gbase = reinterpret_cast<const unsigned long long*>(ws + L.off_gbase) +
+                                        (size_t)c * kSortPasses * kDigits + (size_t)pass * kDigits;
+      const uint32_t tile_first = tile * (uint32_t)kSortTile;
+      const uint32_t count = (n32 - tile_first < (uint32_t)kSortTile) ? n32 - tile_first : (uint32_t)kSortTile;
+      // the next tile's items are asked into L2 while this one is ranked and written
+      auto prefetch_next = [&](uint32_t nt) {
+        if (nt >= total_tickets) return;
+        const uint32_t t2 = nt / n_clients, c2 = nt - t2 * n_clients;
+        const uint32_t line = t2 * (uint32_t)(kSortTile / 16) + tid;  // 128-byte lines of 16 items
+        if (tid < kSortTile / 16 && line * 16u < s_ncand[c2]) {
+          const unsigned long long* p = source(c2, s_mask[c2]) + (size_t)line * 16;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
         }
-      }
-      // the counters become first slots: slot of (value, warp) = first slot of the value + items of earlier warps
-#pragma unroll
-      for (int q = 0; q < kPerThread; ++q) {
-        const uint4 cw = s_wc4[tid + q * kSortThreads];
-        const uint32_t c32[4] = {cw.x, cw.y, cw.z, cw.w};
-        uint32_t w32[4], t = dstart[q];
-#pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          const uint32_t lo16 = t;
-          t += c32[h] & 0xFFFFu;
-          const uint32_t hi16 = t;
-          t += c32[h] >> 16;
-          w32[h] = (lo16 & 0xFFFFu) | (hi16 << 16);
-        }
-        s_wc4[tid + q * kSortThreads] = make_uint4(w32[0], w32[1], w32[2], w32[3]);
-      }
-      for (long long t = (long long)tile - 1; t >= 0; --t) {
-        bool any_open = false;
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-          if (open[q]) {
-            const unsigned long long sv = wait_state(state + (size_t)t * kDigits + tid + q * kSortThreads, &hdr->status);
-            run[q] += sv & kValMask;
-            if (sv == 0 || (sv & kFlagMask) == kFlagPrefix) open[q] = false;  // sv == 0: timed out, status is set
-            any_open |= open[q];
-          }
-        }
-        if (!any_open) break;
-      }
-#pragma unroll
-      for (int q = 0; q < kPerThread; ++q) {
-        const int dg = tid + q * kSortThreads;
-        if (tile > 0) st_relaxed(state + (size_t)tile * kDigits + dg, kFlagPrefix | (run[q] + tot[q]));
-        s_gofs[dg] = gbase[dg] + run[q] - dstart[q];
-      }
+      };
+      if (count == (uint32_t)kSortTile)
+        sort_tile<true>(sh, s_items, src, dst, state, gbase, tile, count, n32, keytop, shift, &hdr->status, next, prefetch_next);
+      else
+        sort_tile<false>(sh, s_items, src, dst, state, gbase, tile, count, n32, keytop, shift, &hdr->status, next, prefetch_next);
     }
-    __syncthreads();
-    // the items go to shared memory in digit order, then out in runs of consecutive addresses
-#pragma unroll
-    for (int i = 0; i < kSortItemsPerThread; ++i) {
-      if ((first + i * 32 + lane) < n) {
-        const uint32_t dig = sort_digit(item[i], pass, keytop);
-        s_items[(uint32_t)s_wc[dig][warp] + rank[i]] = item[i];
-      }
-    }
-    __syncthreads();
-    {
-      const unsigned long long tile_first = (unsigned long long)tile * kSortTile;
-      const uint32_t count = (n - tile_first < (unsigned long long)kSortTile) ? (uint32_t)(n - tile_first) : (uint32_t)kSortTile;
-      for (uint32_t k = tid; k < count; k += kSortThreads) {
-        const unsigned long long it = s_items[k];
-        const unsigned long long o = s_gofs[sort_digit(it, pass, keytop)] + k;
-        if (o < n && o < L.capacity) dst[o] = it;
-      }
-    }
+    if (tid == 0) sh.tile = next;
     __syncthreads();
   }
 }
@@ -1021,7 +1110,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_select<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSelStages * kSelStageBytes));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_sort_pass<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSortTile * 8 + (CVLC_MAX_BATCH + 1) * 4));
+    e = cudaFuncSetAttribute(k_sort_pass<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem_bytes(CVLC_MAX_BATCH));
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
@@ -1051,7 +1140,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   }
   {
     const uint64_t want = L.sort_tiles_max * n;
-    const unsigned grid = (unsigned)(want < (uint64_t)(4 * kNumSM) ? want : 4 * kNumSM);
+    const unsigned grid = (unsigned)(want < (uint64_t)(kSortMinBlocks * kNumSM) ? want : kSortMinBlocks * kNumSM);
     if (!pws) {  // the selection with known offsets has counted the digits already
       LaunchScope ls(kKSortHist, st);
       k_sort_hist<CAP><<<grid, 256, 0, st>>>(batch, w, L);
@@ -1062,7 +1151,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     }
     for (int pass = 0; pass < kSortPasses; ++pass) {
       LaunchScope ls(kKSortPass, st);
-      k_sort_pass<CAP><<<grid, kSortThreads, (size_t)kSortTile * 8 + ((size_t)n + 1) * 4, st>>>(pass, batch, w, L);
+      k_sort_pass<CAP><<<grid, kSortThreads, sort_smem_bytes(n), st>>>(pass, batch, w, L);
     }
   }
   {

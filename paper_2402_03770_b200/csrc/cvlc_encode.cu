@@ -855,218 +855,235 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 // ===================================================================================
 // K5  per-packet centroid distribution (PQ: min/max; QSGD: l2-norm), stochastic quantization, bit packing
 // ===================================================================================
-// One CTA per (packet, client).  Packet r (longest codes first) holds ranks [Z, Z + cap(y_r)).
+// One CTA works through kPackGroup consecutive packets of one client.  Packet r (longest codes first) holds
+// ranks [Z, Z + cap(y_r)).  The packet is assembled in shared memory: every record ORs its bits into the
+// (at most three) 32-bit words it touches, then the words go out with consecutive addresses.  The ranked
+// pairs are read twice from global memory (statistics, then quantization); the second read hits in cache.
 
 constexpr int kPackThreads = 128;
+constexpr int kPackGroup = 4;  // packets per CTA: the length table is set up once for all of them
 
 template <int CAP, bool QSGD>
 __global__ void __launch_bounds__(kPackThreads)
 k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
        const __grid_constant__ EncLayout L) {
-  extern __shared__ unsigned long long recs[];  // [cap(1)], QSGD: then cap(1) squares
+  extern __shared__ __align__(16) unsigned char s_pack[];  // packet words; QSGD: then cap(1) squares
   __shared__ float s_red[2][kPackThreads / 32];
   __shared__ uint32_t s_y;
   __shared__ unsigned long long s_Z;
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t r = blockIdx.x, c = blockIdx.y;
+  const uint32_t c = blockIdx.y;
   const ClientDesc& cd = batch.c[c];
   const cvlc_plan_t* __restrict__ plan = cd.plan;
   const uint32_t s = shape.s;
+  const uint32_t H = shape.header_bits;
+  const uint32_t n_words = shape.packet_bits / 32;
+  uint32_t* words = reinterpret_cast<uint32_t*>(s_pack);
+  uint32_t* stream_words = reinterpret_cast<uint32_t*>(cd.stream);
 
   const uint32_t mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask)[c];
   const int flips = __popc(~mask & ((1u << kSortPasses) - 1u));
   const unsigned long long* __restrict__ sorted =
       reinterpret_cast<const unsigned long long*>(ws + ((flips & 1) ? L.off_buf_b : L.off_buf_a)) + (size_t)c * L.capacity;
 
-  // packet r -> its code length and first rank: lane l of warp 0 holds length 32 - l (longest first)
+  // packet -> its code length and first rank: lane l of warp 0 holds length 32 - l (longest first) with the
+  // inclusive sums of packets and of records up to and including that length
+  uint32_t yl = 0, ny = 0, cum = 0, capl = 0;
+  unsigned long long zc = 0, nz = 0;
   if (warp == 0) {
-    const int yl = CVLC_MAX_CODE_BITS - lane;
-    const unsigned long long ny = plan->n_y[yl];
-    const unsigned long long nz = ny * plan->cap[yl];
-    unsigned long long cum = ny, zc = nz;  // inclusive scans over the lanes
+    yl = CVLC_MAX_CODE_BITS - lane;
+    ny = plan->n_y[yl];
+    capl = plan->cap[yl];
+    nz = (unsigned long long)ny * capl;
+    cum = ny;
+    zc = nz;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-      const unsigned long long a = __shfl_up_sync(kFull, cum, off), b = __shfl_up_sync(kFull, zc, off);
+      const uint32_t a = __shfl_up_sync(kFull, cum, off);
+      const unsigned long long b = __shfl_up_sync(kFull, zc, off);
       if (lane >= off) {
         cum += a;
         zc += b;
       }
     }
-    const unsigned hit = __ballot_sync(kFull, r < cum);
-    if (hit == 0) {
-      if (lane == 0) s_y = 0;
-    } else if (lane == __ffs(hit) - 1) {
-      s_y = (uint32_t)yl;
-      s_Z = (zc - nz) + (r - (cum - ny)) * plan->cap[yl];
-    }
   }
-  __syncthreads();
-  const uint32_t y = s_y;
-  if (y == 0) return;
-  const unsigned long long Z = s_Z;
-  const uint32_t P = plan->cap[y];
-  const uint32_t wd = s + y;
-  float lo, hi;  // the header's two centroid fields
 
-  if constexpr (QSGD) {
-    // ---- QSGD: |x| against the packet's l2-norm; code = sign bit above a level of s_q = 2^(y-1) - 1 steps ----
-    __shared__ float s_norm;
-    double* sqv = reinterpret_cast<double*>(recs + shape.cap[1]);
-    for (uint32_t j = tid; j < P; j += kPackThreads) {
-      const unsigned long long pair = sorted[Z + j];
-      recs[j] = pair;
-      const double a = (double)__uint_as_float((uint32_t)(pair >> 32));
-      sqv[j] = __dmul_rn(a, a);  // exact: 24 x 24 bits
-    }
-    __syncthreads();
-    // the norm is defined with the squares added in rank order in double: one thread walks the chain
-    if (tid == 0) {
-      double sum = 0.0;
-      uint32_t j = 0;
-      for (; j + 8 <= P; j += 8) {
-        double v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = sqv[j + u];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) sum = __dadd_rn(sum, v[u]);
+  for (int g = 0; g < kPackGroup; ++g) {
+    const uint32_t r = blockIdx.x * kPackGroup + g;
+    if (r >= shape.R) break;
+    if (warp == 0) {
+      const unsigned hit = __ballot_sync(kFull, r < cum);
+      if (hit == 0) {
+        if (lane == 0) s_y = 0;
+      } else if (lane == __ffs(hit) - 1) {
+        s_y = yl;
+        s_Z = (zc - nz) + (unsigned long long)(r - (cum - ny)) * capl;
       }
-      for (; j < P; ++j) sum = __dadd_rn(sum, sqv[j]);
-      const double rt = __dsqrt_rn(sum);
-      s_norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
     }
+    for (uint32_t w = tid; w < n_words; w += kPackThreads) words[w] = 0u;
     __syncthreads();
-    const float norm = s_norm;
-    lo = norm;
-    hi = 0.0f;
-    const uint32_t sq = (uint32_t)((1ull << (y - 1)) - 1ull);  // y >= 2: checked with the plan
-    const double sqd = (double)sq;
-    const double dn = (double)norm;
-    const double scale = (norm > 0.0f) ? __ddiv_rn(sqd, dn) : 0.0;
-    for (uint32_t j = tid; j < P; j += kPackThreads) {
-      const unsigned long long pair = recs[j];
-      const uint32_t key = (uint32_t)(pair >> 32);
-      const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
-      const uint32_t sign = key ? (((uint32_t)pair >> 31) & 1u) : 0u;  // -0 is stored as +0
-      uint32_t level = 0;
-      if (norm > 0.0f) {
-        const double a = (double)__uint_as_float(key);
-        const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
-        // t = (a / norm) * s_q decides floor(t) and [u < frac(t)]; a * (s_q / norm) is within a few ulp of it
-        // and decides the same unless its fraction sits that close to 0, 1 or u
-        const double tf = __dmul_rn(a, scale);
-        const double jf = floor(tf);
-        const double ff = __dsub_rn(tf, jf);
-        const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
-        if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < sqd) {
-          level = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
-        } else {
-          const double t = __dmul_rn(__ddiv_rn(a, dn), sqd);
-          double j0 = floor(t);
-          if (j0 > sqd) j0 = sqd;
-          const double frac = __dsub_rn(t, j0);
-          level = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
-          if (level > sq) level = sq;
+    const uint32_t y = s_y;
+    if (y == 0) break;  // fewer packets planned than the stream holds: caught by the plan check
+    const unsigned long long Z = s_Z;
+    const uint32_t P = plan->cap[y];
+    const uint32_t wd = s + y;
+    const unsigned long long* __restrict__ seg = sorted + Z;
+    float lo, hi;  // the header's two centroid fields
+
+    // a record's bits, low bit first from packet bit H + j * wd
+    auto put = [&](uint32_t j, unsigned long long rec) {
+      const uint32_t bitpos = H + j * wd;
+      const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+      const unsigned long long lo64 = rec << sh;
+      const uint32_t p0 = (uint32_t)lo64, p1 = (uint32_t)(lo64 >> 32);
+      const uint32_t p2 = sh ? (uint32_t)(rec >> (64 - sh)) : 0u;
+      if (p0) atomicOr(words + w, p0);
+      if (p1) atomicOr(words + w + 1, p1);
+      if (p2) atomicOr(words + w + 2, p2);
+    };
+
+    if constexpr (QSGD) {
+      // ---- QSGD: |x| against the packet's l2-norm; code = sign bit above a level of s_q = 2^(y-1) - 1 steps ----
+      __shared__ float s_norm;
+      double* sqv = reinterpret_cast<double*>(s_pack + (((size_t)n_words * 4 + 15) & ~(size_t)15));
+      for (uint32_t j = tid; j < P; j += kPackThreads) {
+        const double a = (double)__uint_as_float((uint32_t)(seg[j] >> 32));
+        sqv[j] = __dmul_rn(a, a);  // exact: 24 x 24 bits
+      }
+      __syncthreads();
+      // the norm is defined with the squares added in rank order in double: one thread walks the chain
+      if (tid == 0) {
+        double sum = 0.0;
+        uint32_t j = 0;
+        for (; j + 8 <= P; j += 8) {
+          double v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) v[u] = sqv[j + u];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) sum = __dadd_rn(sum, v[u]);
         }
+        for (; j < P; ++j) sum = __dadd_rn(sum, sqv[j]);
+        const double rt = __dsqrt_rn(sum);
+        s_norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
       }
-      const uint32_t code = (sign << (y - 1)) | level;
-      recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
+      __syncthreads();
+      const float norm = s_norm;
+      lo = norm;
+      hi = 0.0f;
+      const uint32_t sq = (uint32_t)((1ull << (y - 1)) - 1ull);  // y >= 2: checked with the plan
+      const double sqd = (double)sq;
+      const double dn = (double)norm;
+      const double scale = (norm > 0.0f) ? __ddiv_rn(sqd, dn) : 0.0;
+      for (uint32_t j = tid; j < P; j += kPackThreads) {
+        const unsigned long long pair = seg[j];
+        const uint32_t key = (uint32_t)(pair >> 32);
+        const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
+        const uint32_t sign = key ? (((uint32_t)pair >> 31) & 1u) : 0u;  // -0 is stored as +0
+        uint32_t level = 0;
+        if (norm > 0.0f) {
+          const double a = (double)__uint_as_float(key);
+          const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+          // t = (a / norm) * s_q decides floor(t) and [u < frac(t)]; a * (s_q / norm) is within a few ulp of it
+          // and decides the same unless its fraction sits that close to 0, 1 or u
+          const double tf = __dmul_rn(a, scale);
+          const double jf = floor(tf);
+          const double ff = __dsub_rn(tf, jf);
+          const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
+          if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < sqd) {
+            level = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
+          } else {
+            const double t = __dmul_rn(__ddiv_rn(a, dn), sqd);
+            double j0 = floor(t);
+            if (j0 > sqd) j0 = sqd;
+            const double frac = __dsub_rn(t, j0);
+            level = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
+            if (level > sq) level = sq;
+          }
+        }
+        const uint32_t code = (sign << (y - 1)) | level;
+        put(j, (unsigned long long)pid | ((unsigned long long)code << s));
+      }
+    } else {
+      // ---- PQ: minimum / maximum of the packet's signed values (its centroid distribution) ----
+      float vmin = CUDART_INF_F, vmax = -CUDART_INF_F;
+      for (uint32_t j = tid; j < P; j += kPackThreads) {
+        const unsigned long long pair = seg[j];
+        const uint32_t key = (uint32_t)(pair >> 32);
+        const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;  // -0 is stored as +0
+        const float v = __uint_as_float(b);
+        vmin = fminf(vmin, v);
+        vmax = fmaxf(vmax, v);
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        vmin = fminf(vmin, __shfl_xor_sync(kFull, vmin, off));
+        vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, off));
+      }
+      if (lane == 0) {
+        s_red[0][warp] = vmin;
+        s_red[1][warp] = vmax;
+      }
+      __syncthreads();
+      lo = s_red[0][0];
+      hi = s_red[1][0];
+#pragma unroll
+      for (int w = 1; w < kPackThreads / 32; ++w) {
+        lo = fminf(lo, s_red[0][w]);
+        hi = fmaxf(hi, s_red[1][w]);
+      }
+
+      // stochastic rounding onto the 2^y uniform centroids of [lo, hi]
+      const double Lc = (double)((1ull << y) - 1ull);
+      const double dlo = (double)lo;
+      const double den = __dsub_rn((double)hi, dlo);
+      const double scale = (hi != lo) ? __ddiv_rn(Lc, den) : 0.0;
+      for (uint32_t j = tid; j < P; j += kPackThreads) {
+        const unsigned long long pair = seg[j];
+        const uint32_t key = (uint32_t)(pair >> 32);
+        const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
+        const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;
+        uint32_t code = 0;
+        if (hi != lo) {
+          const double num = __dsub_rn((double)__uint_as_float(b), dlo);
+          const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+          // t = (num / den) * L decides floor(t) and [u < frac(t)].  num * (L / den) is within a few ulp of it;
+          // unless its fraction sits that close to 0, 1 or u, both decisions are the same and the division
+          // is not needed.
+          const double tf = __dmul_rn(num, scale);
+          const double jf = floor(tf);
+          const double ff = __dsub_rn(tf, jf);
+          const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
+          if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < Lc) {
+            code = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
+          } else {
+            const double t = __dmul_rn(__ddiv_rn(num, den), Lc);
+            double j0 = floor(t);
+            if (j0 > Lc) j0 = Lc;
+            const double frac = __dsub_rn(t, j0);
+            code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
+          }
+        }
+        put(j, (unsigned long long)pid | ((unsigned long long)code << s));
+      }
+    }  // PQ
+
+    // packet header {s, y, lo, hi} in bits 0..79 (bits 80..H-1 stay zero)
+    if (tid == 0) {
+      const uint32_t blo = __float_as_uint(lo), bhi = __float_as_uint(hi);
+      atomicOr(words + 0, s | (y << 8) | (blo << 16));
+      atomicOr(words + 1, (blo >> 16) | (bhi << 16));
+      atomicOr(words + 2, bhi >> 16);
     }
     __syncthreads();
-  } else {
-  // ---- PQ: minimum / maximum of the packet's signed values (its centroid distribution) ----
-  float vmin = CUDART_INF_F, vmax = -CUDART_INF_F;
-  for (uint32_t j = tid; j < P; j += kPackThreads) {
-    const unsigned long long pair = sorted[Z + j];
-    recs[j] = pair;
-    const uint32_t key = (uint32_t)(pair >> 32);
-    const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;  // -0 is stored as +0
-    const float v = __uint_as_float(b);
-    vmin = fminf(vmin, v);
-    vmax = fmaxf(vmax, v);
-  }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    vmin = fminf(vmin, __shfl_xor_sync(kFull, vmin, off));
-    vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, off));
-  }
-  if (lane == 0) {
-    s_red[0][warp] = vmin;
-    s_red[1][warp] = vmax;
-  }
-  __syncthreads();
-  lo = s_red[0][0];
-  hi = s_red[1][0];
-#pragma unroll
-  for (int w = 1; w < kPackThreads / 32; ++w) {
-    lo = fminf(lo, s_red[0][w]);
-    hi = fmaxf(hi, s_red[1][w]);
-  }
-
-  // stochastic rounding onto the 2^y uniform centroids of [lo, hi]
-  const double Lc = (double)((1ull << y) - 1ull);
-  const double dlo = (double)lo;
-  const double den = __dsub_rn((double)hi, dlo);
-  const double scale = (hi != lo) ? __ddiv_rn(Lc, den) : 0.0;
-  for (uint32_t j = tid; j < P; j += kPackThreads) {
-    const unsigned long long pair = recs[j];
-    const uint32_t key = (uint32_t)(pair >> 32);
-    const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
-    const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;
-    uint32_t code = 0;
-    if (hi != lo) {
-      const double num = __dsub_rn((double)__uint_as_float(b), dlo);
-      const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
-      // t = (num / den) * L decides floor(t) and [u < frac(t)].  num * (L / den) is within a few ulp of it;
-      // unless its fraction sits that close to 0, 1 or u, both decisions are the same and the division
-      // is not needed.
-      const double tf = __dmul_rn(num, scale);
-      const double jf = floor(tf);
-      const double ff = __dsub_rn(tf, jf);
-      const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
-      if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < Lc) {
-        code = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
-      } else {
-        const double t = __dmul_rn(__ddiv_rn(num, den), Lc);
-        double j0 = floor(t);
-        if (j0 > Lc) j0 = Lc;
-        const double frac = __dsub_rn(t, j0);
-        code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
-      }
-    }
-    recs[j] = (unsigned long long)pid | ((unsigned long long)code << s);
-  }
-  __syncthreads();
-  }  // PQ
-
-  // gather the packet's 32-bit words: header {s, y, lo, hi}, then records of wd bits from bit H
-  const uint32_t H = shape.header_bits;
-  const uint32_t n_words = shape.packet_bits / 32;
-  uint32_t* stream_words = reinterpret_cast<uint32_t*>(cd.stream);
-  uint32_t* pkt = stream_words + CVLC_STREAM_HEADER_BYTES / 4 + (size_t)r * n_words;
-  const uint32_t blo = __float_as_uint(lo), bhi = __float_as_uint(hi);
-  const uint32_t payload_end = H + P * wd;
-  for (uint32_t w = tid; w < n_words; w += kPackThreads) {
-    const uint32_t bit0 = w * 32;
-    uint32_t val = 0;
-    if (w == 0) val = s | (y << 8) | (blo << 16);
-    if (w == 1) val = (blo >> 16) | (bhi << 16);
-    if (w == 2) val = bhi >> 16;
-    if (bit0 + 32 > H && bit0 < payload_end) {
-      uint32_t j = (bit0 > H) ? (bit0 - H) / wd : 0u;
-      for (; j < P; ++j) {
-        const int shift = (int)(H + j * wd) - (int)bit0;  // position of the record's bit 0 in this word
-        if (shift >= 32) break;
-        const unsigned long long rec = recs[j];
-        val |= (shift >= 0) ? (uint32_t)(rec << shift) : (uint32_t)(rec >> (-shift));
-      }
-    }
-    pkt[w] = val;
+    uint32_t* pkt = stream_words + CVLC_STREAM_HEADER_BYTES / 4 + (size_t)r * n_words;
+    for (uint32_t w = tid; w < n_words; w += kPackThreads) pkt[w] = words[w];
+    __syncthreads();  // the word buffer (and s_y, s_Z, s_red) are reused by the next packet
   }
 
   // global header (64 bytes), written once per client
-  if (r == 0 && tid < 16) {
+  if (blockIdx.x == 0 && tid < 16) {
     uint32_t v = 0;
     const unsigned long long Bbits = (unsigned long long)__double_as_longlong(cd.scale_B);
     const unsigned long long k = plan->k;
@@ -1121,7 +1138,8 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   const EncLayout L = enc_layout(shape.d, n, capacity);
   unsigned char* w = static_cast<unsigned char*>(ws);
   const bool qsgd = shape.quantizer == CVLC_QUANT_QSGD;
-  const size_t pack_smem = (size_t)shape.cap[1] * (qsgd ? 16 : 8);  // records; QSGD: and their squares
+  // packet words; QSGD: and the squares of a packet's values
+  const size_t pack_smem = (((size_t)shape.packet_bits / 8 + 15) & ~(size_t)15) + (qsgd ? (size_t)shape.cap[1] * 8 : 0);
 
   const Partition part = make_partition(shape.d, n);
   const unsigned char* pws = static_cast<const unsigned char*>(plan_ws);
@@ -1157,9 +1175,9 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   {
     LaunchScope ls(kKPack, st);
     if (qsgd)
-      k_pack<CAP, true><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+      k_pack<CAP, true><<<dim3((shape.R + kPackGroup - 1) / kPackGroup, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
     else
-      k_pack<CAP, false><<<dim3(shape.R, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+      k_pack<CAP, false><<<dim3((shape.R + kPackGroup - 1) / kPackGroup, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
   }
   return cudaGetLastError();
 }

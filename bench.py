@@ -287,7 +287,7 @@ def run_ours(args):
     assert agg.status() == B.CVLC_OK, "decode-aggregate reported a device-side error"
 
     launches_before = B.cvlc_launch_count()
-    per_step_launch_cap = 16 * len(groups) + 8
+    per_step_launch_cap = 16 * len(groups) + 8 + 3 * (d // (24 << 20) + 1)  # decode: one fill + one launch per window
     B.cvlc_profile_select("*", per_step_launch_cap * args.steps)
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -372,6 +372,10 @@ def run_ours(args):
     # whole-step minimum bytes (read every update once, write every stream; read the streams, write the aggregate)
     step_min_bytes = n_clients * (4.0 * d + stream_bytes) + n_clients * stream_bytes + 4.0 * d
     step_frac = step_min_bytes / (ms_per_step * 1e-3) / 1e9 / peak
+    # the same with every pass counted at its own minimum (histogram read, selection read + candidates, three
+    # ranking passes, pack, decode): what this multi-pass design has to move
+    pass_bytes = sum(alg_bytes_per_step[k] for k in ("k_hist", "k_select", "k_sort_pass", "k_pack", "k_decode"))
+    pass_frac = pass_bytes / (ms_per_step * 1e-3) / 1e9 / peak
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -389,6 +393,7 @@ def run_ours(args):
                    "multi_gpu": "replicas only: every rank runs its own clients and aggregator"},
         "params_per_s": units / (ms_per_step * 1e-3),
         "step_min_bytes_frac_of_hbm_peak": step_frac,
+        "step_pass_bytes_frac_of_hbm_peak": pass_frac,
         "per_step_ms": per,
         "plan_of_client_0": {"k": int(plans[0].k), "R": int(plans[0].R), "n_candidates": int(plans[0].n_candidates), "alpha_q": plans[0].alpha_q,
                  "lengths": {str(y): int(plans[0].n_y[y]) for y in range(33) if plans[0].n_y[y]}},

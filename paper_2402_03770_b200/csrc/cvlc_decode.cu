@@ -8,6 +8,7 @@ namespace cvlc {
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kPrepThreads = 1024;
 constexpr int kDecodeThreads = 256;
+constexpr uint64_t kDecodeWindow = 24ull << 20;  // coordinates of the accumulator filled per decode launch (96 MB: inside the L2)
 
 struct StreamHead {
   uint32_t magic, ver_q_s, d_lo, d_hi, R, packet_bits, header_bits, client_id, seed_lo, seed_hi, round, zero, B_lo, B_hi, k_lo, k_hi;
@@ -112,10 +113,33 @@ k_fill_zero(float* __restrict__ out, uint64_t d) {
   if (blockIdx.x == 0 && threadIdx.x < (d & 3)) out[(nvec << 2) + threadIdx.x] = 0.f;
 }
 
-// K6  decode + dequantize + weighted scatter-accumulate, one warp per packet
+// A stream word is read once per window pass and should not push the accumulator's window out of the L2.
+__device__ __forceinline__ uint64_t stream_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint32_t ld_stream(const uint32_t* p, uint64_t pol) {
+  uint32_t v;
+  asm volatile("ld.global.nc.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol));
+  return v;
+}
+
+// asks for n floats into the L2, one request per 128-byte line
+__global__ void __launch_bounds__(256)
+k_prefetch_l2(const float* __restrict__ p, uint64_t n) {
+  const uint64_t lines = (n * 4 + 127) / 128;
+  const char* base = reinterpret_cast<const char*>(p);
+  for (uint64_t l = (uint64_t)blockIdx.x * 256 + threadIdx.x; l < lines; l += (uint64_t)gridDim.x * 256)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + l * 128));
+}
+
+// K6  decode + dequantize + weighted scatter-accumulate, one warp per packet.  Only the records whose
+// position lies in [win_lo, win_hi) are accumulated: an accumulator larger than the L2 is filled window by
+// window (one launch each), so that the reductions stay in the L2 instead of becoming DRAM read-modify-writes.
 __global__ void __launch_bounds__(kDecodeThreads)
 k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uint32_t s, float* __restrict__ out,
-         unsigned char* ws) {
+         unsigned char* ws, uint64_t win_lo, uint64_t win_hi) {
   extern __shared__ uint32_t s_prefix[];  // [n + 1]
   int32_t* status = reinterpret_cast<int32_t*>(ws + kDecWsStatus);
   const float* coef = reinterpret_cast<const float*>(ws + kDecWsCoef);
@@ -128,6 +152,7 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
   const int lane = threadIdx.x & 31;
   const uint32_t warps_total = gridDim.x * (kDecodeThreads / 32);
   const unsigned long long pid_mask = (1ull << s) - 1ull;
+  const uint64_t pol = stream_policy();
 
   for (uint32_t g = blockIdx.x * (kDecodeThreads / 32) + (threadIdx.x >> 5); g < total; g += warps_total) {
     // client of packet g: last c with prefix[c] <= g
@@ -140,10 +165,10 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
     const uint32_t pb = meta[2 * c] & ~31u, quantizer = meta[2 * c] & 31u, H = meta[2 * c + 1];
     const uint32_t n_words = pb >> 5;
     const uint32_t* pkt = reinterpret_cast<const uint32_t*>(streams[c] + CVLC_STREAM_HEADER_BYTES) + (size_t)r * n_words;
-    const uint32_t w0 = __ldg(pkt), w1 = __ldg(pkt + 1), w2 = __ldg(pkt + 2);
+    const uint32_t w0 = ld_stream(pkt, pol), w1 = ld_stream(pkt + 1, pol), w2 = ld_stream(pkt + 2, pol);
     const uint32_t ps = w0 & 0xFF, y = (w0 >> 8) & 0xFF;
     uint32_t y_prev = CVLC_MAX_CODE_BITS;
-    if (r > 0) y_prev = (__ldg(pkt - n_words) >> 8) & 0xFF;
+    if (r > 0) y_prev = (ld_stream(pkt - n_words, pol) >> 8) & 0xFF;
     if (ps != s || y < 1 || y > CVLC_MAX_CODE_BITS || y > y_prev) {  // lengths never increase along a stream
       if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
       continue;
@@ -169,11 +194,11 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
       const uint32_t bit = H + j * wd;
       const uint32_t wi = bit >> 5, sh = bit & 31;
       // a record of up to 63 bits starting at bit sh of word wi spans at most three words
-      const unsigned long long a = __ldg(pkt + wi);
-      const unsigned long long b = (wi + 1 < n_words) ? __ldg(pkt + wi + 1) : 0u;
+      const unsigned long long a = ld_stream(pkt + wi, pol);
+      const unsigned long long b = (wi + 1 < n_words) ? ld_stream(pkt + wi + 1, pol) : 0u;
       unsigned long long rec = (a | (b << 32)) >> sh;
       if (sh + wd > 64) {
-        const unsigned long long c2 = (wi + 2 < n_words) ? __ldg(pkt + wi + 2) : 0u;
+        const unsigned long long c2 = (wi + 2 < n_words) ? ld_stream(pkt + wi + 2, pol) : 0u;
         rec |= c2 << (64 - sh);
       }
       const unsigned long long pid = rec & pid_mask;
@@ -182,6 +207,7 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
         set_status(status, CVLC_ERR_BAD_STREAM);
         continue;
       }
+      if (pid < win_lo || pid >= win_hi) continue;
       float v;
       if (qsgd) {
         const float mag = (float)__dmul_rn((double)(code & level_mask), step);
@@ -199,14 +225,25 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
                           void* ws, cudaStream_t st) {
   unsigned char* w = static_cast<unsigned char*>(ws);
   { LaunchScope ls(kKDecodePrepare, st); k_decode_prepare<<<1, kPrepThreads, 0, st>>>(streams, stream_bytes, weights, n, weight_total, d, s, w); }
-  if (!accumulate) {
-    const uint64_t nvec = d >> 2;
-    uint64_t want = (nvec + 255) / 256;
+  // Windows of equal size (a multiple of 1024 coordinates), none above kDecodeWindow.  Each window is brought
+  // into the L2 right before its decode launch, by the zero fill or, when accumulating, by a prefetch: a
+  // reduction that misses the L2 is a DRAM read-modify-write.
+  const uint64_t n_win = (d + kDecodeWindow - 1) / kDecodeWindow;
+  const uint64_t win = (((d + n_win - 1) / n_win) + 1023) & ~(uint64_t)1023;
+  for (uint64_t lo = 0; lo < d; lo += win) {
+    const uint64_t hi = lo + win < d ? lo + win : d;
+    const uint64_t want = ((hi - lo) / 4 + 255) / 256;
     const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? (want ? want : 1) : 8 * kNumSM);
-    LaunchScope ls(kKFillZero, st);
-    k_fill_zero<<<grid, 256, 0, st>>>(out, d);
+    if (!accumulate) {
+      LaunchScope ls(kKFillZero, st);
+      k_fill_zero<<<grid, 256, 0, st>>>(out + lo, hi - lo);
+    } else if (n_win > 1) {
+      LaunchScope ls(kKFillZero, st);
+      k_prefetch_l2<<<grid, 256, 0, st>>>(out + lo, hi - lo);
+    }
+    LaunchScope ls(kKDecode, st);
+    k_decode<<<8 * kNumSM, kDecodeThreads, ((size_t)n + 1) * 4, st>>>(streams, n, d, s, out, w, lo, hi);
   }
-  { LaunchScope ls(kKDecode, st); k_decode<<<8 * kNumSM, kDecodeThreads, ((size_t)n + 1) * 4, st>>>(streams, n, d, s, out, w); }
   return cudaGetLastError();
 }
 

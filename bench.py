@@ -34,9 +34,10 @@ METRIC = "encode+decode_aggregate throughput (4*d*clients / step time)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the
-# kernel named by --profile-kernel (profiles/); None when no capture matches the current kernel.
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per client and launch from the committed ncu capture
+# (profiles/: resnet18 shape, 2 bits per coordinate, PQ, 8 clients) of the kernels whose traffic grows in
+# proportion to the client count; scaled to the clients of a launch, None for any other configuration.
+NCU_TRAFFIC_BYTES_PER_CLIENT = {"k_select": (358.73e6 + 28.07e6) / 8, "k_hist": (358.52e6 + 5.15e6) / 8}
 
 
 def parse_args():
@@ -357,10 +358,13 @@ def run_ours(args):
         kn, kms = kernel_times[dominant]
         if dominant in alg_bytes_per_step:
             per_launch = alg_bytes_per_step[dominant] * args.steps / kn
+            captured = (w.name == "resnet18" and d == w.d and bpc == 2.0 and args.quantizer == "pq"
+                        and dominant in NCU_TRAFFIC_BYTES_PER_CLIENT)
+            ncu_traffic = NCU_TRAFFIC_BYTES_PER_CLIENT[dominant] * n_clients / n_groups if captured else None
             achieved = per_launch / (kms / kn * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak,
                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                        "traffic": NCU_TRAFFIC_BYTES.get(dominant), "launches_timed": kn,
+                        "traffic": ncu_traffic, "launches_timed": kn,
                         "mean_launch_us": kms / kn * 1e3, "algorithmic_bytes_per_launch": per_launch}
         else:
             # the single-CTA-per-client planner: FP64 series arithmetic with O(1) data, bound by the

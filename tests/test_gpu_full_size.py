@@ -136,3 +136,16 @@ def test_stress_1e8_in_accumulate_batches(env):
     lengths = {y for y in range(33) if enc.read_plan(0).n_y[y]}
     assert enc.read_plan(0).k < w.d // 100 and len(lengths) >= 2        # mostly 0-bit (sparsified) coordinates
     decode_both(outs, [r[2] for r in ref], W.client_weights(w)[clients], w.d, torch, B, batches=2)
+
+
+def test_decode_windows_with_a_ragged_last_window(env):
+    # d just above one accumulator window and not a multiple of 4: two windows, the second 1031 coordinates
+    # short of the first and ending on a scalar tail; first call overwrites, second accumulates
+    torch, B = env
+    w = W.WORKLOADS["stress"]
+    d = (24 << 20) + 1031
+    clients = [0, 1]
+    ref = oracle_encode_clients("stress", clients, d, 0.25, procs=2)
+    enc, outs = gpu_batch_encode("stress", clients, d, 0.25, 0, torch, B)
+    check_against_oracle(enc, outs, ref)
+    decode_both(outs, [r[2] for r in ref], np.array([1.0, 3.0], dtype=np.float32), d, torch, B, batches=2)

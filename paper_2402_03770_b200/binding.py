@@ -433,13 +433,19 @@ class BatchEncoder:
         self._pa = _params_array(self.params)
         self._oa = _ptr_array(self.outs)
 
+    def plan(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0):
+        self._xa = _ptr_array(xs)
+        cvlc_plan_batch(xs, self.params, self.plans, self.plan_ws, fixed_y, stream, _cache=(self._xa, self._pa))
+
+    def encode(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, use_plan_ws: bool = True):
+        cvlc_encode_batch(xs, self.params, self.plans, self.outs, self.enc_ws, self.max_candidates, stream,
+                          _cache=(self._xa, self._pa, self._oa), plan_ws=self.plan_ws if use_plan_ws else None)
+        return self.outs
+
     def run(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0,
             use_plan_ws: bool = True):
-        xa = _ptr_array(xs)
-        cvlc_plan_batch(xs, self.params, self.plans, self.plan_ws, fixed_y, stream, _cache=(xa, self._pa))
-        cvlc_encode_batch(xs, self.params, self.plans, self.outs, self.enc_ws, self.max_candidates, stream,
-                          _cache=(xa, self._pa, self._oa), plan_ws=self.plan_ws if use_plan_ws else None)
-        return self.outs
+        self.plan(xs, stream, fixed_y)
+        return self.encode(xs, stream, use_plan_ws)
 
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         rc = cvlc_read_status(self.plan_ws, stream)

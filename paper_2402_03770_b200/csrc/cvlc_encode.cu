@@ -357,7 +357,11 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const float4* __restrict__ xseg = reinterpret_cast<const float4*>(x) + u0;
     const cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
     const uint32_t thresh = plan->thresh_bin << 19;
-    const float thresh_f = __uint_as_float(thresh);  // finite inputs: |x| >= thresh_f <=> key >= thresh
+    // finite inputs: key >= thresh <=> |x| > the float just below thresh <=> (that float) - |x| is negative.  The
+    // difference of two distinct floats never rounds to zero, so its sign bit is the candidate flag: one
+    // subtraction and one funnel shift per coordinate.  thresh == 0: every coordinate is a candidate.
+    const float below_thresh_f = __uint_as_float(thresh ? thresh - 1u : 0u);
+    const uint32_t cap32 = (uint32_t)L.capacity;  // <= d <= 2^31
     const uint32_t keytop = sort_keytop(plan);
     const uint32_t seg = q + c;
     unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
@@ -404,17 +408,23 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       // this thread's 16 consecutive coordinates: units 4 tid .. 4 tid + 3 of the tile
       uint32_t m = 0;
       const uint32_t g0 = (uint32_t)kSelVec * tid;
+      const uint32_t ct = ((uint32_t)tid >> 1) & (uint32_t)(kSelVec - 1);
       const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < kSelVec) ? n_vec - base - g0 : kSelVec) : 0u;
 #pragma unroll
       for (int j = 0; j < kSelVec; ++j) {
         if ((uint32_t)j < left) {
-          const float4 f = src[sel_slot(g0 + j)];
-          m |= (fabsf(f.x) >= thresh_f ? 1u : 0u) << (4 * j);
-          m |= (fabsf(f.y) >= thresh_f ? 1u : 0u) << (4 * j + 1);
-          m |= (fabsf(f.z) >= thresh_f ? 1u : 0u) << (4 * j + 2);
-          m |= (fabsf(f.w) >= thresh_f ? 1u : 0u) << (4 * j + 3);
+          // units 4 tid + j sit in slots 4 tid + (j ^ ct): the swizzle only touches the two low bits
+          const float4 f = src[g0 + ((uint32_t)j ^ ct)];
+          m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.x))), m, 1);
+          m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.y))), m, 1);
+          m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.z))), m, 1);
+          m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.w))), m, 1);
+        } else {
+          m <<= 4;
         }
       }
+      if (thresh == 0u) m = (left >= (uint32_t)kSelVec) ? 0xFFFFu : (0xFFFFu << (4 * (kSelVec - left))) & 0xFFFFu;
+      // coordinate c of the thread (0 .. 15, ascending index) is bit 15 - c of m
       const uint32_t cnt = __popc(m);
       // block scan of the per-thread counts: inside the warp, then over the warp totals
       uint32_t incl = cnt;
@@ -436,18 +446,20 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       const uint32_t below = __shfl_sync(kFull, wincl - wt, warp);
       parity ^= 1;
       // emit this thread's candidates (few): values are re-read from the staging buffer
-      unsigned long long o = run + below + incl - cnt;
-      const uint32_t* srcw = reinterpret_cast<const uint32_t*>(src);
-      const uint64_t e_base = (u0 + base + g0) * 4;
+      uint32_t o = (uint32_t)run + below + incl - cnt;  // positions inside a client's buffer fit 32 bits
+      const uint32_t* srcw16 = reinterpret_cast<const uint32_t*>(src) + 16 * tid;  // this thread's 16 staged words
+      const uint32_t cx = ct << 2;
+      const uint32_t e32 = (uint32_t)((u0 + base + g0) * 4);  // index of the thread's first coordinate (< 2^31)
       while (m) {
-        const int bit = __ffs(m) - 1;
-        m &= m - 1;
-        const uint32_t b = srcw[sel_slot(g0 + (bit >> 2)) * 4 + (bit & 3)];
-        const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) |
-                                        (unsigned long long)(e_base + bit);
-        if (o < L.capacity) out[o] = pair;
+        const int hb = 31 - __clz(m);  // highest flag = lowest index first
+        m ^= 1u << hb;
+        const uint32_t c16 = 15u - (uint32_t)hb;
+        const uint32_t b = srcw16[c16 ^ cx];
+        const uint32_t key = b & 0x7FFFFFFFu;
+        if (o < cap32) out[o] = ((unsigned long long)key << 32) | (unsigned long long)((b & 0x80000000u) | (e32 + c16));
+        const uint32_t inv = keytop - (key < keytop ? key : keytop);
 #pragma unroll
-        for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + sort_digit(pair, p, keytop)], 1u);
+        for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + ((inv >> (kDigitBits * p)) & (kDigits - 1))], 1u);
         ++o;
       }
       run += tot;

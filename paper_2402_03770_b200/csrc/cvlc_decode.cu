@@ -8,6 +8,7 @@ namespace cvlc {
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kPrepThreads = 1024;
 constexpr int kDecodeThreads = 256;
+constexpr uint32_t kDecStageWords = 512;  // packets up to 2 KB are staged in shared memory
 constexpr uint64_t kDecodeWindow = 24ull << 20;  // coordinates of the accumulator filled per decode launch (96 MB: inside the L2)
 
 struct StreamHead {
@@ -141,6 +142,10 @@ __global__ void __launch_bounds__(kDecodeThreads)
 k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uint32_t s, float* __restrict__ out,
          unsigned char* ws, uint64_t win_lo, uint64_t win_hi) {
   extern __shared__ uint32_t s_prefix[];  // [n + 1]
+  // a packet of up to kDecStageWords words is first copied to the warp's own shared-memory buffer with
+  // coalesced, independent loads; the records are then cut out of shared memory (larger packets: out of global)
+  __shared__ uint32_t s_pkt[kDecodeThreads / 32][kDecStageWords];
+  uint32_t* sp = s_pkt[threadIdx.x >> 5];
   int32_t* status = reinterpret_cast<int32_t*>(ws + kDecWsStatus);
   const float* coef = reinterpret_cast<const float*>(ws + kDecWsCoef);
   const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + dec_off_prefix(n));
@@ -165,10 +170,17 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
     const uint32_t pb = meta[2 * c] & ~31u, quantizer = meta[2 * c] & 31u, H = meta[2 * c + 1];
     const uint32_t n_words = pb >> 5;
     const uint32_t* pkt = reinterpret_cast<const uint32_t*>(streams[c] + CVLC_STREAM_HEADER_BYTES) + (size_t)r * n_words;
-    const uint32_t w0 = ld_stream(pkt, pol), w1 = ld_stream(pkt + 1, pol), w2 = ld_stream(pkt + 2, pol);
-    const uint32_t ps = w0 & 0xFF, y = (w0 >> 8) & 0xFF;
+    const bool staged = n_words <= kDecStageWords;
     uint32_t y_prev = CVLC_MAX_CODE_BITS;
     if (r > 0) y_prev = (ld_stream(pkt - n_words, pol) >> 8) & 0xFF;
+    __syncwarp();  // the previous packet's records have been read
+    if (staged) {
+      for (uint32_t w = lane; w < n_words; w += 32) sp[w] = ld_stream(pkt + w, pol);
+      __syncwarp();
+    }
+    auto word = [&](uint32_t i) -> uint32_t { return staged ? sp[i] : ld_stream(pkt + i, pol); };
+    const uint32_t w0 = word(0), w1 = word(1), w2 = word(2);
+    const uint32_t ps = w0 & 0xFF, y = (w0 >> 8) & 0xFF;
     if (ps != s || y < 1 || y > CVLC_MAX_CODE_BITS || y > y_prev) {  // lengths never increase along a stream
       if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
       continue;
@@ -194,11 +206,11 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
       const uint32_t bit = H + j * wd;
       const uint32_t wi = bit >> 5, sh = bit & 31;
       // a record of up to 63 bits starting at bit sh of word wi spans at most three words
-      const unsigned long long a = ld_stream(pkt + wi, pol);
-      const unsigned long long b = (wi + 1 < n_words) ? ld_stream(pkt + wi + 1, pol) : 0u;
+      const unsigned long long a = word(wi);
+      const unsigned long long b = (wi + 1 < n_words) ? word(wi + 1) : 0u;
       unsigned long long rec = (a | (b << 32)) >> sh;
       if (sh + wd > 64) {
-        const unsigned long long c2 = (wi + 2 < n_words) ? ld_stream(pkt + wi + 2, pol) : 0u;
+        const unsigned long long c2 = (wi + 2 < n_words) ? word(wi + 2) : 0u;
         rec |= c2 << (64 - sh);
       }
       const unsigned long long pid = rec & pid_mask;

@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per client and launch from the committed ncu capture
 # (profiles/: resnet18 shape, 2 bits per coordinate, PQ, 8 clients) of the kernels whose traffic grows in
 # proportion to the client count; scaled to the clients of a launch, None for any other configuration.
-NCU_TRAFFIC_BYTES_PER_CLIENT = {"k_select": (358.73e6 + 28.07e6) / 8, "k_hist": (358.52e6 + 5.15e6) / 8}
+NCU_TRAFFIC_BYTES_PER_CLIENT = {"k_select": (358.79e6 + 27.71e6) / 8, "k_hist": (358.52e6 + 5.20e6) / 8}
 
 
 def parse_args():

@@ -285,8 +285,8 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
   if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
   const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
   if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
-  // a packet is assembled in shared memory (QSGD: next to the squares of its values)
-  if ((size_t)S.packet_bits / 8 + 16 + (S.quantizer == CVLC_QUANT_QSGD ? (size_t)S.cap[1] * 8 : 0) > 200 * 1024) return CVLC_ERR_INVALID_ARG;
+  // four packets at a time are assembled in shared memory (QSGD: each next to the squares of its values)
+  if (4 * ((size_t)S.packet_bits / 8 + 16 + (S.quantizer == CVLC_QUANT_QSGD ? (size_t)S.cap[1] * 8 : 0)) > 200 * 1024) return CVLC_ERR_INVALID_ARG;
   if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
   return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
                                                                                                        : CVLC_ERR_CUDA;

@@ -867,22 +867,22 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 // ===================================================================================
 // K5  per-packet centroid distribution (PQ: min/max; QSGD: l2-norm), stochastic quantization, bit packing
 // ===================================================================================
-// One CTA works through kPackGroup consecutive packets of one client.  Packet r (longest codes first) holds
-// ranks [Z, Z + cap(y_r)).  The packet is assembled in shared memory: every record ORs its bits into the
-// (at most three) 32-bit words it touches, then the words go out with consecutive addresses.  The ranked
-// pairs are read twice from global memory (statistics, then quantization); the second read hits in cache.
+// One warp works through kPackGroup consecutive packets of one client, without block-wide barriers.  Packet r
+// (longest codes first) holds ranks [Z, Z + cap(y_r)).  The packet is assembled in the warp's shared-memory
+// buffer: every record ORs its bits into the (at most three) 32-bit words it touches, then the words go out with
+// consecutive addresses.  The ranked pairs are read twice from global memory (statistics, then quantization);
+// the second read hits in cache.  A lane quantizes about twelve records of a packet: twelve independent Philox
+// chains in flight.
 
 constexpr int kPackThreads = 128;
-constexpr int kPackGroup = 4;  // packets per CTA: the length table is set up once for all of them
+constexpr int kPackWarps = kPackThreads / 32;
+constexpr int kPackGroup = 4;  // packets per warp: the length table is set up once for all of them
 
 template <int CAP, bool QSGD>
 __global__ void __launch_bounds__(kPackThreads)
 k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
-       const __grid_constant__ EncLayout L) {
-  extern __shared__ __align__(16) unsigned char s_pack[];  // packet words; QSGD: then cap(1) squares
-  __shared__ float s_red[2][kPackThreads / 32];
-  __shared__ uint32_t s_y;
-  __shared__ unsigned long long s_Z;
+       const __grid_constant__ EncLayout L, uint32_t warp_bytes) {
+  extern __shared__ __align__(16) unsigned char s_pack[];  // per warp: packet words; QSGD: then cap(1) squares
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
   if (hdr->status != 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -892,7 +892,8 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   const uint32_t s = shape.s;
   const uint32_t H = shape.header_bits;
   const uint32_t n_words = shape.packet_bits / 32;
-  uint32_t* words = reinterpret_cast<uint32_t*>(s_pack);
+  unsigned char* s_mine = s_pack + (size_t)warp * warp_bytes;
+  uint32_t* words = reinterpret_cast<uint32_t*>(s_mine);
   uint32_t* stream_words = reinterpret_cast<uint32_t*>(cd.stream);
 
   const uint32_t mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask)[c];
@@ -900,50 +901,38 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   const unsigned long long* __restrict__ sorted =
       reinterpret_cast<const unsigned long long*>(ws + ((flips & 1) ? L.off_buf_b : L.off_buf_a)) + (size_t)c * L.capacity;
 
-  // packet -> its code length and first rank: lane l of warp 0 holds length 32 - l (longest first) with the
+  // packet -> its code length and first rank: lane l holds length 32 - l (longest first) with the
   // inclusive sums of packets and of records up to and including that length
-  uint32_t yl = 0, ny = 0, cum = 0, capl = 0;
-  unsigned long long zc = 0, nz = 0;
-  if (warp == 0) {
-    yl = CVLC_MAX_CODE_BITS - lane;
-    ny = plan->n_y[yl];
-    capl = plan->cap[yl];
-    nz = (unsigned long long)ny * capl;
-    cum = ny;
-    zc = nz;
+  const uint32_t yl = CVLC_MAX_CODE_BITS - lane;
+  const uint32_t ny = plan->n_y[yl];
+  const uint32_t capl = plan->cap[yl];
+  const unsigned long long nz = (unsigned long long)ny * capl;
+  uint32_t cum = ny;
+  unsigned long long zc = nz;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t a = __shfl_up_sync(kFull, cum, off);
-      const unsigned long long b = __shfl_up_sync(kFull, zc, off);
-      if (lane >= off) {
-        cum += a;
-        zc += b;
-      }
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t a = __shfl_up_sync(kFull, cum, off);
+    const unsigned long long b = __shfl_up_sync(kFull, zc, off);
+    if (lane >= off) {
+      cum += a;
+      zc += b;
     }
   }
 
   for (int g = 0; g < kPackGroup; ++g) {
-    const uint32_t r = blockIdx.x * kPackGroup + g;
+    const uint32_t r = (blockIdx.x * kPackWarps + warp) * kPackGroup + g;
     if (r >= shape.R) break;
-    if (warp == 0) {
-      const unsigned hit = __ballot_sync(kFull, r < cum);
-      if (hit == 0) {
-        if (lane == 0) s_y = 0;
-      } else if (lane == __ffs(hit) - 1) {
-        s_y = yl;
-        s_Z = (zc - nz) + (unsigned long long)(r - (cum - ny)) * capl;
-      }
-    }
-    for (uint32_t w = tid; w < n_words; w += kPackThreads) words[w] = 0u;
-    __syncthreads();
-    const uint32_t y = s_y;
-    if (y == 0) break;  // fewer packets planned than the stream holds: caught by the plan check
-    const unsigned long long Z = s_Z;
-    const uint32_t P = plan->cap[y];
+    const unsigned hit = __ballot_sync(kFull, r < cum);
+    if (hit == 0) break;  // fewer packets planned than the stream holds: caught by the plan check
+    const int src_lane = __ffs(hit) - 1;
+    const uint32_t y = CVLC_MAX_CODE_BITS - (uint32_t)src_lane;
+    const unsigned long long Z = __shfl_sync(kFull, (zc - nz) + (unsigned long long)(r - (cum - ny)) * capl, src_lane);
+    const uint32_t P = __shfl_sync(kFull, capl, src_lane);
+    for (uint32_t w = lane; w < n_words; w += 32) words[w] = 0u;
+    __syncwarp();
     const uint32_t wd = s + y;
     const unsigned long long* __restrict__ seg = sorted + Z;
     float lo, hi;  // the header's two centroid fields
-
     // a record's bits, low bit first from packet bit H + j * wd
     auto put = [&](uint32_t j, unsigned long long rec) {
       const uint32_t bitpos = H + j * wd;
@@ -958,15 +947,15 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
 
     if constexpr (QSGD) {
       // ---- QSGD: |x| against the packet's l2-norm; code = sign bit above a level of s_q = 2^(y-1) - 1 steps ----
-      __shared__ float s_norm;
-      double* sqv = reinterpret_cast<double*>(s_pack + (((size_t)n_words * 4 + 15) & ~(size_t)15));
-      for (uint32_t j = tid; j < P; j += kPackThreads) {
+      double* sqv = reinterpret_cast<double*>(s_mine + (((size_t)n_words * 4 + 15) & ~(size_t)15));
+      for (uint32_t j = lane; j < P; j += 32) {
         const double a = (double)__uint_as_float((uint32_t)(seg[j] >> 32));
         sqv[j] = __dmul_rn(a, a);  // exact: 24 x 24 bits
       }
-      __syncthreads();
-      // the norm is defined with the squares added in rank order in double: one thread walks the chain
-      if (tid == 0) {
+      __syncwarp();
+      // the norm is defined with the squares added in rank order in double: one lane walks the chain
+      float norm = 0.0f;
+      if (lane == 0) {
         double sum = 0.0;
         uint32_t j = 0;
         for (; j + 8 <= P; j += 8) {
@@ -978,17 +967,16 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         }
         for (; j < P; ++j) sum = __dadd_rn(sum, sqv[j]);
         const double rt = __dsqrt_rn(sum);
-        s_norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
+        norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
       }
-      __syncthreads();
-      const float norm = s_norm;
+      norm = __shfl_sync(kFull, norm, 0);
       lo = norm;
       hi = 0.0f;
       const uint32_t sq = (uint32_t)((1ull << (y - 1)) - 1ull);  // y >= 2: checked with the plan
       const double sqd = (double)sq;
       const double dn = (double)norm;
       const double scale = (norm > 0.0f) ? __ddiv_rn(sqd, dn) : 0.0;
-      for (uint32_t j = tid; j < P; j += kPackThreads) {
+      for (uint32_t j = lane; j < P; j += 32) {
         const unsigned long long pair = seg[j];
         const uint32_t key = (uint32_t)(pair >> 32);
         const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
@@ -1020,7 +1008,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     } else {
       // ---- PQ: minimum / maximum of the packet's signed values (its centroid distribution) ----
       float vmin = CUDART_INF_F, vmax = -CUDART_INF_F;
-      for (uint32_t j = tid; j < P; j += kPackThreads) {
+      for (uint32_t j = lane; j < P; j += 32) {
         const unsigned long long pair = seg[j];
         const uint32_t key = (uint32_t)(pair >> 32);
         const uint32_t b = key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u;  // -0 is stored as +0
@@ -1033,25 +1021,15 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         vmin = fminf(vmin, __shfl_xor_sync(kFull, vmin, off));
         vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, off));
       }
-      if (lane == 0) {
-        s_red[0][warp] = vmin;
-        s_red[1][warp] = vmax;
-      }
-      __syncthreads();
-      lo = s_red[0][0];
-      hi = s_red[1][0];
-#pragma unroll
-      for (int w = 1; w < kPackThreads / 32; ++w) {
-        lo = fminf(lo, s_red[0][w]);
-        hi = fmaxf(hi, s_red[1][w]);
-      }
+      lo = vmin;
+      hi = vmax;
 
       // stochastic rounding onto the 2^y uniform centroids of [lo, hi]
       const double Lc = (double)((1ull << y) - 1ull);
       const double dlo = (double)lo;
       const double den = __dsub_rn((double)hi, dlo);
       const double scale = (hi != lo) ? __ddiv_rn(Lc, den) : 0.0;
-      for (uint32_t j = tid; j < P; j += kPackThreads) {
+      for (uint32_t j = lane; j < P; j += 32) {
         const unsigned long long pair = seg[j];
         const uint32_t key = (uint32_t)(pair >> 32);
         const uint32_t pid = (uint32_t)pair & 0x7FFFFFFFu;
@@ -1082,16 +1060,16 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     }  // PQ
 
     // packet header {s, y, lo, hi} in bits 0..79 (bits 80..H-1 stay zero)
-    if (tid == 0) {
+    if (lane == 0) {
       const uint32_t blo = __float_as_uint(lo), bhi = __float_as_uint(hi);
       atomicOr(words + 0, s | (y << 8) | (blo << 16));
       atomicOr(words + 1, (blo >> 16) | (bhi << 16));
       atomicOr(words + 2, bhi >> 16);
     }
-    __syncthreads();
+    __syncwarp();
     uint32_t* pkt = stream_words + CVLC_STREAM_HEADER_BYTES / 4 + (size_t)r * n_words;
-    for (uint32_t w = tid; w < n_words; w += kPackThreads) pkt[w] = words[w];
-    __syncthreads();  // the word buffer (and s_y, s_Z, s_red) are reused by the next packet
+    for (uint32_t w = lane; w < n_words; w += 32) pkt[w] = words[w];
+    __syncwarp();  // the word buffer is reused by the next packet
   }
 
   // global header (64 bytes), written once per client
@@ -1151,7 +1129,9 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   unsigned char* w = static_cast<unsigned char*>(ws);
   const bool qsgd = shape.quantizer == CVLC_QUANT_QSGD;
   // packet words; QSGD: and the squares of a packet's values
-  const size_t pack_smem = (((size_t)shape.packet_bits / 8 + 15) & ~(size_t)15) + (qsgd ? (size_t)shape.cap[1] * 8 : 0);
+  const size_t pack_warp = (((size_t)shape.packet_bits / 8 + 15) & ~(size_t)15) + (qsgd ? (size_t)shape.cap[1] * 8 : 0);
+  const size_t pack_smem = pack_warp * kPackWarps;
+  const unsigned pack_grid = (shape.R + kPackWarps * kPackGroup - 1) / (kPackWarps * kPackGroup);
 
   const Partition part = make_partition(shape.d, n);
   const unsigned char* pws = static_cast<const unsigned char*>(plan_ws);
@@ -1187,9 +1167,9 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   {
     LaunchScope ls(kKPack, st);
     if (qsgd)
-      k_pack<CAP, true><<<dim3((shape.R + kPackGroup - 1) / kPackGroup, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+      k_pack<CAP, true><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp);
     else
-      k_pack<CAP, false><<<dim3((shape.R + kPackGroup - 1) / kPackGroup, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L);
+      k_pack<CAP, false><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp);
   }
   return cudaGetLastError();
 }

@@ -370,8 +370,9 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const uint64_t n_vec = (v_end > u0) ? v_end - u0 : 0;        // float4 units of the segment
     const uint32_t n_tiles = (uint32_t)((n_vec + kTileVec - 1) / kTileVec);
 
-    // copies of a warp are consecutive float4s (coalesced); any thread may stage any unit because a
-    // barrier separates the wait for a tile from its use
+    // A warp stages exactly the 128 units (512 coordinates) its own lanes will read: four copies of 32
+    // consecutive float4s each (coalesced).  Waiting for a tile and reusing a staging slot are then a matter
+    // between the lanes of one warp, and the block meets only once per tile, for the scan.
     uint32_t istage = 0;
     auto issue = [&](uint32_t t) {
       if (t < n_tiles) {
@@ -380,13 +381,13 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         if (base + kTileVec <= n_vec) {
 #pragma unroll
           for (int v = 0; v < kSelVec; ++v) {
-            const uint32_t g = v * kSelThreads + tid;
+            const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
             cp_async16(dst + sel_slot(g), xseg + base + g);
           }
         } else {
 #pragma unroll
           for (int v = 0; v < kSelVec; ++v) {
-            const uint32_t g = v * kSelThreads + tid;
+            const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
             if (base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
           }
         }
@@ -399,8 +400,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     for (int t = 0; t < kSelStages - 1; ++t) issue(t);
     uint32_t stage = 0;
     for (uint32_t t = 0; t < n_tiles; ++t) {
-      cp_async_wait<kSelStages - 2>();  // this thread's copies of tile t have landed
-      __syncthreads();                  // ... and everybody else's; and everybody is done with tile t - 1,
+      cp_async_wait<kSelStages - 2>();  // this lane's copies of tile t have landed
+      __syncwarp();                     // ... and the other lanes'; and the warp is done with its part of tile t - 1,
       issue(t + kSelStages - 1);        // whose staging slot the next copies overwrite
       const float4* src = s_stage + (size_t)stage * kTileVec;
       stage = (stage + 1 == kSelStages) ? 0u : stage + 1;
@@ -876,7 +877,7 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
 
 constexpr int kPackThreads = 128;
 constexpr int kPackWarps = kPackThreads / 32;
-constexpr int kPackGroup = 4;  // packets per warp: the length table is set up once for all of them
+constexpr int kPackGroup = 1;  // packets per warp (more of them amortise the length table but lengthen the tail)
 
 template <int CAP, bool QSGD>
 __global__ void __launch_bounds__(kPackThreads)

@@ -34,11 +34,16 @@ METRIC = "encode+decode_aggregate throughput (4*d*clients / step time)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per client and launch from the committed ncu capture
-# (profiles/: resnet18 shape, 2 bits per coordinate, PQ, 8 clients) of the kernels whose traffic grows in
-# proportion to the client count; scaled to the clients of a launch, None for any other configuration.
-NCU_TRAFFIC_BYTES_PER_CLIENT = {"k_select": (358.79e6 + 27.71e6) / 8, "k_hist": (358.52e6 + 5.20e6) / 8}
-
+# dram__bytes_read.sum + dram__bytes_write.sum per client and launch from the committed ncu captures
+# (profiles/: resnet18 shape, 2 bits per coordinate, PQ; 32 clients, k_hist 8 clients) of the kernels whose
+# traffic grows in proportion to the client count once their working set is beyond the L2; scaled to the
+# clients of a launch, None for any other configuration or fewer than 32 clients per launch.  k_sort_pass:
+# mean over the four launches of a step (three move data, one is skipped on the device).
+NCU_TRAFFIC_BYTES_PER_CLIENT = {
+    "k_select": (1435.80e6 + 169.71e6) / 32,
+    "k_sort_pass": (190.46e6 + 158.26e6 + 193.54e6 + 158.31e6 + 189.75e6 + 158.28e6 + 0.07e6) / 32 / 4,
+    "k_hist": (358.52e6 + 5.28e6) / 8,
+}
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -359,7 +364,7 @@ def run_ours(args):
         if dominant in alg_bytes_per_step:
             per_launch = alg_bytes_per_step[dominant] * args.steps / kn
             captured = (w.name == "resnet18" and d == w.d and bpc == 2.0 and args.quantizer == "pq"
-                        and dominant in NCU_TRAFFIC_BYTES_PER_CLIENT)
+                        and dominant in NCU_TRAFFIC_BYTES_PER_CLIENT and n_clients / n_groups >= 32)
             ncu_traffic = NCU_TRAFFIC_BYTES_PER_CLIENT[dominant] * n_clients / n_groups if captured else None
             achieved = per_launch / (kms / kn * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak,

@@ -13,7 +13,8 @@
  *
  * Parity pins (see tests, "-m 'not gpu'"): every exported function is checked
  * against something other than itself; none is "parity unpinned".  The literal
- * real-valued form of Algorithm 1 (enumerating every k) is not built here.
+ * real-valued form of Algorithm 1 is not built here; the tests restate it in Python
+ * on small instances as one of the pins of the length tuning.
  */
 #ifndef CVLC_ORACLE_H
 #define CVLC_ORACLE_H

@@ -136,9 +136,17 @@ __device__ __forceinline__ double series_exp2(double v) {
   const double n = floor(__dadd_rn(v, 0.5));
   const double r = __dsub_rn(v, n);
   const double u = __dmul_rn(r, 0.6931471805599453);
+  // u / j for j = 1 .. 20: a division by an odd j is done once, the even ones are its exact halvings
+  // (RN(u / 2j) = RN(u / j) / 2: scaling by two commutes with rounding; u is zero or far above the subnormals)
+  double uj[21];
+  uj[1] = u;
+#pragma unroll
+  for (int j = 3; j <= 19; j += 2) uj[j] = div_small_int(u, j);
+#pragma unroll
+  for (int j = 2; j <= 20; j += 2) uj[j] = __dmul_rn(uj[j / 2], 0.5);
   double p = 1.0;
 #pragma unroll
-  for (int j = 20; j >= 1; --j) p = __dadd_rn(1.0, __dmul_rn(div_small_int(u, j), p));
+  for (int j = 20; j >= 1; --j) p = __dadd_rn(1.0, __dmul_rn(uj[j], p));
   const long long ni = (long long)n;
   return __longlong_as_double(__double_as_longlong(p) + ni * (1ll << 52));
 }
@@ -530,13 +538,23 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                 const uint32_t span = (mine && Q.op[lane].lo < Q.op[lane].hi) ? Q.op[lane].hi - Q.op[lane].lo : 0u;
                 const int need_levels = span ? 32 - __clz(span) : 0;  // a bisection of s points takes at most floor(log2 s) + 1 steps
                 const int m_op = mine ? Q.op[lane].m : 0;
-                int depth = 0;
-                for (int cand = 1; cand <= 9; ++cand) {
-                  const int lv = need_levels < cand ? need_levels : cand;
-                  int items = lv ? 2 * ((1 << lv) - 1) * m_op : 0;
+                // items of the whole batch at every candidate depth: nine reductions side by side (one after the
+                // other they are nine chains of five dependent shuffles, as long as the energy evaluation itself)
+                int items_at[9];
 #pragma unroll
-                  for (int off = 16; off > 0; off >>= 1) items += __shfl_xor_sync(kFull, items, off);
-                  if (items <= kPlanThreads) depth = cand; else break;
+                for (int cand = 1; cand <= 9; ++cand) {
+                  const int lvc = need_levels < cand ? need_levels : cand;
+                  items_at[cand - 1] = lvc ? 2 * ((1 << lvc) - 1) * m_op : 0;
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+                  for (int q = 0; q < 9; ++q) items_at[q] += __shfl_xor_sync(kFull, items_at[q], off);
+                }
+                int depth = 0;
+#pragma unroll
+                for (int q = 0; q < 9; ++q) {
+                  if (items_at[q] <= kPlanThreads && depth == q) depth = q + 1;  // the sums grow with the depth
                 }
                 const int lv = need_levels < depth ? need_levels : depth;
                 const int ne = lv ? 2 * ((1 << lv) - 1) : 0;

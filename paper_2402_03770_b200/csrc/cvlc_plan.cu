@@ -192,6 +192,9 @@ struct PlanSolver {
   int eval_end[kMaxBatchOps];
   int n_ops, n_items, n_evals, unfinished;
   int next_i, next_j, moved;      // where the sweep resumes after the batch
+  uint32_t col_warp[32];          // batch collection: warp totals of the (operations, items) scan
+  int col_nops, col_last, col_first_left;  // operations taken; thread of the last one; thread of the first one left over
+  unsigned char ea[1024];         // operation of every evaluation
 };
 
 struct PlanShared {
@@ -493,27 +496,93 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
           int moved = 0;
           int ci = nY - 1, cj = nY - 2;  // cursor of the sweep
           while (ci >= 1) {
-            // ---- collect a batch (every thread computes the same list; thread 0 records it)
+            // ---- collect a batch: thread t looks at the t-th pair of the sweep from the cursor on (at most
+            // 31 + 465 pairs).  The batch is the first pairs, in sweep order, that share packets (X > 0), up to
+            // kMaxBatchOps of them and as long as two evaluations of each fit the block: a prefix of the flagged
+            // pairs, found with one block scan of (operations, items) packed in a word.
             {
-              int bi = ci, bj = cj, n_ops = 0, reserved = 0;
-              const unsigned used = Q.used;
-              while (bi >= 1 && n_ops < kMaxBatchOps) {
-                const uint32_t X = S.n[bi] + S.n[bj];
-                if (X > 0) {
-                  const unsigned need = (used | (1u << bi) | (1u << bj)) & (0xFFFFFFFFu >> (31 - bi));
-                  const int m = __popc(need);
-                  if (reserved + 2 * m > kPlanThreads) break;  // one level at least for every operation
-                  reserved += 2 * m;
-                  if (tid == 0) {
-                    PlanOp& o = Q.op[n_ops];
-                    o.i = bi; o.j = bj; o.X = X; o.na0 = S.n[bi]; o.lo = 0; o.hi = X; o.m = m; o.F_final = 0.0;
-                  }
-                  if (warp == n_ops && (need & (1u << lane)))
-                    Q.op[n_ops].slot_lane[lane == 31 ? 0 : __popc(need >> (lane + 1))] = (unsigned char)lane;
-                  ++n_ops;
+              auto pair_at = [&](int t, int& i, int& j) -> bool {
+                if (t < 0) return false;
+                if (phase == 0) {
+                  i = ci - t;
+                  j = i - 1;
+                  return i >= 1;
                 }
-                next_pair(phase, bi, bj);
+                const int first = cj + 1;  // rest of the cursor's row: j = cj .. 0
+                if (t < first) {
+                  i = ci;
+                  j = cj - t;
+                  return true;
+                }
+                const int rest = (ci - 1) * ci / 2;  // rows ci - 1 .. 1, row r holding the pairs (r, r-1) .. (r, 0)
+                const int tp = t - first;
+                if (tp >= rest) return false;
+                const int u = rest - 1 - tp;  // counted upwards from pair (1, 0)
+                int r = 1;
+                while ((r * (r + 1)) / 2 <= u) ++r;
+                i = r;
+                j = u - (r - 1) * r / 2;
+                return true;
+              };
+              const unsigned used = Q.used;
+              int pi = 0, pj = 0;
+              const bool valid = pair_at(tid, pi, pj);
+              uint32_t X = 0;
+              unsigned need = 0;
+              int m = 0;
+              if (valid) {
+                X = S.n[pi] + S.n[pj];
+                if (X > 0) {
+                  need = (used | (1u << pi) | (1u << pj)) & (0xFFFFFFFFu >> (31 - pi));
+                  m = __popc(need);
+                }
               }
+              const bool flag = valid && X > 0;
+              uint32_t incl = flag ? ((1u << 16) | (uint32_t)(2 * m)) : 0u;  // items stay below 2^16: 496 pairs of at most 64
+#pragma unroll
+              for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_up_sync(kFull, incl, off);
+                if (lane >= off) incl += o;
+              }
+              if (lane == 31) Q.col_warp[warp] = incl;
+              if (tid == 0) {
+                Q.col_nops = 0;
+                Q.col_last = -1;
+                Q.col_first_left = 0x7FFFFFFF;
+              }
+              __syncthreads();
+              {
+                const uint32_t wt = Q.col_warp[lane];
+                uint32_t wi = wt;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                  const uint32_t o = __shfl_up_sync(kFull, wi, off);
+                  if (lane >= off) wi += o;
+                }
+                incl += __shfl_sync(kFull, wi - wt, warp);
+              }
+              const int rank = (int)(incl >> 16) - 1;
+              const bool taken = flag && rank < kMaxBatchOps && (incl & 0xFFFFu) <= (uint32_t)kPlanThreads;
+              if (taken) {
+                PlanOp& o = Q.op[rank];
+                o.i = pi; o.j = pj; o.X = X; o.na0 = S.n[pi]; o.lo = 0; o.hi = X; o.m = m; o.F_final = 0.0;
+                for (unsigned rest_bits = need; rest_bits;) {  // the lengths a trial evaluates, longest first
+                  const int l = 31 - __clz(rest_bits);
+                  rest_bits ^= 1u << l;
+                  o.slot_lane[l == 31 ? 0 : __popc(need >> (l + 1))] = (unsigned char)l;
+                }
+                atomicMax(&Q.col_nops, rank + 1);
+                atomicMax(&Q.col_last, tid);
+              } else if (flag) {
+                atomicMin(&Q.col_first_left, tid);
+              }
+              __syncthreads();
+              const int n_ops = Q.col_nops;
+              // the sweep resumes after the last operation of a full batch, else at the first pair left over
+              const int resume = (n_ops == kMaxBatchOps) ? Q.col_last + 1
+                                                         : (Q.col_first_left != 0x7FFFFFFF ? Q.col_first_left : -1);
+              int bi = 0, bj = 0;
+              if (!pair_at(resume, bi, bj)) bi = bj = 0;
               if (tid == 0) {
                 Q.n_ops = n_ops;
                 Q.next_i = bi;
@@ -523,7 +592,10 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
               }
               ci = bi;
               cj = bj;
-              if (n_ops == 0) continue;  // the rest of the sweep had nothing to split
+              if (n_ops == 0) {  // the rest of the sweep had nothing to split
+                __syncthreads();  // the collection's scratch is reset by the next one
+                continue;
+              }
             }
             __syncthreads();
             const int n_ops = Q.n_ops;
@@ -616,7 +688,10 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   if (l <= o.j) W = W - (uint64_t)S.n[o.j] * T.capY[o.j] + (uint64_t)(o.X - t) * T.capY[o.j];
                   Q.Ev[tid] = energy_E(W, beta, D);
                 }
-                if (sl == 0) Q.tv[o.eval_base + e] = t;
+                if (sl == 0) {
+                  Q.tv[o.eval_base + e] = t;
+                  Q.ea[o.eval_base + e] = (unsigned char)a;
+                }
               }
               __syncthreads();
               // phase 2: the terms g_l * (E_l - E_prev); only the lengths i and j can be unused in a trial
@@ -639,21 +714,31 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
               __syncthreads();
               // phase 3: one thread per evaluation continues the running sum below length i
               if (tid < Q.n_evals) {
-                int lo_a = 0, hi_a = 31;
-                while (lo_a < hi_a) {
-                  const int mid = (lo_a + hi_a) >> 1;
-                  if (tid < Q.eval_end[mid]) hi_a = mid; else lo_a = mid + 1;
-                }
-                const PlanOp& o = Q.op[lo_a];
+                const PlanOp& o = Q.op[Q.ea[tid]];
                 const uint32_t tt = Q.tv[tid];
                 if (tt != 0xFFFFFFFFu) {
                   const int ee = tid - o.eval_base;
                   const double* tm = Q.term + o.item_base + ee * o.m;
                   double F = Q.Fpre[o.i + 1];
-                  for (int z = 0; z < o.m; ++z) {
-                    const int l = o.slot_lane[z];
-                    const uint32_t nn = (l == o.i) ? tt : (l == o.j) ? (o.X - tt) : 1u;
-                    if (nn > 0) F = __dadd_rn(F, tm[z]);
+                  // the terms are added in the order of the lengths; four are fetched ahead of the additions
+                  for (int z0 = 0; z0 < o.m; z0 += 4) {
+                    double tv4[4];
+                    bool on4[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                      const int z = z0 + q;
+                      on4[q] = false;
+                      tv4[q] = 0.0;
+                      if (z < o.m) {
+                        const int l = o.slot_lane[z];
+                        const uint32_t nn = (l == o.i) ? tt : (l == o.j) ? (o.X - tt) : 1u;
+                        on4[q] = nn > 0;
+                        tv4[q] = tm[z];
+                      }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                      if (on4[q]) F = __dadd_rn(F, tv4[q]);
                   }
                   const uint64_t Wtot = Q.Wc[0] - (uint64_t)S.n[o.i] * T.capY[o.i] - (uint64_t)S.n[o.j] * T.capY[o.j] +
                                         (uint64_t)tt * T.capY[o.i] + (uint64_t)(o.X - tt) * T.capY[o.j];

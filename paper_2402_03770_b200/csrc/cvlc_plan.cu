@@ -184,7 +184,6 @@ struct PlanSolver {
   unsigned long long Wc[32];      // ranks covered by lengths >= l, current counts
   unsigned used;                  // lengths with a positive count
   double Ev[1024];                // trial energies, one per item
-  double term[1024];              // g_l * (E - E_prev) of every used item
   double Fv[1024];                // trial objective values, one per evaluation
   uint32_t tv[1024];              // trial split of every evaluation (0xFFFFFFFF: not needed)
   PlanOp op[kMaxBatchOps];
@@ -694,51 +693,40 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                 }
               }
               __syncthreads();
-              // phase 2: the terms g_l * (E_l - E_prev); only the lengths i and j can be unused in a trial
-              if (a >= 0 && t != 0xFFFFFFFFu) {
-                const PlanOp& o = Q.op[a];
-                const int l = o.slot_lane[sl];
-                const uint32_t nn = (l == o.i) ? t : (l == o.j) ? (o.X - t) : 1u;
-                if (nn > 0) {
-                  int p = sl - 1;
-                  while (p >= 0) {
-                    const int lp = o.slot_lane[p];
-                    const uint32_t np = (lp == o.i) ? t : (lp == o.j) ? (o.X - t) : 1u;
-                    if (np > 0) break;
-                    --p;
-                  }
-                  const double Eprev = (p >= 0) ? Q.Ev[tid - sl + p] : Q.Eab[o.i + 1];
-                  Q.term[tid] = __dmul_rn(T.gY[l], __dsub_rn(Q.Ev[tid], Eprev));
-                }
-              }
-              __syncthreads();
-              // phase 3: one thread per evaluation continues the running sum below length i
+              // phase 2: one thread per evaluation continues the running sum below length i with the terms
+              // g_l * (E_l - E_prev) in the order of the lengths; only the lengths i and j can be unused in a trial
+              // (no term, and the next term's E_prev skips them).  The terms do not depend on the sum, so they are
+              // worked out four at a time ahead of the ordered additions.
               if (tid < Q.n_evals) {
                 const PlanOp& o = Q.op[Q.ea[tid]];
                 const uint32_t tt = Q.tv[tid];
                 if (tt != 0xFFFFFFFFu) {
                   const int ee = tid - o.eval_base;
-                  const double* tm = Q.term + o.item_base + ee * o.m;
+                  const double* Ez = Q.Ev + o.item_base + ee * o.m;
                   double F = Q.Fpre[o.i + 1];
-                  // the terms are added in the order of the lengths; four are fetched ahead of the additions
+                  double Eprev = Q.Eab[o.i + 1];
                   for (int z0 = 0; z0 < o.m; z0 += 4) {
-                    double tv4[4];
+                    double term4[4];
                     bool on4[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                       const int z = z0 + q;
                       on4[q] = false;
-                      tv4[q] = 0.0;
+                      term4[q] = 0.0;
                       if (z < o.m) {
                         const int l = o.slot_lane[z];
                         const uint32_t nn = (l == o.i) ? tt : (l == o.j) ? (o.X - tt) : 1u;
-                        on4[q] = nn > 0;
-                        tv4[q] = tm[z];
+                        if (nn > 0) {
+                          const double Ec = Ez[z];
+                          on4[q] = true;
+                          term4[q] = __dmul_rn(T.gY[l], __dsub_rn(Ec, Eprev));
+                          Eprev = Ec;
+                        }
                       }
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
-                      if (on4[q]) F = __dadd_rn(F, tv4[q]);
+                      if (on4[q]) F = __dadd_rn(F, term4[q]);
                   }
                   const uint64_t Wtot = Q.Wc[0] - (uint64_t)S.n[o.i] * T.capY[o.i] - (uint64_t)S.n[o.j] * T.capY[o.j] +
                                         (uint64_t)tt * T.capY[o.i] + (uint64_t)(o.X - tt) * T.capY[o.j];

@@ -600,11 +600,11 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
             const int n_ops = Q.n_ops;
             const double F_cur = Q.Fpre[0];
             // ---- rounds until every operation of the batch has finished its bisection
-            while (true) {
-              // level assignment (warp 0, lane = operation): the planner is bound by the FP64 throughput
-              // of its SM, and every extra level evaluated ahead doubles the work, so all operations get
-              // the same small depth: the largest one whose items fit the block
-              if (warp == 0) {
+            // level assignment (warp 0, lane = operation), before the first round and right after every tree walk:
+            // the planner is bound by the FP64 throughput
+            // of its SM, and every extra level evaluated ahead doubles the work, so all operations get
+            // the same small depth: the largest one whose items fit the block
+            auto assign_levels = [&]() {
                 const bool mine = lane < n_ops;
                 const uint32_t span = (mine && Q.op[lane].lo < Q.op[lane].hi) ? Q.op[lane].hi - Q.op[lane].lo : 0u;
                 const int need_levels = span ? 32 - __clz(span) : 0;  // a bisection of s points takes at most floor(log2 s) + 1 steps
@@ -651,7 +651,9 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   Q.n_evals = evals_incl;
                   Q.unfinished = __popc(unfinished);
                 }
-              }
+                          };
+            if (warp == 0) assign_levels();
+            while (true) {
               __syncthreads();
               if (Q.unfinished == 0) break;
               // phase 1: energies, one thread per (operation, evaluation, slot)
@@ -759,7 +761,10 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   o.F_final = Ff;
                 }
               }
-              __syncthreads();
+              if (warp == 0) {  // the lanes that walked the trees own the same operations in the level assignment
+                __syncwarp();
+                assign_levels();
+              }
             }
             // ---- the first operation of the batch that improves F is applied; the sweep resumes after it
             if (tid == 0) {

@@ -80,7 +80,9 @@ enum {
 typedef struct cvlc_params {
   uint64_t d;             /* coordinates, 2 <= d <= 2^31 */
   uint64_t budget_bits;   /* uplink budget of this client this round; R = floor(budget_bits / packet_bits) */
-  uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes) */
+  uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes).  cvlc_encode assembles four
+                             packets at a time in shared memory: 4 * (b / 8 + 16, plus 8 * cap(1) bytes with QSGD)
+                             must stay within 200 KB, else INVALID_ARG */
   uint32_t header_bits;   /* H; 80 <= H < b; 80 = s (8) + y_r (8) + min,max (64), Fig. 2 */
   uint32_t quantizer;     /* CVLC_QUANT_PQ or CVLC_QUANT_QSGD */
   uint32_t max_code_bits; /* 1..32 */
@@ -235,6 +237,9 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
  *  weight_total      0 = sum of this call's weights; otherwise the total over all
  *                    batches when the clients are fed in several calls
  *  out_dev           d fp32; overwritten when accumulate == 0, added to when 1
+ * A vector of more than 24 Mi coordinates is filled window by window (one pass over the
+ * streams per window) so that the additions stay in the L2 cache; the result does not
+ * depend on it.
  * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL (host); BAD_STREAM (device, at byte 0
  * of ws_dev).
  */

@@ -391,3 +391,29 @@ def test_plan_mismatch_is_detected(torch_cuda):
     assert B.cvlc_read_status(enc.enc_ws) in (B.CVLC_ERR_PLAN_MISMATCH, B.CVLC_OK)
     B.cvlc_encode(xd, p, enc.plan, enc.out, enc.enc_ws)                         # and the right pairing still works
     assert B.cvlc_read_status(enc.enc_ws) == B.CVLC_OK
+
+
+@pytest.mark.parametrize("quantizer", [0, 1])
+def test_large_packets_go_through_the_unstaged_paths(torch_cuda, quantizer):
+    # 8 KB packets: more records per packet than a warp's lanes many times over, a packet image of several KB per
+    # warp in the encoder, and packets too long for the decoder's shared-memory staging (read from global memory)
+    rng = np.random.default_rng(77)
+    d = 300_000
+    x = (rng.standard_t(3, d) * 1e-3).astype(np.float32)
+    pd = params_dict(d, 9 * 65536, packet_bits=65536, header_bits=80, quantizer=quantizer, seed=11, client_id=4)
+    of, ost = run_case(x, pd)
+    assert of["R"] == 9
+    ref = O.decode_aggregate([ost], np.array([2.0], np.float32), d, weight_total=5.0)
+    status, out = gpu_decode_aggregate([ost], np.array([2.0], np.float32), d, weight_total=5.0)
+    assert status == 0
+    assert_aggregate_close(out, ref)
+
+
+def test_packets_beyond_the_encoders_shared_memory_are_rejected(torch_cuda):
+    from paper_2402_03770_b200 import binding as B
+    d = 100_000
+    x = np.linspace(-1.0, 1.0, d).astype(np.float32)
+    pd = params_dict(d, 2 * 524288, packet_bits=524288, scale_B=2.0)   # 64 KB packets: four do not fit 200 KB
+    with pytest.raises(B.CvlcError) as e:
+        gpu_plan_encode(x, pd)
+    assert e.value.code == B.CVLC_ERR_INVALID_ARG

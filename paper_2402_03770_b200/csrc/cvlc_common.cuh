@@ -127,9 +127,9 @@ constexpr int kSelectVecPerThread = 4;                                 // float4
 constexpr int kSelectTile = kSelectThreads * kSelectVecPerThread * 4;  // 8192 coordinates
 
 constexpr int kSortThreads = 256;
-constexpr int kSortItemsPerThread = 16;  // 128 registers per thread hold a tile without spilling: two blocks per SM
+constexpr int kSortItemsPerThread = 20;  // 128 registers per thread hold a tile without spilling: two blocks per SM
 constexpr int kSortMinBlocks = 2;
-constexpr int kSortTile = kSortThreads * kSortItemsPerThread;  // 4096 pairs
+constexpr int kSortTile = kSortThreads * kSortItemsPerThread;  // 5120 pairs
 constexpr int kSortPasses = 4;                                 // digits of 9,9,9,4 bits
 constexpr int kDigitBits = 9;
 constexpr int kDigits = 1 << kDigitBits;                       // 512 digit values

@@ -849,10 +849,12 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
       auto prefetch_next = [&](uint32_t nt) {
         if (nt >= total_tickets) return;
         const uint32_t t2 = nt / n_clients, c2 = nt - t2 * n_clients;
-        const uint32_t line = t2 * (uint32_t)(kSortTile / 16) + tid;  // 128-byte lines of 16 items
-        if (tid < kSortTile / 16 && line * 16u < s_ncand[c2]) {
-          const unsigned long long* p = source(c2, s_mask[c2]) + (size_t)line * 16;
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+        for (uint32_t l = tid; l < (uint32_t)(kSortTile / 16); l += kSortThreads) {  // 128-byte lines of 16 items
+          const uint32_t line = t2 * (uint32_t)(kSortTile / 16) + l;
+          if (line * 16u < s_ncand[c2]) {
+            const unsigned long long* p = source(c2, s_mask[c2]) + (size_t)line * 16;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+          }
         }
       };
       if (count == (uint32_t)kSortTile)

@@ -40,9 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # clients of a launch, None for any other configuration or fewer than 32 clients per launch.  k_sort_pass:
 # mean over the four launches of a step (three move data, one is skipped on the device).
 NCU_TRAFFIC_BYTES_PER_CLIENT = {
-    "k_select": (1435.80e6 + 169.71e6) / 32,
-    "k_sort_pass": (190.46e6 + 158.26e6 + 193.54e6 + 158.31e6 + 189.75e6 + 158.28e6 + 0.07e6) / 32 / 4,
-    "k_hist": (358.52e6 + 5.28e6) / 8,
+    "k_select": (1435.81e6 + 169.36e6) / 32,
+    "k_sort_pass": (189.95e6 + 154.89e6 + 189.80e6 + 154.62e6 + 187.02e6 + 154.29e6 + 0.08e6) / 32 / 4,
+    "k_hist": (358.52e6 + 5.24e6) / 8,
 }
 
 def parse_args():

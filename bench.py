@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--d", type=int, default=0, help="0 = the workload's d (smaller values are for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="clients per plan/encode call; 0 = all clients in one call")
     ap.add_argument("--streams", type=int, default=2, help="CUDA streams the batches are spread over")
+    ap.add_argument("--no-side-stream", action="store_true",
+                    help="run the length tuning on the main stream instead of next to selection and ranking")
     ap.add_argument("--max-candidates", type=int, default=0,
                     help="candidate slots per client in the encode workspace; 0 = 3 * R * cap(1)")
     ap.add_argument("--profile-kernel", default="", help="kernel whose roofline is reported; default: the one with the largest total time")
@@ -220,6 +222,7 @@ def run_ours(args):
     groups = [list(range(i, min(i + batch, n_clients))) for i in range(0, n_clients, batch)]
     n_streams = max(1, min(args.streams, len(groups)))
     streams = [torch.cuda.Stream(device=dev) for _ in range(n_streams)]
+    side_streams = [None if args.no_side_stream else torch.cuda.Stream(device=dev) for _ in range(n_streams)]
     if args.max_candidates:
         max_cand = args.max_candidates
     else:
@@ -241,14 +244,15 @@ def run_ours(args):
         eb = max(1, min(args.e2e_batch, n_clients))
         e2e_groups = [list(range(i, min(i + eb, n_clients))) for i in range(0, n_clients, eb)]
         e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(max(1, min(args.e2e_streams, len(e2e_groups))))]
+        e2e_side = [None if args.no_side_stream else torch.cuda.Stream(device=dev) for _ in e2e_streams]
         e2e_encoders = [B.BatchEncoder([params[c] for c in g], dev, max_candidates=max_cand) for g in e2e_groups]
         e2e_agg = B.Aggregator(n_clients, d, dev)
         e2e_agg.set_clients([o for enc in e2e_encoders for o in enc.outs], weights)
         e2e_done = [torch.cuda.Event() for _ in e2e_streams]
 
     def step(from_host: bool):
-        g_list, s_list, e_list, a, dn = (e2e_groups, e2e_streams, e2e_encoders, e2e_agg, e2e_done) if from_host else \
-            (groups, streams, encoders, agg, done)
+        g_list, s_list, e_list, a, dn, sd = (e2e_groups, e2e_streams, e2e_encoders, e2e_agg, e2e_done, e2e_side) if from_host else \
+            (groups, streams, encoders, agg, done, side_streams)
         fork.record(main)
         for s in s_list:
             s.wait_event(fork)
@@ -258,7 +262,7 @@ def run_ours(args):
                 with torch.cuda.stream(s):
                     for c in g:
                         dev_x[c].copy_(pinned[c], non_blocking=True)
-            e_list[gi].run([dev_x[c] for c in g], stream=s)
+            e_list[gi].compress([dev_x[c] for c in g], stream=s, side_stream=sd[gi % len(s_list)])
         for s, e in zip(s_list, dn):
             e.record(s)
             main.wait_event(e)
@@ -407,7 +411,8 @@ def run_ours(args):
         "plan_of_client_0": {"k": int(plans[0].k), "R": int(plans[0].R), "n_candidates": int(plans[0].n_candidates), "alpha_q": plans[0].alpha_q,
                  "lengths": {str(y): int(plans[0].n_y[y]) for y in range(33) if plans[0].n_y[y]}},
         "phase_ms_per_step": {
-            "plan": sum(kernels[k]["ms_per_step"] for k in ("k_zero_words", "k_hist", "k_plan") if k in kernels),
+            "plan": sum(kernels[k]["ms_per_step"] for k in ("k_zero_words", "k_hist", "k_plan_fit", "k_plan_tune", "k_plan_finish")
+                        if k in kernels),
             "encode": sum(kernels[k]["ms_per_step"] for k in ("k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
                                                                 "k_sort_scan", "k_sort_pass", "k_pack") if k in kernels),
             "decode_aggregate": sum(kernels[k]["ms_per_step"] for k in ("k_decode_prepare", "k_fill_zero", "k_decode")

@@ -13,9 +13,16 @@
  * Conventions
  *  - Every function returns a status (0 = CVLC_OK); nothing throws, prints or aborts.
  *  - Pointers named *_dev are DEVICE pointers owned by the caller; cvlc_params is
- *    read from HOST memory at call time.  The library allocates no device memory,
- *    keeps no state between calls and only enqueues kernels on `cuda_stream`
- *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *    read from HOST memory at call time.  The library allocates no device memory
+ *    and only enqueues kernels on `cuda_stream` (a cudaStream_t passed as void*;
+ *    NULL = the legacy default stream).
+ *  - State the library keeps in the process, all of it outside the data path: per-device
+ *    flags saying that kernel attributes have been set; two CUDA events per device used by
+ *    cvlc_compress_batch to order its two streams; the launch counters and, while
+ *    cvlc_profile_select is active, the profiling events; the built-in scratch of
+ *    cvlc_decode_aggregate_noalloc and its cached device address.  cvlc_set_device changes
+ *    the calling thread's current device.  None of this is synchronised: call the library
+ *    from one host thread at a time.
  *  - Host-detectable errors are returned at once.  Errors only the device can see
  *    (non-finite input, malformed stream, a wait that ran out) are written to the
  *    status word at byte 0 of the plan / workspace and read with cvlc_read_status;
@@ -80,9 +87,9 @@ enum {
 typedef struct cvlc_params {
   uint64_t d;             /* coordinates, 2 <= d <= 2^31 */
   uint64_t budget_bits;   /* uplink budget of this client this round; R = floor(budget_bits / packet_bits) */
-  uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes).  cvlc_encode assembles four
-                             packets at a time in shared memory: 4 * (b / 8 + 16, plus 8 * cap(1) bytes with QSGD)
-                             must stay within 200 KB, else INVALID_ARG */
+  uint32_t packet_bits;   /* b; multiple of 32; the paper uses 12000 (1500 bytes).  cvlc_encode assembles one
+                             packet per warp, four warps per thread block, in shared memory: 4 * (b / 8 + 16,
+                             plus 8 * cap(1) bytes with QSGD) must stay within 200 KB, else INVALID_ARG */
   uint32_t header_bits;   /* H; 80 <= H < b; 80 = s (8) + y_r (8) + min,max (64), Fig. 2 */
   uint32_t quantizer;     /* CVLC_QUANT_PQ or CVLC_QUANT_QSGD */
   uint32_t max_code_bits; /* 1..32 */
@@ -99,9 +106,10 @@ typedef struct cvlc_plan_t {
   uint32_t R;             /* packets */
   uint32_t y_min;         /* shortest length with a positive coefficient in Eq. (5) */
   uint32_t n_lengths;     /* number of candidate lengths */
-  uint32_t thresh_bin;    /* histogram bin that holds rank k */
+  uint32_t thresh_bin;    /* selection threshold: the histogram bin that holds rank min(d, R * cap(shortest
+                             candidate length)), an upper bound of k that is known before the lengths are tuned */
   uint64_t k;             /* transmitted coordinates, sum of n_y * cap */
-  uint64_t n_candidates;  /* coordinates in bins >= thresh_bin (>= k) */
+  uint64_t n_candidates;  /* coordinates in bins >= thresh_bin (>= k): what the encoder selects and ranks */
   double alpha;           /* fitted decay exponent of Definition 1 */
   double alpha_q;         /* alpha rounded to 1/256 and clamped */
   double beta;            /* 2 * alpha_q + 1 */
@@ -226,6 +234,26 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
                       void* cuda_stream);
 
 /*
+ * cvlc_plan_batch followed by cvlc_encode_batch (with the plan's workspace) in one call: Algorithm 1 from the
+ * update to the packets.  Selection and ranking need the histogram but not the tuned lengths (they work on
+ * the candidates down to an upper bound of k, see cvlc_plan_t::thresh_bin), so with a second stream the
+ * length tuning (Algorithm 1 steps 2-14, a latency-bound computation that leaves the memory system idle)
+ * runs on side_stream next to them and is joined right before the packets are assembled.
+ *  plan_ws_dev / enc_ws_dev   workspaces sized by cvlc_plan_batch_workspace_bytes and
+ *                             cvlc_encode_batch_workspace_bytes (with the same max_candidates)
+ *  side_stream                a second stream of the same device, or NULL / the same stream: everything
+ *                             runs on cuda_stream in order.  When the call returns, cuda_stream is
+ *                             ordered after all work of the call; side_stream needs no further care.
+ * Other arguments, results and errors as the two calls; device-detected errors are at byte 0 of either
+ * workspace.  Uses two CUDA events per device that are created at the first two-stream call on that
+ * device (make it outside of any stream capture).
+ */
+int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint32_t fixed_y,
+                        cvlc_plan_t* plans_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                        uint64_t max_candidates, void* plan_ws_dev, size_t plan_ws_bytes, void* enc_ws_dev,
+                        size_t enc_ws_bytes, void* cuda_stream, void* side_stream);
+
+/*
  * Parameter-server aggregation (Section III, step 3) fused with decoding: for every
  * record of every client, value = min + CID * (max - min) / (2^y - 1) (PQ; the QSGD value is
  * given with CVLC_QUANT_QSGD; every stream names its quantizer in its header), scaled by
@@ -301,8 +329,17 @@ int cvlc_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint
 int cvlc_selftest_math(const double* in_dev, uint64_t n, double* log2_out_dev, double* exp2_out_dev,
                        double* div_out_dev, double* div_ref_dev, void* cuda_stream);
 
+/* The bounded wait every look-back scan of the library uses (a block polls a state word of an earlier
+ * tile at most 2^20 times, then gives up), run on word_dev (8 bytes; a value below 2^62 counts as "not
+ * published yet") with a limit of max_polls (1 .. 2^20): when the wait runs out the kernel writes
+ * CVLC_ERR_DEVICE_TIMEOUT to *status_dev (if that still holds 0) and returns.  Nothing hangs. */
+int cvlc_selftest_wait(uint64_t* word_dev, int32_t* status_dev, uint32_t max_polls, void* cuda_stream);
+
 /* Launch accounting: number of kernels this library has launched in this process
- * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist"). */
+ * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist").  Kernel names: k_zero_words,
+ * k_hist, k_plan_fit, k_plan_tune, k_plan_finish, k_encode_init, k_select, k_select_lookback, k_sort_hist,
+ * k_sort_scan, k_sort_pass, k_pack, k_decode_prepare, k_fill_zero, k_prefetch_l2, k_decode,
+ * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply. */
 unsigned long long cvlc_launch_count(const char* kernel_name);
 /* Optional kernel timing: after cvlc_profile_select(name, n) the next n launches of that kernel
  * ("*" = of every kernel) are bracketed by a CUDA event pair on their own stream;

@@ -751,6 +751,8 @@ int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* 
     for (uint32_t i = 0; i < n_clients; ++i) W = W + (double)weights[i];
   }
   if (!(W > 0.0)) return ORC_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n_clients; ++i)
+    if (!(weights[i] > 0.0f) || !isfinite(weights[i])) return ORC_ERR_INVALID_ARG; /* weights are finite and positive */
   double* acc = (double*)calloc((size_t)d, sizeof(double));
   if (!acc) return ORC_ERR_INVALID_ARG;
   int rc = ORC_OK;
@@ -772,6 +774,9 @@ int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* 
         /* lo is the norm field: a finite, non-negative fp32; the code needs a sign and a level bit */
         uint32_t nb = (uint32_t)get_bits(pkt, 16, 32);
         if (y < 2 || nb >= 0x7F800000u) { rc = ORC_ERR_BAD_STREAM; break; }
+      } else {
+        /* PQ: the two centroid fields are the packet's minimum and maximum, finite and in that order */
+        if (!isfinite(lo) || !isfinite(hi) || lo > hi) { rc = ORC_ERR_BAD_STREAM; break; }
       }
       uint32_t P = (h.packet_bits - h.header_bits) / (s + y);
       for (uint32_t j = 0; j < P; ++j) {

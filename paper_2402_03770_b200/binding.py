@@ -46,7 +46,7 @@ EXPORTS = [
     "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_plan_batch_workspace_bytes",
     "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math", "cvlc_histogram_batch", "cvlc_plan_from_histogram_batch", "cvlc_decode_apply",
-    "cvlc_decode_aggregate_noalloc", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
+    "cvlc_decode_aggregate_noalloc", "cvlc_compress_batch", "cvlc_selftest_wait", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -125,6 +125,10 @@ def lib() -> C.CDLL:
     L.cvlc_plan_batch.argtypes = [vp, PP, u32, u32, vp, vp, sz, vp]
     L.cvlc_encode_batch.restype = C.c_int
     L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
+    L.cvlc_compress_batch.restype = C.c_int
+    L.cvlc_compress_batch.argtypes = [vp, PP, u32, u32, vp, vp, sz, u64, vp, sz, vp, sz, vp, vp]
+    L.cvlc_selftest_wait.restype = C.c_int
+    L.cvlc_selftest_wait.argtypes = [vp, vp, u32, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
     L.cvlc_decode_aggregate.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
     L.cvlc_histogram_batch.restype = C.c_int
@@ -275,6 +279,28 @@ def cvlc_encode_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], 
                                    ws.numel() * ws.element_size(), _stream_handle(stream)), "cvlc_encode_batch")
 
 
+def cvlc_compress_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor,
+                        outs: Sequence[torch.Tensor], plan_ws: torch.Tensor, enc_ws: torch.Tensor, max_candidates: int = 0,
+                        fixed_y: int = 0, stream: Optional[torch.cuda.Stream] = None,
+                        side_stream: Optional[torch.cuda.Stream] = None, _cache=None) -> None:
+    """plan + encode of n clients in one call; with side_stream the length tuning runs next to selection and ranking."""
+    n = len(xs)
+    assert len(params) == n and len(outs) == n and plans.numel() >= n * PLAN_BYTES
+    xa, pa, oa = _cache if _cache is not None else (_ptr_array(xs), _params_array(params), _ptr_array(outs))
+    cap = min(o.numel() for o in outs)
+    side = None if side_stream is None else int(side_stream.cuda_stream)
+    _check(lib().cvlc_compress_batch(xa, pa, n, int(fixed_y), _ptr(plans), oa, cap, int(max_candidates), _ptr(plan_ws),
+                                     plan_ws.numel() * plan_ws.element_size(), _ptr(enc_ws),
+                                     enc_ws.numel() * enc_ws.element_size(), _stream_handle(stream), side),
+           "cvlc_compress_batch")
+
+
+def cvlc_selftest_wait(word: torch.Tensor, status: torch.Tensor, max_polls: int,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert word.element_size() == 8 and status.dtype == torch.int32
+    _check(lib().cvlc_selftest_wait(_ptr(word), _ptr(status), int(max_polls), _stream_handle(stream)), "cvlc_selftest_wait")
+
+
 def cvlc_decode_aggregate(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor,
                           n_clients: int, weight_total: float, d: int, out: torch.Tensor, accumulate: bool,
                           ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
@@ -367,8 +393,9 @@ def cvlc_profile_reset() -> None:
     _check(lib().cvlc_profile_reset(), "cvlc_profile_reset")
 
 
-KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan", "k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
-                "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero", "k_decode", "k_hist_check", "k_apply"]
+KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan_fit", "k_plan_tune", "k_plan_finish", "k_encode_init", "k_select",
+                "k_select_lookback", "k_sort_hist", "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero",
+                "k_prefetch_l2", "k_decode", "k_noalloc_publish_status", "k_selftest", "k_hist_check", "k_apply"]
 
 
 def cvlc_profile_read(kernel_name: str = "*"):
@@ -446,6 +473,14 @@ class BatchEncoder:
             use_plan_ws: bool = True):
         self.plan(xs, stream, fixed_y)
         return self.encode(xs, stream, use_plan_ws)
+
+    def compress(self, xs: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None,
+                 side_stream: Optional[torch.cuda.Stream] = None, fixed_y: int = 0):
+        """plan + encode in one call (cvlc_compress_batch)"""
+        self._xa = _ptr_array(xs)
+        cvlc_compress_batch(xs, self.params, self.plans, self.outs, self.plan_ws, self.enc_ws, self.max_candidates,
+                            fixed_y, stream, side_stream, _cache=(self._xa, self._pa, self._oa))
+        return self.outs
 
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
         rc = cvlc_read_status(self.plan_ws, stream)

@@ -1,5 +1,8 @@
 // C ABI of libcvlc: argument validation, derived constants, workspace carving and
-// stream-ordered kernel launches.  No allocation, no global state, no CPU fallback.
+// stream-ordered kernel launches.  No device allocation, no CPU fallback.  Process-wide state is
+// limited to what include/cvlc.h lists (per-device set-up flags, two events per device for
+// cvlc_compress_batch, launch counters, the profiling events, the scratch of the allocation-free
+// decode); host calls are not thread-safe.
 #include <math.h>
 #include <string.h>
 
@@ -104,6 +107,14 @@ bool same_shape(const cvlc_params& a, const cvlc_params& b) {
 
 bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+size_t plan_ws_bytes_of(uint64_t d, uint32_t n) { return plan_ws_bytes(make_partition(d, n), n); }
+
+// the packing kernel assembles one packet per warp, four warps per block, in shared memory (QSGD: each next to the
+// squares of the packet's values): four of them must fit
+bool pack_fits(const Shape& S) {
+  return 4 * ((size_t)S.packet_bits / 8 + 16 + (S.quantizer == CVLC_QUANT_QSGD ? (size_t)S.cap[1] * 8 : 0)) <= 200 * 1024;
+}
+
 }  // namespace
 
 extern "C" {
@@ -153,7 +164,7 @@ size_t cvlc_plan_workspace_bytes(const cvlc_params* p) { return cvlc_plan_batch_
 
 size_t cvlc_plan_batch_workspace_bytes(const cvlc_params* p, uint32_t n) {
   if (!params_ok(p) || n == 0 || n > CVLC_MAX_BATCH) return 0;
-  return plan_ws_bytes(n, make_partition(p->d, n).max_segments);
+  return plan_ws_bytes_of(p->d, n);
 }
 
 size_t cvlc_encode_workspace_bytes(const cvlc_params* p) { return cvlc_encode_batch_workspace_bytes(p, 1, 0); }
@@ -189,7 +200,7 @@ int cvlc_plan_batch(const float* const* x_dev, const cvlc_params* params, uint32
     desc[i].round = params[i].round;
   }
   if (!aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
-  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < plan_ws_bytes_of(S.d, n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   return launch_plan(desc, n, S, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
@@ -210,7 +221,7 @@ int cvlc_histogram_batch(const float* const* x_dev, const cvlc_params* params, u
   memset(&S, 0, sizeof S);
   S.d = params[0].d;
   if (!aligned(hist_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
-  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < plan_ws_bytes_of(S.d, n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   return launch_histogram(desc, n, S, ws_dev, reinterpret_cast<unsigned long long*>(hist_dev),
                           static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
@@ -233,7 +244,7 @@ int cvlc_plan_from_histogram_batch(const uint64_t* hist_dev, const cvlc_params* 
     desc[i].round = params[i].round;
   }
   if (!aligned(hist_dev, 8) || !aligned(plans_dev, 8) || !aligned(ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
-  if (ws_bytes < plan_ws_bytes(n, make_partition(S.d, n).max_segments)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < plan_ws_bytes_of(S.d, n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   return launch_plan_from_hist(desc, n, S, reinterpret_cast<const unsigned long long*>(hist_dev), ws_dev,
                                static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
@@ -285,11 +296,77 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
   if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
   const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
   if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
-  // four packets at a time are assembled in shared memory (QSGD: each next to the squares of its values)
-  if (4 * ((size_t)S.packet_bits / 8 + 16 + (S.quantizer == CVLC_QUANT_QSGD ? (size_t)S.cap[1] * 8 : 0)) > 200 * 1024) return CVLC_ERR_INVALID_ARG;
+  if (!pack_fits(S)) return CVLC_ERR_INVALID_ARG;
   if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
-  return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
-                                                                                                       : CVLC_ERR_CUDA;
+  return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream), nullptr) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
+}
+
+// Two events per device order the two streams of cvlc_compress_batch (created on first use, kept until exit).
+static cudaError_t compress_events(cudaEvent_t* fork, cudaEvent_t* join) {
+  static cudaEvent_t ev[64][2];
+  static bool made[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!made[dev]) {
+    for (int i = 0; i < 2; ++i) {
+      e = cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming);
+      if (e != cudaSuccess) return e;
+    }
+    made[dev] = true;
+  }
+  *fork = ev[dev][0];
+  *join = ev[dev][1];
+  return cudaSuccess;
+}
+
+int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, uint32_t fixed_y,
+                        cvlc_plan_t* plans_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                        uint64_t max_candidates, void* plan_ws_dev, size_t plan_ws_bytes, void* enc_ws_dev,
+                        size_t enc_ws_bytes, void* cuda_stream, void* side_stream) {
+  if (!x_dev || !params || !streams_dev || n == 0 || n > CVLC_MAX_BATCH || fixed_y > CVLC_MAX_CODE_BITS) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  for (uint32_t i = 0; i < n; ++i) {
+    Shape Si;
+    const int rc = build_shape(&params[i], fixed_y, i == 0 ? &S : &Si);
+    if (rc != CVLC_OK) return rc;
+    if (i && !same_shape(params[0], params[i])) return CVLC_ERR_INVALID_ARG;
+    if (!aligned(x_dev[i], 16) || !aligned(streams_dev[i], 16)) return CVLC_ERR_INVALID_ARG;
+    desc[i].x = x_dev[i];
+    desc[i].plan = plans_dev + i;
+    desc[i].stream = streams_dev[i];
+    desc[i].seed = params[i].seed;
+    desc[i].scale_B = params[i].scale_B;
+    desc[i].client_id = params[i].client_id;
+    desc[i].round = params[i].round;
+  }
+  if (!aligned(plans_dev, 8) || !aligned(plan_ws_dev, 256) || !aligned(enc_ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (plan_ws_bytes < plan_ws_bytes_of(S.d, n)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (stream_capacity < cvlc_stream_bytes(&params[0])) return CVLC_ERR_OUTPUT_TOO_SMALL;
+  const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
+  if (enc_ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (!pack_fits(S)) return CVLC_ERR_INVALID_ARG;
+  if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
+  cudaStream_t main_st = static_cast<cudaStream_t>(cuda_stream), side_st = static_cast<cudaStream_t>(side_stream);
+  const bool two = side_stream != nullptr && side_st != main_st;
+  Shape Senc = S;
+  Senc.fixed_y = 0;
+  if (launch_plan_front(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
+  if (!two) {
+    if (launch_plan_back(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
+    return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, nullptr) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+  }
+  // the length tuning reads the histograms' fit only; selection and ranking do not need its result
+  cudaEvent_t fork, join;
+  if (compress_events(&fork, &join) != cudaSuccess) return CVLC_ERR_CUDA;
+  if (cudaEventRecord(fork, main_st) != cudaSuccess || cudaStreamWaitEvent(side_st, fork, 0) != cudaSuccess) return CVLC_ERR_CUDA;
+  if (launch_plan_back(desc, n, S, plan_ws_dev, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
+  if (cudaEventRecord(join, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
+  return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, join) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, const void* plan_ws_dev,
@@ -333,6 +410,14 @@ int cvlc_read_status(const void* plan_or_ws_dev, void* cuda_stream) {
   if (cudaMemcpyAsync(&v, plan_or_ws_dev, sizeof v, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CVLC_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return CVLC_ERR_CUDA;
   return (int)v;
+}
+
+int cvlc_selftest_wait(uint64_t* word_dev, int32_t* status_dev, uint32_t max_polls, void* cuda_stream) {
+  if (!aligned(word_dev, 8) || !aligned(status_dev, 4) || max_polls == 0 || max_polls > (1u << 20)) return CVLC_ERR_INVALID_ARG;
+  return launch_selftest_wait(reinterpret_cast<unsigned long long*>(word_dev), status_dev, max_polls,
+                              static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
 }
 
 int cvlc_selftest_philox(uint64_t seed, uint32_t client_id, uint32_t round, uint64_t first, uint64_t n, uint32_t* out_dev,

@@ -93,9 +93,24 @@ CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
   return P;
 }
 
+// Rows: the float4 units of a segment are also grouped into rows of 32 units (128 coordinates, one warp-wide load)
+// and tiles of 64 rows (the selection kernel's tile).  The histogram kernel leaves the largest magnitude key of every
+// row; once the selection threshold is known the planner turns them into one bit per row ("holds a candidate"), 64
+// rows = one tile per 64-bit word, and the selection kernel skips rows and whole tiles without candidates.  Tile t
+// of the segment that starts at position p0 of the concatenated array has index p0 / 2048 + segment id + t: the
+// index ranges of different segments do not overlap.
+constexpr int kRowUnits = 32;
+constexpr int kTileRows = 64;
+constexpr int kTileUnits = kRowUnits * kTileRows;  // 2048 float4 = 8192 coordinates
+CVLC_HD inline uint64_t row_tiles_total(const Partition& P) { return P.total / kTileUnits + P.max_segments + 1; }
+CVLC_HD inline uint64_t seg_first_tile(uint64_t p0, uint32_t seg) { return p0 / kTileUnits + seg; }
+
 // plan workspace:
-//   [0] PlanWsHeader | [256] uint64 hist[n][4096] | uint32 nonfinite[n] | uint32 seg_count[S]
-//   | uint64 seg_prefix[S] | uint32 seg_hist[S][4096]          (S = max_segments)
+//   [0] PlanWsHeader | [256] uint64 hist[n][4096] | uint32 nonfinite[n] | uint64 tune_key[n][2] | uint32 leader[n]
+//   | uint32 seg_count[S] | uint64 seg_prefix[S] | uint32 row_max[64 * tiles] | uint64 row_flags[tiles]
+//   | uint32 seg_hist[S][4096]          (S = max_segments, tiles = row_tiles_total)
+// tune_key = (bits of alpha_q, bits of scale_B): clients of a batch with equal keys have the same code lengths;
+// leader[c] = the first client of the batch with c's key (it runs the length tuning, the others copy its result).
 struct PlanWsHeader {
   int32_t status;   // byte 0
   uint32_t n;       // clients of the batch the workspace was filled for
@@ -106,12 +121,21 @@ struct PlanWsHeader {
 constexpr uint32_t kPlanWsMagic = 0x53454743u;
 constexpr size_t kPlanWsHist = 256;
 CVLC_HD constexpr size_t plan_off_flags(uint32_t n) { return kPlanWsHist + (size_t)n * CVLC_HIST_BINS * 8; }
-CVLC_HD constexpr size_t plan_off_seg_count(uint32_t n) { return align256(plan_off_flags(n) + (size_t)n * 4); }
+CVLC_HD constexpr size_t plan_off_keys(uint32_t n) { return align256(plan_off_flags(n) + (size_t)n * 4); }
+CVLC_HD constexpr size_t plan_off_leader(uint32_t n) { return align256(plan_off_keys(n) + (size_t)n * 16); }
+CVLC_HD constexpr size_t plan_off_seg_count(uint32_t n) { return align256(plan_off_leader(n) + (size_t)n * 4); }
 CVLC_HD constexpr size_t plan_off_seg_prefix(uint32_t n, uint32_t S) { return align256(plan_off_seg_count(n) + (size_t)S * 4); }
-CVLC_HD constexpr size_t plan_off_seg_hist(uint32_t n, uint32_t S) { return align256(plan_off_seg_prefix(n, S) + (size_t)S * 8); }
-CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n, uint32_t S) {
-  return align256(plan_off_seg_hist(n, S) + (size_t)S * CVLC_HIST_BINS * 4);
+CVLC_HD constexpr size_t plan_off_row_max(uint32_t n, uint32_t S) { return align256(plan_off_seg_prefix(n, S) + (size_t)S * 8); }
+CVLC_HD constexpr size_t plan_off_row_flags(uint32_t n, uint32_t S, uint64_t tiles) {
+  return align256(plan_off_row_max(n, S) + (size_t)tiles * kTileRows * 4);
 }
+CVLC_HD constexpr size_t plan_off_seg_hist(uint32_t n, uint32_t S, uint64_t tiles) {
+  return align256(plan_off_row_flags(n, S, tiles) + (size_t)tiles * 8);
+}
+CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n, uint32_t S, uint64_t tiles) {
+  return align256(plan_off_seg_hist(n, S, tiles) + (size_t)S * CVLC_HIST_BINS * 4);
+}
+CVLC_HD inline size_t plan_ws_bytes(const Partition& P, uint32_t n) { return plan_ws_bytes(n, P.max_segments, row_tiles_total(P)); }
 
 // encode workspace header (first 256 bytes), zeroed at the start of a call
 struct EncHeader {
@@ -181,8 +205,9 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 // ---- launch accounting and optional per-kernel timing ------------------------------
 
 enum KernelId {
-  kKZeroWords = 0, kKHist, kKPlan, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan, kKSortPass, kKPack,
-  kKDecodePrepare, kKFillZero, kKDecode, kKSelftest, kKHistCheck, kKApply, kNumKernelIds
+  kKZeroWords = 0, kKHist, kKPlanFit, kKPlanTune, kKPlanFinish, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan,
+  kKSortPass, kKPack, kKDecodePrepare, kKFillZero, kKPrefetchL2, kKDecode, kKNoallocStatus, kKSelftest, kKHistCheck, kKApply,
+  kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -199,14 +224,22 @@ struct LaunchScope {
 
 // ---- launchers (one per translation unit) ---------------------------------------
 
+// Planning is launched in two parts.  The front (histogram, exponent fit, selection threshold, per-segment candidate
+// counts) is all the selection and ranking kernels need; the back (length tuning, copied to the clients that share a
+// tuning key) is only needed by the packing kernel, so it may run on another stream next to selection and ranking.
+cudaError_t launch_plan_front(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
+cudaError_t launch_plan_back(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
 cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st);
 cudaError_t launch_histogram(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
                              unsigned long long* hist_out, cudaStream_t st);
 cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const Shape& shape,
                                   const unsigned long long* hist, void* ws, cudaStream_t st);
 cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st);
+// wait_before_pack: an event the stream waits for right before the packing kernel (the length tuning on
+// another stream), or nullptr
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                          const void* plan_ws, void* ws, cudaStream_t st);
+                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack);
+cudaError_t launch_selftest_wait(unsigned long long* word, int32_t* status, uint32_t max_polls, cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
                           void* ws, cudaStream_t st);

@@ -71,7 +71,9 @@ k_decode_prepare(const uint8_t* const* __restrict__ streams, const uint64_t* __r
         if (ok) ok = ((uint64_t)CVLC_STREAM_HEADER_BYTES + (uint64_t)sR * (pb / 8) == nbytes);
         if (ok) {
           R = sR;
-          coef[i] = (float)((double)weights[i] / (W * B));
+          const float wi = weights[i];
+          if (!(wi > 0.0f) || __float_as_uint(wi) >= 0x7F800000u) set_status(status, CVLC_ERR_INVALID_ARG);  // weights are finite and positive
+          coef[i] = (float)((double)wi / (W * B));
           meta[2 * i] = pb | ((ver_q_s >> 16) & 0xFF);  // packet bits are a multiple of 32: the quantizer rides below
           meta[2 * i + 1] = hb;
         }
@@ -150,9 +152,12 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
   const float* coef = reinterpret_cast<const float*>(ws + kDecWsCoef);
   const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + dec_off_prefix(n));
   const uint32_t* meta = reinterpret_cast<const uint32_t*>(ws + dec_off_meta(n));
-  if (*status != 0) return;
+  // blocks that run later may see an error set by earlier ones: one thread reads the word, the whole block follows it
+  __shared__ int s_err;
+  if (threadIdx.x == 0) s_err = *reinterpret_cast<const volatile int32_t*>(status);
   for (uint32_t i = threadIdx.x; i <= n; i += kDecodeThreads) s_prefix[i] = prefix[i];
   __syncthreads();
+  if (s_err != 0) return;
   const uint32_t total = s_prefix[n];
   const int lane = threadIdx.x & 31;
   const uint32_t warps_total = gridDim.x * (kDecodeThreads / 32);
@@ -193,6 +198,11 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
     // QSGD: the first centroid field is the packet's l2-norm (finite, not negative); a code is the sign
     // bit above a level of 2^(y-1) - 1 steps, so one bit is not a code
     if (qsgd && (y < 2 || __float_as_uint(lo) >= 0x7F800000u)) {
+      if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
+      continue;
+    }
+    // PQ: minimum and maximum are finite and ordered
+    if (!qsgd && ((__float_as_uint(lo) & 0x7FFFFFFFu) >= 0x7F800000u || (__float_as_uint(hi) & 0x7FFFFFFFu) >= 0x7F800000u || lo > hi)) {
       if (lane == 0) set_status(status, CVLC_ERR_BAD_STREAM);
       continue;
     }
@@ -250,7 +260,7 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
       LaunchScope ls(kKFillZero, st);
       k_fill_zero<<<grid, 256, 0, st>>>(out + lo, hi - lo);
     } else if (n_win > 1) {
-      LaunchScope ls(kKFillZero, st);
+      LaunchScope ls(kKPrefetchL2, st);
       k_prefetch_l2<<<grid, 256, 0, st>>>(out + lo, hi - lo);
     }
     LaunchScope ls(kKDecode, st);
@@ -353,7 +363,7 @@ extern "C" int cvlc_decode_aggregate_noalloc(const uint8_t* const* streams_dev, 
                     accumulate ? 1 : 0, scratch, st) != cudaSuccess)
     return CVLC_ERR_CUDA;
   {
-    LaunchScope ls(kKDecodePrepare, st);
+    LaunchScope ls(kKNoallocStatus, st);
     k_noalloc_publish_status<<<1, 1, 0, st>>>(status_dev);
   }
   return cudaGetLastError() == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;

@@ -1,7 +1,8 @@
 // Encoding kernels (Algorithm 1, steps 15-17), batched over clients: top-k candidate
 // selection by the plan's histogram threshold, stable LSD radix ranking of the candidates
-// by |x|, per-packet minimum/maximum, PQ stochastic quantization with Philox4x32-10 and
-// bit packing of (position ID, centroid ID) pairs into fixed-size packets (Fig. 2).
+// by |x|, the per-packet centroid distribution (PQ: minimum and maximum; QSGD: l2-norm),
+// stochastic quantization with Philox4x32-10 (PQ or QSGD) and bit packing of
+// (position ID, centroid ID) pairs into fixed-size packets (Fig. 2).
 #include "cvlc_common.cuh"
 
 namespace cvlc {
@@ -23,11 +24,11 @@ __device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long 
 }
 
 // Waits (bounded) until a look-back state word carries a flag.  Returns 0 after a timeout.
-__device__ __forceinline__ unsigned long long wait_state(const unsigned long long* p, int32_t* status) {
+__device__ __forceinline__ unsigned long long wait_state(const unsigned long long* p, int32_t* status, int max_polls = kMaxPolls) {
   unsigned long long v = ld_relaxed(p);
   int polls = 0;
   while ((v & kFlagMask) == 0) {
-    if (++polls > kMaxPolls) {
+    if (++polls > max_polls) {
       set_status(status, CVLC_ERR_DEVICE_TIMEOUT);
       return 0;
     }
@@ -35,6 +36,15 @@ __device__ __forceinline__ unsigned long long wait_state(const unsigned long lon
     v = ld_relaxed(p);
   }
   return v;
+}
+
+// Whether an earlier kernel of the call has reported an error.  Other blocks may set the word while this kernel
+// runs, so one thread reads it and the whole block takes the same branch.
+__device__ __forceinline__ bool block_sees_error(const int32_t* status) {
+  __shared__ int s_err;
+  if (threadIdx.x == 0) s_err = *reinterpret_cast<const volatile int32_t*>(status);
+  __syncthreads();
+  return s_err != 0;
 }
 
 __device__ __forceinline__ uint32_t sort_tiles_of(unsigned long long n_candidates, unsigned long long capacity) {
@@ -53,13 +63,27 @@ __global__ void __launch_bounds__(256)
 k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
               const __grid_constant__ EncLayout L, const unsigned char* plan_ws, const __grid_constant__ Partition part) {
   __shared__ unsigned long long s_total;
-  __shared__ int s_bad;
+  __shared__ int s_bad, s_pass3;
+  __shared__ uint32_t s_tiles[CVLC_MAX_BATCH];  // sort tiles of every client
   const uint32_t n = batch.n;
   if (threadIdx.x == 0) {
-    unsigned long long t = 0;
-    for (uint32_t c = 0; c < n; ++c) t += sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
-    s_total = t;
+    s_total = 0;
     s_bad = 0;
+    s_pass3 = 0;
+  }
+  __syncthreads();
+  {
+    unsigned long long t = 0;
+    int pass3 = 0;
+    for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {  // the plans are read side by side, not one after the other
+      const cvlc_plan_t* plan = batch.c[c].plan;
+      const uint32_t tiles = sort_tiles_of(plan->n_candidates, L.capacity);
+      s_tiles[c] = tiles;
+      t += tiles;
+      if (plan->top_bin + 1u - plan->thresh_bin > 256u) pass3 = 1;  // see top_digit_is_zero
+    }
+    if (t) atomicAdd(&s_total, t);
+    if (pass3) atomicOr(&s_pass3, 1);
   }
   __syncthreads();
   const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -71,28 +95,27 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
     const size_t nb = (L.off_sort_state - L.off_ghist) / 8;  // digit histograms, their scans, selection tile states
     for (size_t i = gtid; i < nb; i += gstride) b[i] = 0ull;
   }
+  // look-back states of the digit passes that will run (the fourth only if some client's keys span more than 2^27)
   const size_t per_pass = (size_t)s_total * kDigits;
-  for (int p = 0; p < kSortPasses; ++p) {
-    unsigned long long* st = reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) + (size_t)p * n * L.sort_tiles_max * kDigits;
-    for (size_t i = gtid; i < per_pass; i += gstride) st[i] = 0ull;
+  const int n_passes = s_pass3 ? kSortPasses : kSortPasses - 1;
+  for (int p = 0; p < n_passes; ++p) {
+    ulonglong2* st = reinterpret_cast<ulonglong2*>(reinterpret_cast<unsigned long long*>(ws + L.off_sort_state) +
+                                                   (size_t)p * n * L.sort_tiles_max * kDigits);
+    for (size_t i = gtid; i < per_pass / 2; i += gstride) st[i] = make_ulonglong2(0ull, 0ull);
   }
   if (blockIdx.x != 0) return;
 
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   uint32_t* prefix = reinterpret_cast<uint32_t*>(ws + L.off_sort_prefix);
   for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+    // Only what selection and ranking use is checked here (the code lengths may still be on their way on
+    // another stream); the packing kernel checks the lengths.
     const cvlc_plan_t* plan = batch.c[c].plan;
-    unsigned long long k = 0, nsum = 0;
-    for (int y = 1; y <= CVLC_MAX_CODE_BITS; ++y) {
-      k += (unsigned long long)plan->n_y[y] * plan->cap[y];
-      nsum += plan->n_y[y];
-    }
     int bad = 0;
     if (plan->status != CVLC_OK)
       bad = plan->status;
-    else if (plan->s != shape.s || plan->R != shape.R || nsum != shape.R || k != plan->k || k == 0 ||
-             k > plan->n_candidates || plan->n_candidates > shape.d || plan->thresh_bin >= CVLC_HIST_BINS ||
-             (shape.quantizer == CVLC_QUANT_QSGD && plan->n_y[1] != 0))  // a one-bit QSGD code holds no level
+    else if (plan->s != shape.s || plan->R != shape.R || plan->n_candidates == 0 || plan->n_candidates > shape.d ||
+             plan->thresh_bin >= CVLC_HIST_BINS || plan->top_bin >= CVLC_HIST_BINS || plan->top_bin < plan->thresh_bin)
       bad = CVLC_ERR_PLAN_MISMATCH;
     else if (plan->n_candidates > L.capacity)
       bad = CVLC_ERR_WORKSPACE_TOO_SMALL;
@@ -103,7 +126,7 @@ k_encode_init(unsigned char* ws, const __grid_constant__ BatchDesc<CAP> batch, c
     uint32_t run = 0, mx = 0;
     for (uint32_t c = 0; c < n; ++c) {
       prefix[c] = run;
-      const uint32_t t = sort_tiles_of(batch.c[c].plan->n_candidates, L.capacity);
+      const uint32_t t = s_tiles[c];
       run += t;
       if (t > mx) mx = t;
     }
@@ -139,7 +162,7 @@ k_select_lookback(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, unsi
   __shared__ unsigned long long s_look_sum[kSelectThreads / 32];
   __shared__ uint32_t s_look_flag[kSelectThreads / 32];
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  if (block_sees_error(&hdr->status)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint64_t tiles_per_client = L.select_tiles;
   const uint64_t total_tiles = tiles_per_client * batch.n;
@@ -300,6 +323,9 @@ __device__ __forceinline__ void cp_async_wait() {
 
 // sort key digits (see the ranking kernels below); the selection kernel already counts them
 __device__ __forceinline__ uint32_t sort_keytop(const cvlc_plan_t* plan) { return ((plan->top_bin + 1u) << 19) - 1u; }
+// With at most 256 histogram bins between the threshold and the top, keytop - key stays below 2^27 for every
+// candidate: the fourth digit is zero throughout and neither counted nor ranked.
+__device__ __forceinline__ bool top_digit_is_zero(const cvlc_plan_t* plan) { return plan->top_bin + 1u - plan->thresh_bin <= 256u; }
 
 __device__ __forceinline__ uint32_t sort_digit(unsigned long long pair, int pass, uint32_t keytop) {
   const uint32_t key = (uint32_t)(pair >> 32);
@@ -326,15 +352,19 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
   for (int i = threadIdx.x; i < kSortPasses * kDigits; i += kSelThreads) s_dhist[i] = 0;
   __syncthreads();
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  if (block_sees_error(&hdr->status)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t S = part.max_segments;
   const uint32_t* seg_count = reinterpret_cast<const uint32_t*>(plan_ws + plan_off_seg_count(batch.n));
   const unsigned long long* seg_prefix = reinterpret_cast<const unsigned long long*>(plan_ws + plan_off_seg_prefix(batch.n, S));
+  // one bit per row of 32 units (does it hold a candidate?), one 64-bit word per tile, from the planner
+  const unsigned long long* row_flags =
+      reinterpret_cast<const unsigned long long*>(plan_ws + plan_off_row_flags(batch.n, S, row_tiles_total(part)));
   unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;
   constexpr uint32_t kTileVec = kSelTileVec;
+  static_assert(kSelTileVec == kTileUnits && kSelThreads / 32 * 4 == kTileRows, "a warp stages four rows of a tile");
   int parity = 0;
   __shared__ uint32_t s_chunk;
 
@@ -363,6 +393,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const float below_thresh_f = __uint_as_float(thresh ? thresh - 1u : 0u);
     const uint32_t cap32 = (uint32_t)L.capacity;  // <= d <= 2^31
     const uint32_t keytop = sort_keytop(plan);
+    const bool count_top = !top_digit_is_zero(plan);
     const uint32_t seg = q + c;
     unsigned long long* __restrict__ out = reinterpret_cast<unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     unsigned long long run = seg_prefix[seg];
@@ -373,47 +404,52 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     // A warp stages exactly the 128 units (512 coordinates) its own lanes will read: four copies of 32
     // consecutive float4s each (coalesced).  Waiting for a tile and reusing a staging slot are then a matter
     // between the lanes of one warp, and the block meets only once per tile, for the scan.
+    // Rows without a candidate are neither copied nor looked at, tiles without one are passed over altogether.
+    const unsigned long long* __restrict__ tile_flags = row_flags + seg_first_tile(pos, seg);
+    auto flags_of = [&](uint32_t t) -> unsigned long long { return t < n_tiles ? __ldg(tile_flags + t) : 0ull; };
     uint32_t istage = 0;
-    auto issue = [&](uint32_t t) {
-      if (t < n_tiles) {
+    auto issue = [&](uint32_t t, unsigned long long tf) {
+      const uint32_t rows = (uint32_t)(tf >> (4 * warp)) & 0xFu;  // this warp's four rows of the tile
+      if (rows) {  // (a tile past the end has no flags)
         float4* dst = s_stage + (size_t)istage * kTileVec;
         const uint64_t base = (uint64_t)t * kTileVec;
-        if (base + kTileVec <= n_vec) {
 #pragma unroll
-          for (int v = 0; v < kSelVec; ++v) {
-            const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
-            cp_async16(dst + sel_slot(g), xseg + base + g);
-          }
-        } else {
-#pragma unroll
-          for (int v = 0; v < kSelVec; ++v) {
-            const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
-            if (base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
-          }
+        for (int v = 0; v < kSelVec; ++v) {
+          const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
+          if (((rows >> v) & 1u) && base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
         }
       }
       istage = (istage + 1 == kSelStages) ? 0u : istage + 1;
       cp_async_commit();  // one group per tile slot, empty past the end, keeps the group count uniform
     };
 
-#pragma unroll
-    for (int t = 0; t < kSelStages - 1; ++t) issue(t);
+    static_assert(kSelStages == 3, "the flag words of three tiles are carried along");
+    unsigned long long f0 = flags_of(0), f1 = flags_of(1), f2 = flags_of(2);
+    issue(0, f0);
+    issue(1, f1);
     uint32_t stage = 0;
     for (uint32_t t = 0; t < n_tiles; ++t) {
+      const unsigned long long tile_rows = f0;
+      const unsigned long long f3 = flags_of(t + 3);  // asked for one tile before it is needed
       cp_async_wait<kSelStages - 2>();  // this lane's copies of tile t have landed
       __syncwarp();                     // ... and the other lanes'; and the warp is done with its part of tile t - 1,
-      issue(t + kSelStages - 1);        // whose staging slot the next copies overwrite
+      issue(t + kSelStages - 1, f2);    // whose staging slot the next copies overwrite
+      f0 = f1;
+      f1 = f2;
+      f2 = f3;
       const float4* src = s_stage + (size_t)stage * kTileVec;
       stage = (stage + 1 == kSelStages) ? 0u : stage + 1;
+      if (tile_rows == 0ull) continue;  // the same for the whole block
       const uint64_t base = (uint64_t)t * kTileVec;
       // this thread's 16 consecutive coordinates: units 4 tid .. 4 tid + 3 of the tile
       uint32_t m = 0;
       const uint32_t g0 = (uint32_t)kSelVec * tid;
       const uint32_t ct = ((uint32_t)tid >> 1) & (uint32_t)(kSelVec - 1);
       const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < kSelVec) ? n_vec - base - g0 : kSelVec) : 0u;
+      const bool row_on = (tile_rows >> (4 * warp + (lane >> 3))) & 1ull;  // the thread's four units lie in one row
 #pragma unroll
       for (int j = 0; j < kSelVec; ++j) {
-        if ((uint32_t)j < left) {
+        if (row_on && (uint32_t)j < left) {
           // units 4 tid + j sit in slots 4 tid + (j ^ ct): the swizzle only touches the two low bits
           const float4 f = src[g0 + ((uint32_t)j ^ ct)];
           m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.x))), m, 1);
@@ -460,7 +496,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         if (o < cap32) out[o] = ((unsigned long long)key << 32) | (unsigned long long)((b & 0x80000000u) | (e32 + c16));
         const uint32_t inv = keytop - (key < keytop ? key : keytop);
 #pragma unroll
-        for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + ((inv >> (kDigitBits * p)) & (kDigits - 1))], 1u);
+        for (int p = 0; p < kSortPasses - 1; ++p) atomicAdd(&s_dhist[p * kDigits + ((inv >> (kDigitBits * p)) & (kDigits - 1))], 1u);
+        if (count_top) atomicAdd(&s_dhist[(kSortPasses - 1) * kDigits + (inv >> (kDigitBits * (kSortPasses - 1)))], 1u);
         ++o;
       }
       run += tot;
@@ -473,7 +510,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
         if ((b & 0x7FFFFFFFu) >= thresh) {
           const unsigned long long pair = ((unsigned long long)(b & 0x7FFFFFFFu) << 32) | (unsigned long long)(b & 0x80000000u) | (unsigned long long)e;
           if (run < L.capacity) out[run] = pair;
-          for (int p = 0; p < kSortPasses; ++p) atomicAdd(&s_dhist[p * kDigits + sort_digit(pair, p, keytop)], 1u);
+          for (int p = 0; p < kSortPasses; ++p)
+            if (p < kSortPasses - 1 || count_top) atomicAdd(&s_dhist[p * kDigits + sort_digit(pair, p, keytop)], 1u);
           ++run;
         }
       }
@@ -518,7 +556,7 @@ __global__ void __launch_bounds__(256)
 k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ uint32_t sh[kSortPasses * kDigits];
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  if (block_sees_error(&hdr->status)) return;
   const uint32_t* prefix = reinterpret_cast<const uint32_t*>(ws + L.off_sort_prefix);
   unsigned long long* ghist_all = reinterpret_cast<unsigned long long*>(ws + L.off_ghist);
   for (int i = threadIdx.x; i < kSortPasses * kDigits; i += 256) sh[i] = 0;
@@ -533,6 +571,7 @@ k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
     const uint32_t seg_end = prefix[c + 1] < t_end ? prefix[c + 1] : t_end;
     const unsigned long long n = batch.c[c].plan->n_candidates;
     const uint32_t keytop = sort_keytop(batch.c[c].plan);
+    const int n_count = top_digit_is_zero(batch.c[c].plan) ? kSortPasses - 1 : kSortPasses;
     const unsigned long long* __restrict__ in = reinterpret_cast<const unsigned long long*>(ws + L.off_buf_a) + (size_t)c * L.capacity;
     const unsigned long long i0 = (unsigned long long)(t - prefix[c]) * kSortTile;
     unsigned long long i1 = (unsigned long long)(seg_end - prefix[c]) * kSortTile;
@@ -540,7 +579,8 @@ k_sort_hist(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, con
     for (unsigned long long i = i0 + threadIdx.x; i < i1; i += 256) {
       const unsigned long long pair = in[i];
 #pragma unroll
-      for (int p = 0; p < kSortPasses; ++p) atomicAdd(&sh[p * kDigits + sort_digit(pair, p, keytop)], 1u);
+      for (int p = 0; p < kSortPasses; ++p)
+        if (p < n_count) atomicAdd(&sh[p * kDigits + sort_digit(pair, p, keytop)], 1u);
     }
     __syncthreads();
     unsigned long long* ghist = ghist_all + (size_t)c * kSortPasses * kDigits;
@@ -560,13 +600,13 @@ __global__ void __launch_bounds__(kDigits)
 k_sort_scan(const __grid_constant__ BatchDesc<CAP> batch, unsigned char* ws, const __grid_constant__ EncLayout L) {
   __shared__ unsigned long long s_scan[kDigits / 32];
   const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  if (block_sees_error(&hdr->status)) return;
   const uint32_t c = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long n = batch.c[c].plan->n_candidates;
   const unsigned long long* ghist = reinterpret_cast<const unsigned long long*>(ws + L.off_ghist) + (size_t)c * kSortPasses * kDigits;
   unsigned long long* gbase = reinterpret_cast<unsigned long long*>(ws + L.off_gbase) + (size_t)c * kSortPasses * kDigits;
-  uint32_t mask = 0;
+  uint32_t mask = top_digit_is_zero(batch.c[c].plan) ? 1u << (kSortPasses - 1) : 0u;  // not counted: known to be constant
   for (int p = 0; p < kSortPasses; ++p) {
     const unsigned long long cnt = ghist[p * kDigits + tid];
     if (__syncthreads_or(cnt == n)) mask |= 1u << p;
@@ -792,7 +832,7 @@ k_sort_pass(int pass, const __grid_constant__ BatchDesc<CAP> batch, unsigned cha
   uint32_t* s_keytop = s_ncand + batch.n;        // [n] top of its key range
   uint32_t* s_mask = s_keytop + batch.n;         // [n] its constant digits
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  if (block_sees_error(&hdr->status)) return;
   const int tid = threadIdx.x;
   const uint32_t n_clients = batch.n;
   {
@@ -886,8 +926,8 @@ __global__ void __launch_bounds__(kPackThreads)
 k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
        const __grid_constant__ EncLayout L, uint32_t warp_bytes) {
   extern __shared__ __align__(16) unsigned char s_pack[];  // per warp: packet words; QSGD: then cap(1) squares
-  const EncHeader* hdr = reinterpret_cast<const EncHeader*>(ws);
-  if (hdr->status != 0) return;
+  EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
+  if (block_sees_error(&hdr->status)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t c = blockIdx.y;
   const ClientDesc& cd = batch.c[c];
@@ -921,12 +961,23 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
       zc += b;
     }
   }
+  {
+    // the code lengths must fill the stream's R packets with k of the selected candidates (every warp of every
+    // block of the client sees the same plan and takes the same branch)
+    const uint32_t tot_packets = __shfl_sync(kFull, cum, 31);
+    const unsigned long long tot_records = __shfl_sync(kFull, zc, 31);
+    const bool qsgd_one_bit = QSGD && __shfl_sync(kFull, ny, 31) != 0;  // a one-bit QSGD code holds no level
+    if (tot_packets != shape.R || tot_records != plan->k || tot_records == 0 || tot_records > plan->n_candidates || qsgd_one_bit) {
+      if (blockIdx.x == 0 && tid == 0) set_status(&hdr->status, CVLC_ERR_PLAN_MISMATCH);
+      return;
+    }
+  }
 
   for (int g = 0; g < kPackGroup; ++g) {
     const uint32_t r = (blockIdx.x * kPackWarps + warp) * kPackGroup + g;
     if (r >= shape.R) break;
     const unsigned hit = __ballot_sync(kFull, r < cum);
-    if (hit == 0) break;  // fewer packets planned than the stream holds: caught by the plan check
+    if (hit == 0) break;
     const int src_lane = __ffs(hit) - 1;
     const uint32_t y = CVLC_MAX_CODE_BITS - (uint32_t)src_lane;
     const unsigned long long Z = __shfl_sync(kFull, (zc - nz) + (unsigned long long)(r - (cum - ny)) * capl, src_lane);
@@ -1108,7 +1159,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
 
 template <int CAP>
 static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                                   const void* plan_ws, void* ws, cudaStream_t st) {
+                                   const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -1167,6 +1218,10 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
       k_sort_pass<CAP><<<grid, kSortThreads, sort_smem_bytes(n), st>>>(pass, batch, w, L);
     }
   }
+  if (wait_before_pack) {
+    const cudaError_t ew = cudaStreamWaitEvent(st, wait_before_pack, 0);
+    if (ew != cudaSuccess) return ew;
+  }
   {
     LaunchScope ls(kKPack, st);
     if (qsgd)
@@ -1178,9 +1233,20 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
 }
 
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                          const void* plan_ws, void* ws, cudaStream_t st) {
-  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, plan_ws, ws, st);
-  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, plan_ws, ws, st);
+                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack) {
+  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack);
+  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack);
+}
+
+// The bounded wait of the look-back scans, run on a word nobody publishes: after max_polls polls it gives up,
+// reports DEVICE_TIMEOUT and the kernel returns.
+__global__ void k_selftest_wait(const unsigned long long* word, int32_t* status, int max_polls) {
+  wait_state(word, status, max_polls);
+}
+
+cudaError_t launch_selftest_wait(unsigned long long* word, int32_t* status, uint32_t max_polls, cudaStream_t st) {
+  { LaunchScope ls(kKSelftest, st); k_selftest_wait<<<1, 32, 0, st>>>(word, status, (int)max_polls); }
+  return cudaGetLastError();
 }
 
 }  // namespace cvlc

@@ -1,6 +1,6 @@
-// Planning kernels: magnitude histogram (Algorithm 1, step 1) and the single-CTA
-// planner (power-law exponent of Definition 1, code-length tuning by atomic
-// operations on Eq. (5), Algorithm 1 steps 2-14).
+// Planning kernels: magnitude histogram (Algorithm 1, step 1), the exponent fit of Definition 1 with the
+// selection threshold, and the code-length tuning by atomic operations on Eq. (5) (Algorithm 1 steps 2-14),
+// one CTA per client, run once per distinct (exponent, scale) of a batch.
 //
 // The planner's floating point is IEEE binary64 with every multiply and add
 // rounded separately (the *_rn intrinsics keep the compiler from contracting
@@ -20,6 +20,8 @@ constexpr int kHistSub = 4;  // shared sub-histograms per block (64 KB)
 // plus one ragged-tail unit per client) that is cut into equal contiguous chunks, one per
 // block, so the load is even whatever the number of clients; a block that crosses a client
 // boundary merges its shared histogram into that client's global one and starts afresh.
+
+// counts the four magnitude keys of a float4; returns the largest of them
 __device__ __forceinline__ uint32_t hist_add4(uint32_t* my, const float4 a) {
   const uint32_t k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
   const uint32_t k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
@@ -27,17 +29,20 @@ __device__ __forceinline__ uint32_t hist_add4(uint32_t* my, const float4 a) {
   atomicAdd(my + (k1 >> 19), 1u);
   atomicAdd(my + (k2 >> 19), 1u);
   atomicAdd(my + (k3 >> 19), 1u);
-  return (k0 >= 0x7F800000u) | (k1 >= 0x7F800000u) | (k2 >= 0x7F800000u) | (k3 >= 0x7F800000u);
+  const uint32_t m01 = k0 > k1 ? k0 : k1, m23 = k2 > k3 ? k2 : k3;
+  return m01 > m23 ? m01 : m23;
 }
 
 template <int CAP>
 __global__ void __launch_bounds__(kHistThreads, 2)
 k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_constant__ Partition part,
-       unsigned long long* __restrict__ hist_all, uint32_t* __restrict__ nonfinite_all, uint32_t* __restrict__ seg_hist_all) {
+       unsigned long long* __restrict__ hist_all, uint32_t* __restrict__ nonfinite_all, uint32_t* __restrict__ seg_hist_all,
+       uint32_t* __restrict__ row_max_all) {
   extern __shared__ uint32_t sh_hist[];  // [kHistSub][4096]
   for (int i = threadIdx.x; i < kHistSub * CVLC_HIST_BINS; i += kHistThreads) sh_hist[i] = 0;
   __syncthreads();
   uint32_t* my = sh_hist + ((threadIdx.x >> 5) & (kHistSub - 1)) * CVLC_HIST_BINS;
+  const int lane = threadIdx.x & 31;
 
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;  // per client: nvec float4 units and one tail unit
@@ -52,24 +57,35 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     const float* __restrict__ x = batch.c[c].x;
     const float4* xv = reinterpret_cast<const float4*>(x);
     const uint64_t v1 = (u1 < nvec) ? u1 : nvec;  // float4 units of this segment: [u0, v1)
-    uint32_t bad = 0;
+    // largest key of every row (32 consecutive units from u0 on: what one warp loads at a time)
+    uint32_t* __restrict__ row_max = row_max_all + seg_first_tile(pos, (uint32_t)(q + c)) * kTileRows;
+    uint32_t top = 0;
     uint64_t v = u0 + threadIdx.x;
-    // four independent 128-bit loads in flight per thread
-    for (; v + 3 * kHistThreads < v1; v += 4 * kHistThreads) {
+    // four independent 128-bit loads in flight per thread; the loop condition is the same for the lanes of a warp
+    for (; (v - lane) + 31 + 3 * kHistThreads < v1; v += 4 * kHistThreads) {
       float4 a[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * kHistThreads);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) bad |= hist_add4(my, a[u]);
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, hist_add4(my, a[u]));
+        top = m > top ? m : top;
+        if (lane == 0) row_max[(v - u0 + u * kHistThreads) >> 5] = m;
+      }
     }
-    for (; v < v1; v += kHistThreads) bad |= hist_add4(my, __ldg(xv + v));
+    for (; v - lane < v1; v += kHistThreads) {  // rows that may end inside the warp
+      const bool on = v < v1;
+      const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, on ? hist_add4(my, __ldg(xv + v)) : 0u);
+      top = m > top ? m : top;
+      if (lane == 0) row_max[(v - u0) >> 5] = m;
+    }
     // ragged tail of the client (d not a multiple of 4)
     if (u1 == units && threadIdx.x < (d & 3)) {
       const uint32_t k0 = __float_as_uint(x[(nvec << 2) + threadIdx.x]) & 0x7FFFFFFFu;
-      bad |= (k0 >= 0x7F800000u);
+      top = k0 > top ? k0 : top;
       atomicAdd(my + (k0 >> 19), 1u);
     }
-    if (bad) atomicOr(nonfinite_all + c, 1u);
+    if (top >= 0x7F800000u) atomicOr(nonfinite_all + c, 1u);  // a key of exponent 255: Inf or NaN
     __syncthreads();
     // merge into the client's histogram and keep this segment's own counts (segment = chunk + client):
     // the selection kernel derives its output offsets from them
@@ -162,7 +178,14 @@ __device__ __forceinline__ double energy_E(uint64_t Z, double beta, double D) {
 // K2  planner: one CTA of 1024 threads
 // ===================================================================================
 
-constexpr int kPlanThreads = 1024;
+constexpr int kPlanThreads = 1024;  // the fit kernel: one thread per four histogram bins
+// The tuning kernel evaluates up to kPlanItems (evaluation, length) items per round with kTuneThreads threads (an item
+// is a chain of about 175 dependent FP64 operations) and leaves most of its SM to the kernels that run next to it:
+// measured on the 100-client benchmark, 256 threads take 0.84 ms instead of 0.62 ms with 512 or 1024, all of it hidden
+// behind selection and ranking, and slow those down the least.
+constexpr int kTuneThreads = 256;
+constexpr int kPlanItems = 1024;
+constexpr int kPairSlots = (496 + kTuneThreads - 1) / kTuneThreads;  // pairs of a sweep a thread looks at
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
 // scratch of the length-tuning loop (lives in the dynamic shared memory of the fit points)
@@ -216,28 +239,81 @@ struct PlanTab {
   double QY[32];      // PQ error factor Q(Y[i]) = cap / (2^y - 1)^2
 };
 
+// candidate lengths: g(y) > 0 (the paper's B > (Q+1)/2) and not dominated; called by one full warp
+__device__ __forceinline__ void build_plan_tab(PlanTab& T, const Shape& shape, double B_in, int lane) {
+  const uint32_t y = lane + 1;
+  const double B = B_in;
+  const bool in_range = y <= shape.max_code_bits;
+  const uint32_t cap_y = in_range ? shape.cap[y] : 0u;
+  double Q;  // error factor of cap(y) values at y bits (Appendix, case study)
+  if (shape.quantizer == CVLC_QUANT_QSGD) {
+    // min(P / s_q^2, sqrt(P) / s_q), s_q = 2^(y-1) - 1 levels beside the sign bit; one bit holds no level
+    const double sq = (double)((1ull << (y - 1)) - 1ull);
+    const double Q1 = __ddiv_rn((double)cap_y, __dmul_rn(sq, sq));
+    const double Q2 = __ddiv_rn(__dsqrt_rn((double)cap_y), sq);
+    Q = (y < 2) ? CUDART_INF : ((Q1 < Q2) ? Q1 : Q2);
+  } else {
+    const double L = (double)((1ull << y) - 1ull);  // PQ: P / (2^y - 1)^2
+    Q = __ddiv_rn((double)cap_y, __dmul_rn(L, L));
+  }
+  const double one_m = __dsub_rn(1.0, __ddiv_rn(1.0, B));
+  const double g = __dsub_rn(1.0, __dadd_rn(__ddiv_rn(Q, __dmul_rn(B, B)), __dmul_rn(one_m, one_m)));
+  unsigned member;
+  uint32_t y_min;
+  if (shape.fixed_y) {
+    y_min = shape.fixed_y;
+    member = 1u << (shape.fixed_y - 1);
+  } else {
+    const unsigned pos = __ballot_sync(kFull, in_range && g > 0.0);
+    y_min = pos ? (uint32_t)__ffs(pos) : 1u;  // the host has checked that one exists
+    const uint32_t cap_next = __shfl_down_sync(kFull, cap_y, 1);
+    const bool keep = in_range && y >= y_min && (y == shape.max_code_bits || cap_y > cap_next);
+    member = __ballot_sync(kFull, keep);
+  }
+  if (member & (1u << lane)) {
+    const int i = __popc(member & ((1u << lane) - 1u));
+    T.Y[i] = y;
+    T.capY[i] = cap_y;
+    T.gY[i] = g;
+    T.QY[i] = Q;
+  }
+  if (lane == 0) {
+    T.d = shape.d;
+    T.s = shape.s;
+    T.R = shape.R;
+    T.nY = (uint32_t)__popc(member);
+    T.y_min = y_min;
+    T.fixed_y = shape.fixed_y;
+  }
+}
+
+// K2a  per client: survival counts, exponent fit, the threshold bin of the selection and the candidates per segment.
+// Everything here depends on the histogram alone.  The number of transmitted coordinates k is not known before the
+// lengths are tuned, but it never exceeds k_sel = R * cap(shortest candidate length) (every packet at the shortest
+// code; with a fixed length, exactly R * cap(y)), so the selection keeps every coordinate down to the bin that holds
+// rank min(k_sel, d): a superset of the top k whose first k ranks are the top k.
 template <int CAP>
 __global__ void __launch_bounds__(kPlanThreads, 1)
-k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restrict__ nonfinite_all,
-       const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
-       const __grid_constant__ Partition part, unsigned char* ws, int have_segments) {
+k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __restrict__ nonfinite_all,
+           const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape,
+           const __grid_constant__ Partition part, unsigned char* ws, int have_segments) {
   extern __shared__ unsigned char smem_raw[];
   unsigned long long* Nsuf = reinterpret_cast<unsigned long long*>(smem_raw);  // [4096] survival counts
   double* ptX = reinterpret_cast<double*>(smem_raw + 4096 * 8);                // fit points, ascending bin
   double* ptY = ptX + 4096;
   __shared__ PlanShared S;
   __shared__ PlanTab T;
-  __shared__ uint32_t s_thresh_bin, s_top_bin;
+  __shared__ uint32_t s_thresh_bin;
   int32_t* ws_status = reinterpret_cast<int32_t*>(ws);
 
   // blockIdx.x = client
   const unsigned long long* __restrict__ hist = hist_all + (size_t)blockIdx.x * CVLC_HIST_BINS;
-  const uint32_t* __restrict__ nonfinite = nonfinite_all + blockIdx.x;
+  const uint32_t nonfinite = nonfinite_all[blockIdx.x];
   cvlc_plan_t* __restrict__ plan = batch.c[blockIdx.x].plan;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  if (*nonfinite & 2u) {  // a histogram from outside whose counts do not add up to d
+  if (nonfinite & 2u) {  // a histogram from outside whose counts do not add up to d (its tuning key stays zero: no tuning)
     if (tid == 0) {
       plan->status = CVLC_ERR_INVALID_ARG;
       set_status(ws_status, CVLC_ERR_INVALID_ARG);
@@ -245,54 +321,10 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     return;
   }
 
-  // ---- candidate lengths: g(y) > 0 (the paper's B > (Q+1)/2) and not dominated --------
-  if (warp == 0) {
-    const uint32_t y = lane + 1;
-    const double B = batch.c[blockIdx.x].scale_B;
-    const bool in_range = y <= shape.max_code_bits;
-    const uint32_t cap_y = in_range ? shape.cap[y] : 0u;
-    double Q;  // error factor of cap(y) values at y bits (Appendix, case study)
-    if (shape.quantizer == CVLC_QUANT_QSGD) {
-      // min(P / s_q^2, sqrt(P) / s_q), s_q = 2^(y-1) - 1 levels beside the sign bit; one bit holds no level
-      const double sq = (double)((1ull << (y - 1)) - 1ull);
-      const double Q1 = __ddiv_rn((double)cap_y, __dmul_rn(sq, sq));
-      const double Q2 = __ddiv_rn(__dsqrt_rn((double)cap_y), sq);
-      Q = (y < 2) ? CUDART_INF : ((Q1 < Q2) ? Q1 : Q2);
-    } else {
-      const double L = (double)((1ull << y) - 1ull);  // PQ: P / (2^y - 1)^2
-      Q = __ddiv_rn((double)cap_y, __dmul_rn(L, L));
-    }
-    const double one_m = __dsub_rn(1.0, __ddiv_rn(1.0, B));
-    const double g = __dsub_rn(1.0, __dadd_rn(__ddiv_rn(Q, __dmul_rn(B, B)), __dmul_rn(one_m, one_m)));
-    unsigned member;
-    uint32_t y_min;
-    if (shape.fixed_y) {
-      y_min = shape.fixed_y;
-      member = 1u << (shape.fixed_y - 1);
-    } else {
-      const unsigned pos = __ballot_sync(kFull, in_range && g > 0.0);
-      y_min = pos ? (uint32_t)__ffs(pos) : 1u;  // the host has checked that one exists
-      const uint32_t cap_next = __shfl_down_sync(kFull, cap_y, 1);
-      const bool keep = in_range && y >= y_min && (y == shape.max_code_bits || cap_y > cap_next);
-      member = __ballot_sync(kFull, keep);
-    }
-    if (member & (1u << lane)) {
-      const int i = __popc(member & ((1u << lane) - 1u));
-      T.Y[i] = y;
-      T.capY[i] = cap_y;
-      T.gY[i] = g;
-      T.QY[i] = Q;
-    }
-    if (lane == 0) {
-      T.d = shape.d;
-      T.s = shape.s;
-      T.R = shape.R;
-      T.nY = (uint32_t)__popc(member);
-      T.y_min = y_min;
-      T.fixed_y = shape.fixed_y;
-    }
-  }
+  if (warp == 0) build_plan_tab(T, shape, batch.c[blockIdx.x].scale_B, lane);
   __syncthreads();
+
+  // ---- survival counts N_j = #{bin >= j} ------------------------------------------
 
   // ---- survival counts N_j = #{bin >= j} ------------------------------------------
   unsigned long long h[4];
@@ -384,16 +416,153 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
     S.alpha_q = -1.0;
   }
   __syncthreads();
+
+  // ---- selection threshold: the bin that holds rank min(k_sel, d) (1-based), how many coordinates sit in it
+  // or above, and the highest non-empty bin
+  unsigned long long k_sel = (unsigned long long)T.R * T.capY[0];
+  if (k_sel > T.d) k_sel = T.d;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int j = 4 * tid + i;
+    const unsigned long long N = Nsuf[j];
+    const unsigned long long Nn = (j == CVLC_HIST_BINS - 1) ? 0ull : Nsuf[j + 1];
+    if (N >= k_sel && Nn < k_sel) {
+      plan->thresh_bin = (uint32_t)j;
+      plan->n_candidates = N;
+      s_thresh_bin = (uint32_t)j;
+    }
+    if (N > 0 && Nn == 0) plan->top_bin = (uint32_t)j;
+  }
   if (tid == 0) {
-    const double beta = __dadd_rn(__dmul_rn(2.0, S.alpha_q), 1.0);
+    const double aq = S.alpha_q;
+    plan->status = nonfinite ? CVLC_ERR_NONFINITE_INPUT : CVLC_OK;
+    if (nonfinite) set_status(ws_status, CVLC_ERR_NONFINITE_INPUT);
+    plan->s = T.s;
+    plan->R = T.R;
+    plan->y_min = T.y_min;
+    plan->n_lengths = T.nY;
+    plan->k = 0;
+    plan->alpha = S.alpha;
+    plan->alpha_q = aq;
+    plan->beta = __dadd_rn(__dmul_rn(2.0, aq), 1.0);
+    plan->gamma = 0.0;
+    plan->B_next = 0.0;
+    for (int y = 0; y <= CVLC_MAX_CODE_BITS; ++y) {
+      plan->n_y[y] = 0;
+      plan->cap[y] = shape.cap[y];
+    }
+    // clients with the same quantised exponent and the same scale get the same lengths
+    unsigned long long* key = reinterpret_cast<unsigned long long*>(ws + plan_off_keys(batch.n)) + 2 * (size_t)blockIdx.x;
+    key[0] = (unsigned long long)__double_as_longlong(aq);
+    key[1] = (unsigned long long)__double_as_longlong(batch.c[blockIdx.x].scale_B);
+  }
+  __syncthreads();
+
+  // candidates per segment of this client (segment = part of the client inside one block's chunk of
+  // the histogram / selection kernels) and their exclusive prefix: the selection kernel's offsets.
+  // A plan made from a histogram alone has no segments; its workspace header stays unmarked.
+
+  if (have_segments) {
+    const uint32_t c = blockIdx.x;
+    const uint32_t S = part.max_segments;
+    uint32_t* seg_count = reinterpret_cast<uint32_t*>(ws + plan_off_seg_count(batch.n));
+    unsigned long long* seg_prefix = reinterpret_cast<unsigned long long*>(ws + plan_off_seg_prefix(batch.n, S));
+    const uint64_t row_tiles = row_tiles_total(part);
+    const uint32_t* seg_hist = reinterpret_cast<const uint32_t*>(ws + plan_off_seg_hist(batch.n, S, row_tiles));
+    const uint64_t first = (uint64_t)c * part.units, last = first + part.units - 1;
+    const uint32_t b0 = (uint32_t)(first / part.chunk), b1 = (uint32_t)(last / part.chunk);
+    const uint32_t jt = s_thresh_bin;
+    for (uint32_t b = b0 + warp; b <= b1; b += kPlanThreads / 32) {
+      const uint32_t* hsrc = seg_hist + ((size_t)b + c) * CVLC_HIST_BINS;
+      uint32_t sum = 0;
+      for (uint32_t j = jt + lane; j < CVLC_HIST_BINS; j += 32) sum += hsrc[j];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+      if (lane == 0) seg_count[b + c] = sum;
+    }
+    // one bit per row of 128 coordinates: does the row hold a candidate (a key at or above the threshold)?
+    // Tile t (64 rows) of a segment is one 64-bit word; lanes 2w, 2w+1 ... : a warp turns 32 rows into one half word.
+    {
+      const uint32_t* row_max = reinterpret_cast<const uint32_t*>(ws + plan_off_row_max(batch.n, S));
+      uint32_t* row_flags = reinterpret_cast<uint32_t*>(ws + plan_off_row_flags(batch.n, S, row_tiles));
+      const uint32_t thresh_key = jt << 19;
+      const uint64_t nvec = shape.d >> 2;
+      for (uint32_t b = b0; b <= b1; ++b) {
+        const uint64_t p0 = (first > (uint64_t)b * part.chunk) ? first : (uint64_t)b * part.chunk;
+        uint64_t p1 = ((uint64_t)(b + 1) * part.chunk < first + part.units) ? (uint64_t)(b + 1) * part.chunk : first + part.units;
+        if (p1 > first + nvec) p1 = first + nvec;  // the client's last unit is its ragged tail, not a float4
+        const uint64_t n_units = p1 > p0 ? p1 - p0 : 0;
+        const uint64_t n_rows = (n_units + kRowUnits - 1) / kRowUnits;
+        const uint64_t n_words = (n_rows + 31) / 32;          // half words of row flags
+        const uint64_t tile0 = seg_first_tile(p0, b + c);
+        for (uint64_t w = warp; w < ((n_words + 1) & ~(uint64_t)1); w += kPlanThreads / 32) {  // whole 64-bit words
+          const uint64_t r = w * 32 + lane;
+          const bool flag = (r < n_rows) && row_max[tile0 * kTileRows + r] >= thresh_key;
+          const unsigned bits = __ballot_sync(kFull, flag);
+          if (lane == 0) row_flags[tile0 * 2 + w] = bits;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long run = 0;
+      for (uint32_t b = b0; b <= b1; ++b) {
+        seg_prefix[b + c] = run;
+        run += seg_count[b + c];
+      }
+      if (c == 0) {
+        PlanWsHeader* hdr = reinterpret_cast<PlanWsHeader*>(ws);
+        hdr->n = batch.n;
+        hdr->d = shape.d;
+        hdr->n_chunks = part.n_chunks;
+        hdr->magic = kPlanWsMagic;
+      }
+    }
+  }
+}
+
+// K2b  code-length tuning, one CTA per client; only the first client of every tuning key does the work
+template <int CAP>
+__global__ void __launch_bounds__(kTuneThreads, 1)
+k_plan_tune(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ PlanShared S;
+  __shared__ PlanTab T;
+  __shared__ uint32_t s_leader;
+  const uint32_t c = blockIdx.x;
+  cvlc_plan_t* __restrict__ plan = batch.c[c].plan;
+  uint32_t* leader = reinterpret_cast<uint32_t*>(ws + plan_off_leader(batch.n));
+  const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(ws + plan_off_keys(batch.n));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  const unsigned long long key0 = keys[2 * (size_t)c], key1 = keys[2 * (size_t)c + 1];
+  if (tid == 0) s_leader = c;
+  __syncthreads();
+  if (key1 == 0ull) {  // no key: the fit refused this client's histogram
+    if (tid == 0) leader[c] = 0xFFFFFFFFu;
+    return;
+  }
+  for (uint32_t i = tid; i < c; i += kTuneThreads)
+    if (keys[2 * (size_t)i] == key0 && keys[2 * (size_t)i + 1] == key1) atomicMin(&s_leader, i);
+  __syncthreads();
+  if (tid == 0) leader[c] = s_leader;
+  if (s_leader != c) return;  // an earlier client of the batch tunes for this key; k_plan_finish copies its result
+
+  if (warp == 0) build_plan_tab(T, shape, batch.c[c].scale_B, lane);
+  if (tid == 0) {
+    const double aq = __longlong_as_double((long long)key0);
+    const double beta = __dadd_rn(__dmul_rn(2.0, aq), 1.0);
+    S.alpha_q = aq;
     S.beta = beta;
-    S.D = __dsub_rn(series_powr((double)T.d, beta), 1.0);
+    S.D = __dsub_rn(series_powr((double)shape.d, beta), 1.0);
   }
   if (tid < 32) S.n[tid] = 0;
   __syncthreads();
   const double beta = S.beta, D = S.D;
   const int nY = (int)T.nY;
   const uint32_t my_cap = (lane < nY) ? T.capY[lane] : 0u;
+  double* ptX = reinterpret_cast<double*>(smem_raw);  // the solver's scratch
+
 
   // ---- objective bookkeeping -----------------------------------------------------------
   // F(n) = 1 - gamma of Eq. (5) is a running sum over the used lengths, longest first:
@@ -523,57 +692,65 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                 j = u - (r - 1) * r / 2;
                 return true;
               };
+              // a thread looks at the pairs t = tid, tid + kTuneThreads, ...; the scan runs over t in order
               const unsigned used = Q.used;
-              int pi = 0, pj = 0;
-              const bool valid = pair_at(tid, pi, pj);
-              uint32_t X = 0;
-              unsigned need = 0;
-              int m = 0;
-              if (valid) {
-                X = S.n[pi] + S.n[pj];
-                if (X > 0) {
-                  need = (used | (1u << pi) | (1u << pj)) & (0xFFFFFFFFu >> (31 - pi));
-                  m = __popc(need);
-                }
-              }
-              const bool flag = valid && X > 0;
-              uint32_t incl = flag ? ((1u << 16) | (uint32_t)(2 * m)) : 0u;  // items stay below 2^16: 496 pairs of at most 64
-#pragma unroll
-              for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t o = __shfl_up_sync(kFull, incl, off);
-                if (lane >= off) incl += o;
-              }
-              if (lane == 31) Q.col_warp[warp] = incl;
               if (tid == 0) {
                 Q.col_nops = 0;
                 Q.col_last = -1;
                 Q.col_first_left = 0x7FFFFFFF;
               }
-              __syncthreads();
-              {
-                const uint32_t wt = Q.col_warp[lane];
-                uint32_t wi = wt;
+              uint32_t carry = 0;
+#pragma unroll
+              for (int slot = 0; slot < kPairSlots; ++slot) {
+                const int t = slot * kTuneThreads + tid;
+                int pi = 0, pj = 0;
+                const bool valid = pair_at(t, pi, pj);
+                uint32_t X = 0;
+                unsigned need = 0;
+                int m = 0;
+                if (valid) {
+                  X = S.n[pi] + S.n[pj];
+                  if (X > 0) {
+                    need = (used | (1u << pi) | (1u << pj)) & (0xFFFFFFFFu >> (31 - pi));
+                    m = __popc(need);
+                  }
+                }
+                const bool flag = valid && X > 0;
+                uint32_t incl = flag ? ((1u << 16) | (uint32_t)(2 * m)) : 0u;  // items stay below 2^16: 496 pairs of at most 64
 #pragma unroll
                 for (int off = 1; off < 32; off <<= 1) {
-                  const uint32_t o = __shfl_up_sync(kFull, wi, off);
-                  if (lane >= off) wi += o;
+                  const uint32_t o = __shfl_up_sync(kFull, incl, off);
+                  if (lane >= off) incl += o;
                 }
-                incl += __shfl_sync(kFull, wi - wt, warp);
-              }
-              const int rank = (int)(incl >> 16) - 1;
-              const bool taken = flag && rank < kMaxBatchOps && (incl & 0xFFFFu) <= (uint32_t)kPlanThreads;
-              if (taken) {
-                PlanOp& o = Q.op[rank];
-                o.i = pi; o.j = pj; o.X = X; o.na0 = S.n[pi]; o.lo = 0; o.hi = X; o.m = m; o.F_final = 0.0;
-                for (unsigned rest_bits = need; rest_bits;) {  // the lengths a trial evaluates, longest first
-                  const int l = 31 - __clz(rest_bits);
-                  rest_bits ^= 1u << l;
-                  o.slot_lane[l == 31 ? 0 : __popc(need >> (l + 1))] = (unsigned char)l;
+                if (lane == 31) Q.col_warp[warp] = incl;
+                __syncthreads();
+                {
+                  const uint32_t wt = (lane < kTuneThreads / 32) ? Q.col_warp[lane] : 0u;
+                  uint32_t wi = wt;
+#pragma unroll
+                  for (int off = 1; off < 32; off <<= 1) {
+                    const uint32_t o = __shfl_up_sync(kFull, wi, off);
+                    if (lane >= off) wi += o;
+                  }
+                  incl += carry + __shfl_sync(kFull, wi - wt, warp);
+                  carry += __shfl_sync(kFull, wi, 31);
                 }
-                atomicMax(&Q.col_nops, rank + 1);
-                atomicMax(&Q.col_last, tid);
-              } else if (flag) {
-                atomicMin(&Q.col_first_left, tid);
+                const int rank = (int)(incl >> 16) - 1;
+                const bool taken = flag && rank < kMaxBatchOps && (incl & 0xFFFFu) <= (uint32_t)kPlanItems;
+                if (taken) {
+                  PlanOp& o = Q.op[rank];
+                  o.i = pi; o.j = pj; o.X = X; o.na0 = S.n[pi]; o.lo = 0; o.hi = X; o.m = m; o.F_final = 0.0;
+                  for (unsigned rest_bits = need; rest_bits;) {  // the lengths a trial evaluates, longest first
+                    const int l = 31 - __clz(rest_bits);
+                    rest_bits ^= 1u << l;
+                    o.slot_lane[l == 31 ? 0 : __popc(need >> (l + 1))] = (unsigned char)l;
+                  }
+                  atomicMax(&Q.col_nops, rank + 1);
+                  atomicMax(&Q.col_last, t);
+                } else if (flag) {
+                  atomicMin(&Q.col_first_left, t);
+                }
+                if (slot + 1 < kPairSlots) __syncthreads();  // the warp totals are reused by the next slot
               }
               __syncthreads();
               const int n_ops = Q.col_nops;
@@ -625,7 +802,7 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                 int depth = 0;
 #pragma unroll
                 for (int q = 0; q < 9; ++q) {
-                  if (items_at[q] <= kPlanThreads && depth == q) depth = q + 1;  // the sums grow with the depth
+                  if (items_at[q] <= kPlanItems && depth == q) depth = q + 1;  // the sums grow with the depth
                 }
                 const int lv = need_levels < depth ? need_levels : depth;
                 const int ne = lv ? 2 * ((1 << lv) - 1) : 0;
@@ -657,18 +834,18 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
               __syncthreads();
               if (Q.unfinished == 0) break;
               // phase 1: energies, one thread per (operation, evaluation, slot)
-              int a = -1, e = 0, sl = 0;
-              uint32_t t = 0xFFFFFFFFu;
-              if (tid < Q.n_items) {
-                // the operation whose item range holds this thread: first a with tid < item_end[a]
+              for (int vt = tid; vt < Q.n_items; vt += kTuneThreads) {
+                int a = -1, e = 0, sl = 0;
+                uint32_t t = 0xFFFFFFFFu;
+                // the operation whose item range holds this item: first a with vt < item_end[a]
                 int lo_a = 0, hi_a = 31;
                 while (lo_a < hi_a) {
                   const int mid = (lo_a + hi_a) >> 1;
-                  if (tid < Q.item_end[mid]) hi_a = mid; else lo_a = mid + 1;
+                  if (vt < Q.item_end[mid]) hi_a = mid; else lo_a = mid + 1;
                 }
                 a = lo_a;
                 const PlanOp& o = Q.op[a];
-                const int rel = tid - o.item_base;
+                const int rel = vt - o.item_base;
                 e = rel / o.m;
                 sl = rel - e * o.m;
                 const int hnode = (e >> 1) + 1;
@@ -687,7 +864,7 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   // pair's current share, plus the trial's
                   uint64_t W = Q.Wc[l] - (uint64_t)S.n[o.i] * T.capY[o.i] + (uint64_t)t * T.capY[o.i];
                   if (l <= o.j) W = W - (uint64_t)S.n[o.j] * T.capY[o.j] + (uint64_t)(o.X - t) * T.capY[o.j];
-                  Q.Ev[tid] = energy_E(W, beta, D);
+                  Q.Ev[vt] = energy_E(W, beta, D);
                 }
                 if (sl == 0) {
                   Q.tv[o.eval_base + e] = t;
@@ -699,11 +876,11 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
               // g_l * (E_l - E_prev) in the order of the lengths; only the lengths i and j can be unused in a trial
               // (no term, and the next term's E_prev skips them).  The terms do not depend on the sum, so they are
               // worked out four at a time ahead of the ordered additions.
-              if (tid < Q.n_evals) {
-                const PlanOp& o = Q.op[Q.ea[tid]];
-                const uint32_t tt = Q.tv[tid];
+              for (int vt = tid; vt < Q.n_evals; vt += kTuneThreads) {
+                const PlanOp& o = Q.op[Q.ea[vt]];
+                const uint32_t tt = Q.tv[vt];
                 if (tt != 0xFFFFFFFFu) {
-                  const int ee = tid - o.eval_base;
+                  const int ee = vt - o.eval_base;
                   const double* Ez = Q.Ev + o.item_base + ee * o.m;
                   double F = Q.Fpre[o.i + 1];
                   double Eprev = Q.Eab[o.i + 1];
@@ -732,7 +909,7 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
                   }
                   const uint64_t Wtot = Q.Wc[0] - (uint64_t)S.n[o.i] * T.capY[o.i] - (uint64_t)S.n[o.j] * T.capY[o.j] +
                                         (uint64_t)tt * T.capY[o.i] + (uint64_t)(o.X - tt) * T.capY[o.j];
-                  Q.Fv[tid] = (Wtot > T.d) ? -CUDART_INF : F;
+                  Q.Fv[vt] = (Wtot > T.d) ? -CUDART_INF : F;
                 }
               }
               __syncthreads();
@@ -801,84 +978,37 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
   }
 
   // ---- outputs ---------------------------------------------------------------------
-  unsigned long long k = 0;
-  for (int i = 0; i < nY; ++i) k += (unsigned long long)S.n[i] * T.capY[i];
   if (tid == 0) {
+    unsigned long long k = 0;
     double Qmax = 0.0;
-    for (int i = 0; i < nY; ++i)
+    for (int i = 0; i < nY; ++i) {
+      k += (unsigned long long)S.n[i] * T.capY[i];
       if (S.n[i] > 0 && T.QY[i] > Qmax) Qmax = T.QY[i];
-    plan->status = (*nonfinite) ? CVLC_ERR_NONFINITE_INPUT : CVLC_OK;
-    if (*nonfinite) set_status(ws_status, CVLC_ERR_NONFINITE_INPUT);
-    plan->s = T.s;
-    plan->R = T.R;
-    plan->y_min = T.y_min;
-    plan->n_lengths = T.nY;
+    }
     plan->k = k;
-    plan->alpha = S.alpha;
-    plan->alpha_q = S.alpha_q;
-    plan->beta = beta;
     plan->gamma = __dsub_rn(1.0, Q.Fpre[0]);
     plan->B_next = __dadd_rn(1.0, Qmax);
-    for (int y = 0; y <= CVLC_MAX_CODE_BITS; ++y) {
-      plan->n_y[y] = 0;
-      plan->cap[y] = shape.cap[y];
-    }
     for (int i = 0; i < nY; ++i) plan->n_y[T.Y[i]] = S.n[i];
   }
-  // threshold bin: the bin that holds rank k (1-based), how many coordinates sit in it or above,
-  // and the highest non-empty bin
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int j = 4 * tid + i;
-    const unsigned long long N = Nsuf[j];
-    const unsigned long long Nn = (j == CVLC_HIST_BINS - 1) ? 0ull : Nsuf[j + 1];
-    if (N >= k && Nn < k) {
-      plan->thresh_bin = (uint32_t)j;
-      plan->n_candidates = N;
-      s_thresh_bin = (uint32_t)j;
-    }
-    if (N > 0 && Nn == 0) {
-      plan->top_bin = (uint32_t)j;
-      s_top_bin = (uint32_t)j;
-    }
-  }
-  __syncthreads();
+}
 
-  // candidates per segment of this client (segment = part of the client inside one block's chunk of
-  // the histogram / selection kernels) and their exclusive prefix: the selection kernel's offsets.
-  // A plan made from a histogram alone has no segments; its workspace header stays unmarked.
-  if (have_segments) {
-    const uint32_t c = blockIdx.x;
-    const uint32_t S = part.max_segments;
-    uint32_t* seg_count = reinterpret_cast<uint32_t*>(ws + plan_off_seg_count(batch.n));
-    unsigned long long* seg_prefix = reinterpret_cast<unsigned long long*>(ws + plan_off_seg_prefix(batch.n, S));
-    const uint32_t* seg_hist = reinterpret_cast<const uint32_t*>(ws + plan_off_seg_hist(batch.n, S));
-    const uint64_t first = (uint64_t)c * part.units, last = first + part.units - 1;
-    const uint32_t b0 = (uint32_t)(first / part.chunk), b1 = (uint32_t)(last / part.chunk);
-    const uint32_t jt = s_thresh_bin;
-    for (uint32_t b = b0 + warp; b <= b1; b += kPlanThreads / 32) {
-      const uint32_t* hsrc = seg_hist + ((size_t)b + c) * CVLC_HIST_BINS;
-      uint32_t sum = 0;
-      for (uint32_t j = jt + lane; j < CVLC_HIST_BINS; j += 32) sum += hsrc[j];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
-      if (lane == 0) seg_count[b + c] = sum;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      unsigned long long run = 0;
-      for (uint32_t b = b0; b <= b1; ++b) {
-        seg_prefix[b + c] = run;
-        run += seg_count[b + c];
-      }
-      if (c == 0) {
-        PlanWsHeader* hdr = reinterpret_cast<PlanWsHeader*>(ws);
-        hdr->n = batch.n;
-        hdr->d = shape.d;
-        hdr->n_chunks = part.n_chunks;
-        hdr->magic = kPlanWsMagic;
-      }
-    }
+// K2c  the clients that share a tuning key take the lengths of the client that tuned for it
+template <int CAP>
+__global__ void __launch_bounds__(256)
+k_plan_finish(const __grid_constant__ BatchDesc<CAP> batch, const unsigned char* ws) {
+  const uint32_t c = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (c >= batch.n) return;
+  const uint32_t l = reinterpret_cast<const uint32_t*>(ws + plan_off_leader(batch.n))[c];
+  if (l == 0xFFFFFFFFu || l == c || l >= batch.n) return;
+  cvlc_plan_t* dst = batch.c[c].plan;
+  const cvlc_plan_t* src = batch.c[l].plan;
+  dst->n_y[lane] = src->n_y[lane];
+  if (lane == 0) {
+    dst->n_y[CVLC_MAX_CODE_BITS] = src->n_y[CVLC_MAX_CODE_BITS];
+    dst->k = src->k;
+    dst->gamma = src->gamma;
+    dst->B_next = src->B_next;
   }
 }
 
@@ -886,9 +1016,11 @@ k_plan(const unsigned long long* __restrict__ hist_all, const uint32_t* __restri
 // launchers
 // ===================================================================================
 
+constexpr size_t kFitSmem = 3 * 4096 * 8;  // survival counts and the fit points
+constexpr size_t kTuneSmem = (sizeof(PlanSolver) + 255) & ~(size_t)255;
+
 template <int CAP>
-static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
-                                 unsigned long long* hist_out, cudaStream_t st) {
+static cudaError_t plan_attributes() {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -896,29 +1028,47 @@ static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Sh
   if (dev >= 0 && dev < 64 && !attr_done[dev]) {
     e = cudaFuncSetAttribute(k_hist<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSub * CVLC_HIST_BINS * 4);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_plan<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
+    e = cudaFuncSetAttribute(k_plan_fit<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFitSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_plan_tune<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTuneSmem);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
-  BatchDesc<CAP> batch;
+  return cudaSuccess;
+}
+
+template <int CAP>
+static void fill_batch(BatchDesc<CAP>& batch, const ClientDesc* clients, uint32_t n) {
   batch.n = n;
   batch.pad = 0;
   for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
+}
+
+// histogram of every client, then (unless only the histograms are wanted) fit, threshold and segment tables
+template <int CAP>
+static cudaError_t launch_plan_front_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
+                                       unsigned long long* hist_out, cudaStream_t st) {
+  cudaError_t e = plan_attributes<CAP>();
+  if (e != cudaSuccess) return e;
+  BatchDesc<CAP> batch;
+  fill_batch(batch, clients, n);
   unsigned char* w = static_cast<unsigned char*>(ws);
   unsigned long long* hist = reinterpret_cast<unsigned long long*>(w + kPlanWsHist);
   uint32_t* flags = reinterpret_cast<uint32_t*>(w + plan_off_flags(n));
   const Partition part = make_partition(shape.d, n);
-  uint32_t* seg_hist = reinterpret_cast<uint32_t*>(w + plan_off_seg_hist(n, part.max_segments));
+  const uint64_t row_tiles = row_tiles_total(part);
+  uint32_t* seg_hist = reinterpret_cast<uint32_t*>(w + plan_off_seg_hist(n, part.max_segments, row_tiles));
+  uint32_t* row_max = reinterpret_cast<uint32_t*>(w + plan_off_row_max(n, part.max_segments));
   {
-    // header, histograms, flags and segment tables start at zero; the per-segment histograms are
-    // written in full by the histogram kernel
+    // header, histograms, flags, tuning keys and segment tables start at zero; the per-segment histograms and the
+    // rows' maxima are written in full by the histogram kernel
     LaunchScope ls(kKZeroWords, st);
-    k_zero_words<<<2 * kNumSM, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), plan_off_seg_hist(n, part.max_segments) / 4);
+    k_zero_words<<<2 * kNumSM, 1024, 0, st>>>(reinterpret_cast<uint32_t*>(w), plan_off_row_max(n, part.max_segments) / 4);
   }
   {
     // two resident blocks per SM share the concatenated updates evenly
     LaunchScope ls(kKHist, st);
-    k_hist<CAP><<<part.grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, part, hist, flags, seg_hist);
+    k_hist<CAP><<<part.grid, kHistThreads, kHistSub * CVLC_HIST_BINS * 4, st>>>(batch, shape.d, part, hist, flags, seg_hist, row_max);
   }
   if (hist_out) {
     // the histograms alone: what a client sends when the parameter server plans for it.  The workspace
@@ -928,21 +1078,50 @@ static cudaError_t launch_plan_t(const ClientDesc* clients, uint32_t n, const Sh
     return cudaMemcpyAsync(hist_out, hist, (size_t)n * CVLC_HIST_BINS * 8, cudaMemcpyDeviceToDevice, st);
   }
   {
-    LaunchScope ls(kKPlan, st);
-    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w, 1);
+    LaunchScope ls(kKPlanFit, st);
+    k_plan_fit<CAP><<<n, kPlanThreads, kFitSmem, st>>>(hist, flags, batch, shape, part, w, 1);
   }
   return cudaGetLastError();
 }
 
+template <int CAP>
+static cudaError_t launch_plan_back_t(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
+  cudaError_t e = plan_attributes<CAP>();
+  if (e != cudaSuccess) return e;
+  BatchDesc<CAP> batch;
+  fill_batch(batch, clients, n);
+  unsigned char* w = static_cast<unsigned char*>(ws);
+  {
+    LaunchScope ls(kKPlanTune, st);
+    k_plan_tune<CAP><<<n, kTuneThreads, kTuneSmem, st>>>(batch, shape, w);
+  }
+  {
+    LaunchScope ls(kKPlanFinish, st);
+    k_plan_finish<CAP><<<(n + 7) / 8, 256, 0, st>>>(batch, w);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plan_front(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_front_t<kSmallBatch>(clients, n, shape, ws, nullptr, st);
+  return launch_plan_front_t<kLargeBatch>(clients, n, shape, ws, nullptr, st);
+}
+
+cudaError_t launch_plan_back(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_back_t<kSmallBatch>(clients, n, shape, ws, st);
+  return launch_plan_back_t<kLargeBatch>(clients, n, shape, ws, st);
+}
+
 cudaError_t launch_plan(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws, cudaStream_t st) {
-  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, nullptr, st);
-  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, nullptr, st);
+  const cudaError_t e = launch_plan_front(clients, n, shape, ws, st);
+  if (e != cudaSuccess) return e;
+  return launch_plan_back(clients, n, shape, ws, st);
 }
 
 cudaError_t launch_histogram(const ClientDesc* clients, uint32_t n, const Shape& shape, void* ws,
                              unsigned long long* hist_out, cudaStream_t st) {
-  if (n <= (uint32_t)kSmallBatch) return launch_plan_t<kSmallBatch>(clients, n, shape, ws, hist_out, st);
-  return launch_plan_t<kLargeBatch>(clients, n, shape, ws, hist_out, st);
+  if (n <= (uint32_t)kSmallBatch) return launch_plan_front_t<kSmallBatch>(clients, n, shape, ws, hist_out, st);
+  return launch_plan_front_t<kLargeBatch>(clients, n, shape, ws, hist_out, st);
 }
 
 // Checks histograms that come from outside: flag bit 0 = a value of exponent 255 (Inf, NaN),
@@ -974,37 +1153,34 @@ k_hist_check(const unsigned long long* __restrict__ hist_all, uint64_t d, uint32
 template <int CAP>
 static cudaError_t launch_plan_from_hist_t(const ClientDesc* clients, uint32_t n, const Shape& shape,
                                            const unsigned long long* hist, void* ws, cudaStream_t st) {
-  static bool attr_done[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  cudaError_t e = plan_attributes<CAP>();
   if (e != cudaSuccess) return e;
-  if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-    e = cudaFuncSetAttribute(k_plan<CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * 4096 * 8);
-    if (e != cudaSuccess) return e;
-    attr_done[dev] = true;
-  }
   BatchDesc<CAP> batch;
-  batch.n = n;
-  batch.pad = 0;
-  for (uint32_t i = 0; i < n; ++i) batch.c[i] = clients[i];
+  fill_batch(batch, clients, n);
   unsigned char* w = static_cast<unsigned char*>(ws);
   uint32_t* flags = reinterpret_cast<uint32_t*>(w + plan_off_flags(n));
   const Partition part = make_partition(shape.d, n);
   {
-    // status word and header start at zero: the header stays unmarked, so an encode call cannot take
-    // this workspace for one that holds segment tables
+    // status word, header, tuning keys and leaders start at zero: the header stays unmarked, so an encode call
+    // cannot take this workspace for one that holds segment tables
     LaunchScope ls(kKZeroWords, st);
     k_zero_words<<<1, 64, 0, st>>>(reinterpret_cast<uint32_t*>(w), kPlanWsHist / 4);
+  }
+  {
+    LaunchScope ls(kKZeroWords, st);
+    k_zero_words<<<8, 256, 0, st>>>(reinterpret_cast<uint32_t*>(w + plan_off_keys(n)), (plan_off_seg_count(n) - plan_off_keys(n)) / 4);
   }
   {
     LaunchScope ls(kKHistCheck, st);
     k_hist_check<<<n, 256, 0, st>>>(hist, shape.d, flags);
   }
   {
-    LaunchScope ls(kKPlan, st);
-    k_plan<CAP><<<n, kPlanThreads, 3 * 4096 * 8, st>>>(hist, flags, batch, shape, part, w, 0);
+    LaunchScope ls(kKPlanFit, st);
+    k_plan_fit<CAP><<<n, kPlanThreads, kFitSmem, st>>>(hist, flags, batch, shape, part, w, 0);
   }
-  return cudaGetLastError();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_plan_back_t<CAP>(clients, n, shape, ws, st);
 }
 
 cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const Shape& shape,

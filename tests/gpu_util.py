@@ -73,16 +73,24 @@ def oracle_encode_clients(workload_name: str, clients: Sequence[int], d: Optiona
 # ---- GPU side ----------------------------------------------------------------------------
 
 def gpu_plan_encode(x: np.ndarray, pd: dict, fixed_y: int = 0, device: str = "cuda:0", want_hist: bool = False,
-                    use_plan_ws: bool = True):
-    """returns (CvlcPlan host copy, stream np.uint8[, histogram np.uint64])"""
+                    use_plan_ws: bool = True, compress: int = 0):
+    """returns (status, CvlcPlan host copy, stream np.uint8[, histogram np.uint64]).
+    compress: 0 = cvlc_plan then cvlc_encode; 1 = cvlc_compress_batch on one stream; 2 = with a side stream"""
     import torch
     from paper_2402_03770_b200 import binding as B
     dev = torch.device(device)
     p = gpu_params(pd)
     xd = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(dev)
-    enc = B.ClientEncoder(p, dev)
-    enc.out.fill_(0xAB)  # the encoder must write every byte of the stream
-    out = enc.run(xd, fixed_y=fixed_y, use_plan_ws=use_plan_ws)
+    if compress:
+        enc = B.BatchEncoder([p], dev)
+        enc.outs[0].fill_(0xAB)  # the encoder must write every byte of the stream
+        enc.plan = enc.plans
+        side = torch.cuda.Stream(device=dev) if compress == 2 else None
+        out = enc.compress([xd], side_stream=side, fixed_y=fixed_y)[0]
+    else:
+        enc = B.ClientEncoder(p, dev)
+        enc.out.fill_(0xAB)
+        out = enc.run(xd, fixed_y=fixed_y, use_plan_ws=use_plan_ws)
     status = enc.status()
     plan = B.read_plan(enc.plan)
     st = out.cpu().numpy().copy()

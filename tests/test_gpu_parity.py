@@ -94,16 +94,18 @@ def test_division_by_small_constants_is_correctly_rounded(torch_cuda):
 
 def run_case(x, pd, fixed_y=0):
     of, ost = oracle_plan_encode(x, pd, fixed_y)
-    # both selection kernels: offsets from the plan's per-segment counts, and the look-back scan
-    for use_plan_ws in (True, False):
-        status, gp, gst = gpu_plan_encode(x, pd, fixed_y, use_plan_ws=use_plan_ws)
-        assert status == 0, (status, use_plan_ws)
+    # both selection kernels (offsets from the plan's per-segment counts, and the look-back scan), then the
+    # one-call form on one stream and with the length tuning on a side stream
+    for use_plan_ws, compress in ((True, 0), (False, 0), (True, 1), (True, 2)):
+        status, gp, gst = gpu_plan_encode(x, pd, fixed_y, use_plan_ws=use_plan_ws, compress=compress)
+        assert status == 0, (status, use_plan_ws, compress)
         assert_plan_equal(gp, of)
+        assert gp.k <= gp.n_candidates <= pd["d"]
         assert gst.size == ost.size
         if not (gst == ost).all():
             bad = np.nonzero(gst != ost)[0]
             raise AssertionError(f"stream differs at {bad.size} bytes, first at {bad[0]} of {gst.size} "
-                                 f"(use_plan_ws={use_plan_ws})")
+                                 f"(use_plan_ws={use_plan_ws}, compress={compress})")
     return of, ost
 
 
@@ -322,8 +324,16 @@ def test_decode_rejects_malformed_streams(torch_cuda):
     bits[80:80 + 15] = 1                                                        # PID 32767 >= d
     pid_bad = st.copy()
     pid_bad[64:64 + 128] = np.packbits(bits, bitorder="little")
+    # the PQ centroid fields (bytes 2..5 minimum, 6..9 maximum of a packet): not finite, or in the wrong order
+    hi_nan = st.copy()
+    hi_nan[64 + 8:64 + 10] = [0xC0, 0x7F]
+    lo_inf = st.copy()
+    lo_inf[64 + 2:64 + 6] = [0x00, 0x00, 0x80, 0xFF]
+    swapped = st.copy()
+    swapped[64 + 2:64 + 6], swapped[64 + 6:64 + 10] = st[64 + 6:64 + 10].copy(), st[64 + 2:64 + 6].copy()
+    assert st[64 + 2:64 + 6].tobytes() != st[64 + 6:64 + 10].tobytes()
     cases = [corrupt(0, 0), corrupt(4, 2), corrupt(6, 1), corrupt(7, 3), corrupt(16, 9), corrupt(65, 33),
-             corrupt(65, 0), corrupt(64 + 128 * 5 + 1, 32), pid_bad]
+             corrupt(65, 0), corrupt(64 + 128 * 5 + 1, 32), pid_bad, hi_nan, lo_inf, swapped]
     for bad in cases:
         with pytest.raises(O.OracleError):
             O.decode_aggregate([good[0], bad, good[1]], w3, d)
@@ -332,6 +342,13 @@ def test_decode_rejects_malformed_streams(torch_cuda):
     # a stream length that disagrees with its header
     status, _ = gpu_decode_aggregate([good[0], st[:-128], good[1]], w3, d)
     assert status == B.CVLC_ERR_BAD_STREAM
+    # weights are finite and positive
+    for wbad in (np.array([1, -1, 1], np.float32), np.array([1, np.inf, 1], np.float32), np.array([0, 1, 1], np.float32)):
+        with pytest.raises(O.OracleError) as oe:
+            O.decode_aggregate([good[0], st, good[1]], wbad, d)
+        assert oe.value.code == O.ORC_ERR_INVALID_ARG
+        status, _ = gpu_decode_aggregate([good[0], st, good[1]], wbad, d)
+        assert status == B.CVLC_ERR_INVALID_ARG
     # the context is still usable
     status, out = gpu_decode_aggregate([good[0], st, good[1]], w3, d)
     assert status == 0
@@ -386,11 +403,56 @@ def test_plan_mismatch_is_detected(torch_cuda):
     enc2 = B.ClientEncoder(p2, dev)
     B.cvlc_encode(xd, p2, enc.plan, enc2.out, enc2.enc_ws)                      # plan made for another budget
     assert B.cvlc_read_status(enc2.enc_ws) == B.CVLC_ERR_PLAN_MISMATCH
-    x2 = torch.from_numpy((x * 3.0).astype(np.float32)).to(dev)                 # plan made for another update
-    B.cvlc_encode(x2, p, enc.plan, enc.out, enc.enc_ws)
-    assert B.cvlc_read_status(enc.enc_ws) in (B.CVLC_ERR_PLAN_MISMATCH, B.CVLC_OK)
-    B.cvlc_encode(xd, p, enc.plan, enc.out, enc.enc_ws)                         # and the right pairing still works
-    assert B.cvlc_read_status(enc.enc_ws) == B.CVLC_OK
+    # plan made for another update: three times the values put more coordinates above the plan's threshold,
+    # which both selection kernels notice (per-segment counts with the plan's workspace, the total without)
+    x2 = torch.from_numpy((x * 3.0).astype(np.float32)).to(dev)
+    assert int((np.abs(x * 3.0).astype(np.float32).view(np.uint32) >> 19 >= B.read_plan(enc.plan).thresh_bin).sum()) \
+        != B.read_plan(enc.plan).n_candidates
+    for plan_ws in (enc.plan_ws, None):
+        B.cvlc_encode(x2, p, enc.plan, enc.out, enc.enc_ws, plan_ws=plan_ws)
+        assert B.cvlc_read_status(enc.enc_ws) == B.CVLC_ERR_PLAN_MISMATCH
+    # code lengths that do not fill the stream's packets are refused by the packing kernel
+    plan_host = bytearray(enc.plan.cpu().numpy().tobytes())
+    tampered = B.CvlcPlan.from_buffer_copy(bytes(plan_host))
+    y_used = max(y for y in range(33) if tampered.n_y[y])
+    tampered.n_y[y_used] -= 1
+    bad_plan = torch.frombuffer(bytearray(bytes(tampered)), dtype=torch.uint8).to(dev)
+    B.cvlc_encode(xd, p, bad_plan, enc.out, enc.enc_ws, plan_ws=enc.plan_ws)
+    assert B.cvlc_read_status(enc.enc_ws) == B.CVLC_ERR_PLAN_MISMATCH
+    for plan_ws in (enc.plan_ws, None):                                         # and the right pairing still works
+        B.cvlc_encode(xd, p, enc.plan, enc.out, enc.enc_ws, plan_ws=plan_ws)
+        assert B.cvlc_read_status(enc.enc_ws) == B.CVLC_OK
+
+
+def test_bounded_wait_runs_out_without_hanging(torch_cuda):
+    """the look-back wait on a word nobody publishes gives up after its poll limit and reports DEVICE_TIMEOUT"""
+    torch = torch_cuda
+    from paper_2402_03770_b200 import binding as B
+    word = torch.zeros(1, dtype=torch.int64, device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    B.cvlc_selftest_wait(word, status, 64)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.CVLC_ERR_DEVICE_TIMEOUT
+    # a published word ends the wait at once and leaves the status alone
+    word.fill_((1 << 62) | 5)
+    status.zero_()
+    B.cvlc_selftest_wait(word, status, 64)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.CVLC_OK
+    with pytest.raises(B.CvlcError):
+        B.cvlc_selftest_wait(word, status, 0)
+
+
+def test_subnormal_threshold(torch_cuda):
+    """an update so small that the selection threshold lies among the subnormals (no flush to zero anywhere)"""
+    rng = np.random.default_rng(31)
+    d = 60_000
+    x = (rng.laplace(0, 1.0, d) * 1e-41).astype(np.float32)
+    assert 0 < np.count_nonzero(x) and np.abs(x).max() < 1.2e-38
+    pd = params_dict(d, 8 * 4096, packet_bits=4096, seed=4, client_id=2)
+    of, ost = run_case(x, pd)
+    x[::2] *= np.float32(1e3)                                                    # threshold bin among the smallest normals
+    run_case(x, pd)
 
 
 @pytest.mark.parametrize("quantizer", [0, 1])

@@ -56,6 +56,10 @@ def test_noalloc_matches_workspace_variant_on_two_calls_in_a_row():
     torch.cuda.synchronize()
     assert int(status.item()) == B.CVLC_OK
     _close(got1, ref1)
+    # ... and what the CPU oracle computes from the same streams
+    import oracle as O
+    want1 = O.decode_aggregate([s.cpu().numpy() for s in s1], np.array([3, 1, 4, 1, 5, 9, 2], np.float32), d)
+    _close(got1, torch.from_numpy(want1))
 
     # call 2, right after, fewer clients and accumulating: nothing of call 1 may leak through the scratch
     s2 = _encode_clients(torch, B, 3, d, seed0=40)
@@ -81,6 +85,34 @@ def test_noalloc_matches_workspace_variant_on_two_calls_in_a_row():
     torch.cuda.synchronize()
     assert int(status.item()) == B.CVLC_OK
     _close(got1, ref1)
+
+
+def test_noalloc_at_its_largest_client_count():
+    """exactly NOALLOC_MAX_CLIENTS small streams: the built-in scratch is used to its last table entry"""
+    import torch
+    import oracle as O
+    from paper_2402_03770_b200 import binding as B
+    B.lib()
+    B.cvlc_set_device(0)
+    dev = torch.device("cuda:0")
+    d, n = 3000, B.NOALLOC_MAX_CLIENTS
+    host_streams = []
+    for i in range(n):
+        x = np.random.default_rng(900 + i).standard_normal(d).astype(np.float32)
+        po = O.make_params(d, 2 * 1024, packet_bits=1024, seed=i, client_id=i)
+        host_streams.append(O.encode(x, po, O.plan(x, po)))
+    weights = np.random.default_rng(5).uniform(1, 9, n).astype(np.float32)
+    streams = [torch.from_numpy(s).to(dev) for s in host_streams]
+    ptrs, sizes, w = _tables(torch, streams, weights.tolist())
+    status = torch.full((1,), -1, dtype=torch.int32, device=dev)
+    got = torch.full((d,), float("nan"), dtype=torch.float32, device=dev)
+    B.cvlc_decode_aggregate_noalloc(ptrs, sizes, w, n, 0.0, d, got, False, status)
+    ref = torch.full((d,), float("nan"), dtype=torch.float32, device=dev)
+    B.cvlc_decode_aggregate(ptrs, sizes, w, n, 0.0, d, ref, False, B.alloc_bytes(B.cvlc_decode_workspace_bytes(n), dev))
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.CVLC_OK
+    _close(got, ref)
+    _close(got, torch.from_numpy(O.decode_aggregate(host_streams, weights, d)))
 
 
 def test_noalloc_rejects_more_clients_than_its_scratch_holds():

@@ -186,6 +186,40 @@ int cvlc_plan_from_histogram_batch(const uint64_t* hist_dev, const cvlc_params* 
                                    cvlc_plan_t* plans_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Problem P2 of Section IV-C as the paper solves it, with real-valued packet sizes P_1 <= ... <= P_R and code
+ * lengths y_r = (b - H) / P_r - s: k runs over n_k equidistant values of its range (Section IV-D, "equidistant
+ * spanning search"); for every k the packets start equal and consecutive packets are re-split by the atomic
+ * operation on Eq. (7) (Lemma 2: strongly convex in the split) in sweeps r = 2 .. R until a sweep moves no packet
+ * by more than 2^-30 of the largest packet, or max_sweeps; Eq. (5) then picks k*.  The result is a plan only:
+ * real-valued code lengths cannot be packed, so cvlc_encode does not take it; it serves to compare its error
+ * bound with the integer-length rule of cvlc_plan (whose alpha_q is the input here).  The atomic operation is a
+ * bracketing search (8 rounds of 32 equidistant splits, one per lane); the sweep inside one k is sequential, as
+ * the algorithm states, and the values of k run side by side, one warp each.  The number of sweeps grows about
+ * with R^2: meant for R up to a few dozen.
+ *  out_dev          the result header (64 bytes); status at byte 0
+ *  P_star_dev       R doubles: the packet sizes at k*, or NULL
+ *  ws_dev           cvlc_plan_literal_workspace_bytes(p, n_k) bytes; afterwards it holds, per value of k, at byte 256
+ *                   the values of k (uint64), then 256-byte aligned their error bounds (double), their sweeps
+ *                   (uint32) and their packet sizes (R doubles each)
+ * Errors: INVALID_ARG (alpha_q not below 0 or equal to -1/2, n_k outside 1 .. 4096, max_sweeps == 0, more than
+ * 2048 packets), BUDGET_*, PACKET_TOO_SMALL, WORKSPACE_TOO_SMALL.
+ */
+typedef struct cvlc_literal_plan_t {
+  int32_t status;
+  uint32_t R;           /* packets */
+  uint32_t n_k;         /* values of k tried */
+  uint32_t sweeps;      /* sweeps spent at k* */
+  uint64_t k_star;      /* the value of k with the smallest error bound (the first one on ties) */
+  double gamma_star;    /* Eq. (5) there */
+  double alpha_q, beta;
+  uint8_t reserved[16];
+} cvlc_literal_plan_t;
+size_t cvlc_plan_literal_workspace_bytes(const cvlc_params* p, uint32_t n_k);
+int cvlc_plan_literal(const cvlc_params* p, double alpha_q, uint32_t n_k, uint32_t max_sweeps,
+                      cvlc_literal_plan_t* out_dev, double* P_star_dev, void* ws_dev, size_t ws_bytes,
+                      void* cuda_stream);
+
+/*
  * Algorithm 1, steps 15-17.  Ranks the coordinates of x_dev by |x| (ties by
  * ascending index), gives packet r the next cap(y_r) ranks, stores the packet's
  * centroid distribution (PQ: minimum and maximum; QSGD: l2-norm), quantizes each value
@@ -339,7 +373,7 @@ int cvlc_selftest_wait(uint64_t* word_dev, int32_t* status_dev, uint32_t max_pol
  * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist").  Kernel names: k_zero_words,
  * k_hist, k_plan_fit, k_plan_tune, k_plan_finish, k_encode_init, k_select, k_select_lookback, k_sort_hist,
  * k_sort_scan, k_sort_pass, k_pack, k_decode_prepare, k_fill_zero, k_prefetch_l2, k_decode,
- * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply. */
+ * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply, k_plan_literal. */
 unsigned long long cvlc_launch_count(const char* kernel_name);
 /* Optional kernel timing: after cvlc_profile_select(name, n) the next n launches of that kernel
  * ("*" = of every kernel) are bracketed by a CUDA event pair on their own stream;

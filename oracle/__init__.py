@@ -99,6 +99,9 @@ def lib() -> C.CDLL:
         L.cvlc_plan_from_histogram_oracle.argtypes = [C.c_void_p, P(OrcParams), P(OrcPlan)]
         L.cvlc_decode_apply_oracle.restype = C.c_int
         L.cvlc_decode_apply_oracle.argtypes = [P(C.c_void_p), P(u64), C.c_void_p, u32, f64, u64, C.c_void_p]
+        L.cvlc_plan_literal_oracle.restype = C.c_int
+        L.cvlc_plan_literal_oracle.argtypes = [P(OrcParams), f64, u32, u32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               P(u64), P(f64), C.c_void_p]
         L.cvlc_plan_fixed_oracle.restype = C.c_int
         L.cvlc_plan_fixed_oracle.argtypes = [P(OrcParams), u32, P(OrcPlan)]
         L.cvlc_rank_oracle.restype = C.c_int
@@ -243,6 +246,34 @@ def plan_fixed(p: OrcParams, y: int) -> OrcPlan:
     if rc != ORC_OK:
         raise OracleError(rc, "plan_fixed")
     return pl
+
+
+@dataclass
+class LiteralPlan:
+    k_star: int
+    gamma_star: float
+    P_star: np.ndarray        # R real-valued packet sizes at k_star
+    k_grid: np.ndarray        # the values of k that were tried
+    gamma_of_k: np.ndarray    # Eq. (5) after tuning, per value of k
+    sweeps_of_k: np.ndarray
+
+
+def plan_literal(p: OrcParams, alpha_q: float, n_k: int, max_sweeps: int = 1 << 20) -> LiteralPlan:
+    """problem P2 with real-valued packet sizes: k on an equidistant grid, pairwise tuning of consecutive packets"""
+    rc0, s, R, cap = derive(p)
+    if rc0 != ORC_OK:
+        raise OracleError(rc0, "plan_literal")
+    k_grid = np.zeros(n_k, dtype=np.uint64)
+    gam = np.zeros(n_k, dtype=np.float64)
+    sw = np.zeros(n_k, dtype=np.uint32)
+    P_star = np.zeros(R, dtype=np.float64)
+    k_star, g_star = C.c_uint64(), C.c_double()
+    rc = lib().cvlc_plan_literal_oracle(C.byref(p), float(alpha_q), int(n_k), int(max_sweeps), k_grid.ctypes.data,
+                                        gam.ctypes.data, sw.ctypes.data, C.byref(k_star), C.byref(g_star),
+                                        P_star.ctypes.data)
+    if rc != ORC_OK:
+        raise OracleError(rc, "plan_literal")
+    return LiteralPlan(int(k_star.value), float(g_star.value), P_star, k_grid, gam, sw)
 
 
 def rank(x: np.ndarray, k: int) -> np.ndarray:

@@ -482,6 +482,137 @@ int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan) {
 }
 
 /* ======================================================================== */
+/* Problem P2 with real-valued packet sizes (Section IV-C): enumerate k, and   */
+/* for every k tune P_1 .. P_R two consecutive packets at a time               */
+/* ======================================================================== */
+
+/* What a real-valued packet of P records contributes per unit of energy: the bracket of
+ * Eq. (5) with the code length the packet constraint leaves, y = (b - H) / P - s. */
+static double packet_cost(double P, double bH, double s, uint32_t quantizer, double B) {
+  double y = bH / P - s;
+  double Q;
+  if (quantizer == ORC_QUANT_QSGD) {
+    double sq = cvlc_exp2_oracle(y - 1.0) - 1.0;
+    double Q1 = P / (sq * sq);
+    double Q2 = sqrt(P) / sq;
+    Q = (Q1 < Q2) ? Q1 : Q2;
+  } else {
+    double L = cvlc_exp2_oracle(y) - 1.0;
+    Q = P / (L * L);
+  }
+  return Q / (B * B) + (1.0 - 1.0 / B) * (1.0 - 1.0 / B);
+}
+
+/* share of the energy in the top Z ranks for real Z (same boundary as energy_E) */
+static double energy_real(double Z, double beta, double D) { return (cvlc_powr_oracle(Z + 1.0, beta) - 1.0) / D; }
+
+/* Eq. (7): the part of gamma that the split of X = P_{r-1} + P_r records between the packets r-1 and r
+ * decides, as a function of p = P_r; Z0 = Z_{r-2}, Z2 = Z_r. */
+static double pair_f(double p, double X, double Z0, double Z2, double bH, double s, uint32_t quantizer, double B,
+                     double beta, double D) {
+  double Em = energy_real(Z0 + (X - p), beta, D);
+  double hi_part = packet_cost(p, bH, s, quantizer, B) * (energy_real(Z2, beta, D) - Em);
+  double lo_part = packet_cost(X - p, bH, s, quantizer, B) * (Em - energy_real(Z0, beta, D));
+  return hi_part + lo_part;
+}
+
+int cvlc_plan_literal_oracle(const orc_params* p, double alpha_q, uint32_t n_k, uint32_t max_sweeps, uint64_t* k_grid,
+                             double* gamma_of_k, uint32_t* sweeps_of_k, uint64_t* k_star, double* gamma_star, double* P_star) {
+  if (!params_ok(p) || n_k < 1 || n_k > 4096 || max_sweeps < 1 || !(alpha_q < 0.0) || alpha_q == -0.5) return ORC_ERR_INVALID_ARG;
+  uint32_t si, R, cap[ORC_MAX_Y + 1];
+  int rc = cvlc_derive_oracle(p, &si, &R, cap);
+  if (rc != ORC_OK) return rc;
+  const uint32_t y_lo = (p->quantizer == ORC_QUANT_QSGD) ? 2u : 1u; /* a one-bit QSGD code holds no level */
+  if (p->max_code_bits < y_lo) return ORC_ERR_INVALID_ARG;
+  const double s = (double)si, bH = (double)(p->packet_bits - p->header_bits), B = p->scale_B;
+  const double P_min = bH / (s + (double)p->max_code_bits), P_max = bH / (s + (double)y_lo);
+  /* the range of k: at least one record per packet and no code longer than max_code_bits, no code shorter than
+   * y_lo, no more than d coordinates */
+  double klo = ceil((double)R * P_min), khi = floor((double)R * P_max);
+  if (klo < (double)R) klo = (double)R;
+  if (khi > (double)p->d) khi = (double)p->d;
+  if (!(klo <= khi)) return ORC_ERR_BUDGET_TOO_LARGE;
+  const uint64_t k_lo = (uint64_t)klo, k_hi = (uint64_t)khi;
+  const double beta = 2.0 * alpha_q + 1.0;
+  const double D = cvlc_powr_oracle((double)p->d, beta) - 1.0;
+  const double tol = P_max * (1.0 / 1073741824.0);
+
+  double* P = (double*)malloc(sizeof(double) * (size_t)R);
+  double* Z = (double*)malloc(sizeof(double) * ((size_t)R + 1));
+  if (!P || !Z) { free(P); free(Z); return ORC_ERR_INVALID_ARG; }
+  int have = 0;
+  for (uint32_t ik = 0; ik < n_k; ++ik) {
+    /* equidistant values of k (Section IV-D) */
+    uint64_t k = (n_k == 1) ? k_lo : k_lo + (uint64_t)(((unsigned __int128)ik * (k_hi - k_lo)) / (n_k - 1));
+    for (uint32_t r = 0; r < R; ++r) P[r] = (double)k / (double)R; /* equal packets */
+    uint32_t sweep = 0;
+    for (; sweep < max_sweeps; ++sweep) {
+      Z[0] = 0.0;
+      for (uint32_t r = 0; r < R; ++r) Z[r + 1] = Z[r] + P[r];
+      double moved = 0.0;
+      for (uint32_t r = 1; r < R; ++r) { /* packets r-1 and r (0-based), the later one the larger (Eq. (4)) */
+        double X = P[r - 1] + P[r], Z0 = Z[r - 1], Z2 = Z[r + 1];
+        double lo = X / 2.0, hi = X - P_min;
+        if (lo < P_min) lo = P_min;
+        if (lo < X - P_max) lo = X - P_max;
+        if (hi > P_max) hi = P_max;
+        if (!(lo < hi)) continue;
+        /* the atomic operation: f is strongly convex in p (Lemma 2); eight times, 32 equidistant points of the
+         * bracket are tried and the bracket shrinks to the neighbours of the best one */
+        double best_x = lo;
+        for (int round = 0; round < 8; ++round) {
+          double step = (hi - lo) / 31.0;
+          int best_j = 0;
+          double best_f = 0.0;
+          for (int j = 0; j < 32; ++j) {
+            double xj = (j == 31) ? hi : lo + (double)j * step;
+            double fj = pair_f(xj, X, Z0, Z2, bH, s, p->quantizer, B, beta, D);
+            if (j == 0 || fj < best_f) { best_f = fj; best_j = j; }
+          }
+          double nlo = (best_j == 0) ? lo : lo + (double)(best_j - 1) * step;
+          double nhi = (best_j >= 30) ? hi : lo + (double)(best_j + 1) * step;
+          best_x = (best_j == 31) ? hi : lo + (double)best_j * step;
+          lo = nlo;
+          hi = nhi;
+        }
+        double f_new = pair_f(best_x, X, Z0, Z2, bH, s, p->quantizer, B, beta, D);
+        double f_old = pair_f(P[r], X, Z0, Z2, bH, s, p->quantizer, B, beta, D);
+        if (f_new < f_old) {
+          double delta = fabs(best_x - P[r]);
+          if (delta > moved) moved = delta;
+          P[r - 1] = X - best_x;
+          P[r] = best_x;
+          Z[r] = Z0 + P[r - 1];
+        }
+      }
+      if (!(moved > tol)) { ++sweep; break; }
+    }
+    /* Eq. (5) at these packet sizes */
+    Z[0] = 0.0;
+    for (uint32_t r = 0; r < R; ++r) Z[r + 1] = Z[r] + P[r];
+    double gamma = 1.0 - energy_real(Z[R], beta, D);
+    double Eprev = 0.0;
+    for (uint32_t r = 0; r < R; ++r) {
+      double Ecur = energy_real(Z[r + 1], beta, D);
+      gamma = gamma + packet_cost(P[r], bH, s, p->quantizer, B) * (Ecur - Eprev);
+      Eprev = Ecur;
+    }
+    if (k_grid) k_grid[ik] = k;
+    if (gamma_of_k) gamma_of_k[ik] = gamma;
+    if (sweeps_of_k) sweeps_of_k[ik] = sweep;
+    if (!have || gamma < *gamma_star) {
+      have = 1;
+      *gamma_star = gamma;
+      *k_star = k;
+      if (P_star) memcpy(P_star, P, sizeof(double) * (size_t)R);
+    }
+  }
+  free(P);
+  free(Z);
+  return ORC_OK;
+}
+
+/* ======================================================================== */
 /* Ranking ("ranked in a descending order of their absolute values")          */
 /* ======================================================================== */
 

@@ -12,9 +12,7 @@
  * multiply-add (build with -ffp-contract=off), operations in written order.
  *
  * Parity pins (see tests, "-m 'not gpu'"): every exported function is checked
- * against something other than itself; none is "parity unpinned".  The literal
- * real-valued form of Algorithm 1 is not built here; the tests restate it in Python
- * on small instances as one of the pins of the length tuning.
+ * against something other than itself; none is "parity unpinned".
  */
 #ifndef CVLC_ORACLE_H
 #define CVLC_ORACLE_H
@@ -99,6 +97,16 @@ int cvlc_plan_oracle(const float* x, const orc_params* p, orc_plan* plan);
 /* planning at the parameter server from a client's histogram (Section IV-C, last paragraph) */
 int cvlc_plan_from_histogram_oracle(const uint64_t h[ORC_HIST_BINS], const orc_params* p, orc_plan* plan);
 int cvlc_plan_fixed_oracle(const orc_params* p, uint32_t y, orc_plan* plan);
+
+/* Problem P2 with real-valued packet sizes, as Section IV-C solves it: k runs over n_k equidistant values of
+ * its range; for each, P_1 .. P_R start equal and consecutive packets are re-split (atomic operation on Eq. (7),
+ * a fixed 8 x 32-point bracketing search) in sweeps r = 2 .. R until a sweep moves no packet by more than
+ * 2^-30 of the largest packet, or max_sweeps; gamma of Eq. (5) with y_r = (b - H) / P_r - s picks k*.  A plan
+ * only (real-valued code lengths cannot be packed).  Outputs: k_grid, gamma_of_k, sweeps_of_k (n_k entries each,
+ * may be NULL), k_star, gamma_star, P_star (R doubles, may be NULL). */
+int cvlc_plan_literal_oracle(const orc_params* p, double alpha_q, uint32_t n_k, uint32_t max_sweeps, uint64_t* k_grid,
+                             double* gamma_of_k, uint32_t* sweeps_of_k, uint64_t* k_star, double* gamma_star,
+                             double* P_star);
 
 /* --- encoding ------------------------------------------------------------ */
 /* first k ranks of the order (|x| descending, index ascending) */

@@ -46,7 +46,8 @@ EXPORTS = [
     "cvlc_plan", "cvlc_plan_fixed", "cvlc_encode", "cvlc_plan_batch_workspace_bytes",
     "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math", "cvlc_histogram_batch", "cvlc_plan_from_histogram_batch", "cvlc_decode_apply",
-    "cvlc_decode_aggregate_noalloc", "cvlc_compress_batch", "cvlc_selftest_wait", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
+    "cvlc_decode_aggregate_noalloc", "cvlc_compress_batch", "cvlc_selftest_wait", "cvlc_plan_literal",
+    "cvlc_plan_literal_workspace_bytes", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -127,6 +128,10 @@ def lib() -> C.CDLL:
     L.cvlc_encode_batch.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
     L.cvlc_compress_batch.restype = C.c_int
     L.cvlc_compress_batch.argtypes = [vp, PP, u32, u32, vp, vp, sz, u64, vp, sz, vp, sz, vp, vp]
+    L.cvlc_plan_literal_workspace_bytes.restype = sz
+    L.cvlc_plan_literal_workspace_bytes.argtypes = [PP, u32]
+    L.cvlc_plan_literal.restype = C.c_int
+    L.cvlc_plan_literal.argtypes = [PP, f64, u32, u32, vp, vp, vp, sz, vp]
     L.cvlc_selftest_wait.restype = C.c_int
     L.cvlc_selftest_wait.argtypes = [vp, vp, u32, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
@@ -293,6 +298,39 @@ def cvlc_compress_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams]
                                      plan_ws.numel() * plan_ws.element_size(), _ptr(enc_ws),
                                      enc_ws.numel() * enc_ws.element_size(), _stream_handle(stream), side),
            "cvlc_compress_batch")
+
+
+class CvlcLiteralPlan(C.Structure):
+    _fields_ = [("status", C.c_int32), ("R", C.c_uint32), ("n_k", C.c_uint32), ("sweeps", C.c_uint32),
+                ("k_star", C.c_uint64), ("gamma_star", C.c_double), ("alpha_q", C.c_double), ("beta", C.c_double),
+                ("reserved", C.c_uint8 * 16)]
+
+
+assert C.sizeof(CvlcLiteralPlan) == 64
+
+
+def cvlc_plan_literal(p: CvlcParams, alpha_q: float, n_k: int, max_sweeps: int, device: torch.device,
+                      stream: Optional[torch.cuda.Stream] = None):
+    """Problem P2 with real-valued packet sizes (plan only).  Returns (CvlcLiteralPlan, P_star, k_grid, gamma_of_k,
+    sweeps_of_k) as host copies; allocates its buffers itself (marshalling and allocation only)."""
+    nbytes = int(lib().cvlc_plan_literal_workspace_bytes(C.byref(p), int(n_k)))
+    R = int(p.budget_bits // p.packet_bits)
+    ws = alloc_bytes(max(nbytes, 256), device)
+    out = alloc_bytes(64, device)
+    P_star = torch.zeros(max(R, 1), dtype=torch.float64, device=device)
+    _check(lib().cvlc_plan_literal(C.byref(p), float(alpha_q), int(n_k), int(max_sweeps), _ptr(out), _ptr(P_star), _ptr(ws),
+                                   ws.numel(), _stream_handle(stream)), "cvlc_plan_literal")
+    head = CvlcLiteralPlan.from_buffer_copy(bytes(out.cpu().numpy().tobytes()))
+    raw = ws.cpu().numpy()
+    a256 = lambda v: (v + 255) & ~255
+    off_k = 256
+    off_g = a256(off_k + 8 * n_k)
+    off_s = a256(off_g + 8 * n_k)
+    import numpy as np
+    k_grid = raw[off_k:off_k + 8 * n_k].view(np.uint64).copy()
+    gamma = raw[off_g:off_g + 8 * n_k].view(np.float64).copy()
+    sweeps = raw[off_s:off_s + 4 * n_k].view(np.uint32).copy()
+    return head, P_star.cpu().numpy(), k_grid, gamma, sweeps
 
 
 def cvlc_selftest_wait(word: torch.Tensor, status: torch.Tensor, max_polls: int,

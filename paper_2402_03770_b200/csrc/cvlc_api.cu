@@ -249,6 +249,38 @@ int cvlc_plan_from_histogram_batch(const uint64_t* hist_dev, const cvlc_params* 
                                static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
+size_t cvlc_plan_literal_workspace_bytes(const cvlc_params* p, uint32_t n_k) {
+  Derived D;
+  if (derive(p, &D) != CVLC_OK || n_k == 0 || n_k > kLiteralMaxK || D.R > kLiteralMaxR) return 0;
+  return literal_ws_bytes(n_k, D.R);
+}
+
+int cvlc_plan_literal(const cvlc_params* p, double alpha_q, uint32_t n_k, uint32_t max_sweeps, cvlc_literal_plan_t* out_dev,
+                      double* P_star_dev, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  Derived D;
+  const int rc = derive(p, &D);
+  if (rc != CVLC_OK) return rc;
+  if (n_k == 0 || n_k > kLiteralMaxK || max_sweeps == 0 || !(alpha_q < 0.0) || alpha_q == -0.5 || D.R > kLiteralMaxR)
+    return CVLC_ERR_INVALID_ARG;
+  const uint32_t y_lo = (p->quantizer == CVLC_QUANT_QSGD) ? 2u : 1u;  // a one-bit QSGD code holds no level
+  if (p->max_code_bits < y_lo) return CVLC_ERR_INVALID_ARG;
+  if (!aligned(out_dev, 8) || !aligned(ws_dev, 256) || (P_star_dev && !aligned(P_star_dev, 8))) return CVLC_ERR_INVALID_ARG;
+  if (ws_bytes < literal_ws_bytes(n_k, D.R)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  // the range of k: no code longer than max_code_bits or shorter than y_lo, at least one record per packet, at
+  // most d coordinates (plain IEEE operations, compiled without contraction)
+  const double s = (double)D.s, bH = (double)(p->packet_bits - p->header_bits);
+  const double P_min = bH / (s + (double)p->max_code_bits), P_max = bH / (s + (double)y_lo);
+  double klo = ceil((double)D.R * P_min), khi = floor((double)D.R * P_max);
+  if (klo < (double)D.R) klo = (double)D.R;
+  if (khi > (double)p->d) khi = (double)p->d;
+  if (!(klo <= khi)) return CVLC_ERR_BUDGET_TOO_LARGE;
+  const double tol = P_max * (1.0 / 1073741824.0);
+  return launch_plan_literal(*p, alpha_q, D.s, D.R, n_k, max_sweeps, (unsigned long long)klo, (unsigned long long)khi, P_min,
+                             P_max, tol, out_dev, P_star_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
+}
+
 int cvlc_plan(const float* x_dev, const cvlc_params* p, cvlc_plan_t* plan_dev, void* ws_dev, size_t ws_bytes,
               void* cuda_stream) {
   return cvlc_plan_batch(&x_dev, p, 1, 0, plan_dev, ws_dev, ws_bytes, cuda_stream);

@@ -207,7 +207,7 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 enum KernelId {
   kKZeroWords = 0, kKHist, kKPlanFit, kKPlanTune, kKPlanFinish, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan,
   kKSortPass, kKPack, kKDecodePrepare, kKFillZero, kKPrefetchL2, kKDecode, kKNoallocStatus, kKSelftest, kKHistCheck, kKApply,
-  kNumKernelIds
+  kKPlanLiteral, kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -234,6 +234,17 @@ cudaError_t launch_histogram(const ClientDesc* clients, uint32_t n, const Shape&
                              unsigned long long* hist_out, cudaStream_t st);
 cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const Shape& shape,
                                   const unsigned long long* hist, void* ws, cudaStream_t st);
+// workspace of cvlc_plan_literal: per value of k its value, its error bound, its sweeps and its packet sizes
+CVLC_HD constexpr size_t literal_off_k(uint32_t) { return 256; }
+CVLC_HD constexpr size_t literal_off_gamma(uint32_t n_k) { return align256(literal_off_k(n_k) + (size_t)n_k * 8); }
+CVLC_HD constexpr size_t literal_off_sweeps(uint32_t n_k) { return align256(literal_off_gamma(n_k) + (size_t)n_k * 8); }
+CVLC_HD constexpr size_t literal_off_P(uint32_t n_k) { return align256(literal_off_sweeps(n_k) + (size_t)n_k * 4); }
+CVLC_HD constexpr size_t literal_ws_bytes(uint32_t n_k, uint32_t R) { return align256(literal_off_P(n_k) + (size_t)n_k * R * 8); }
+constexpr uint32_t kLiteralMaxR = 2048;   // packet sizes and their running sums of one k live in shared memory
+constexpr uint32_t kLiteralMaxK = 4096;
+cudaError_t launch_plan_literal(const cvlc_params& p, double alpha_q, uint32_t s, uint32_t R, uint32_t n_k, uint32_t max_sweeps,
+                                unsigned long long k_lo, unsigned long long k_hi, double P_min, double P_max, double tol,
+                                cvlc_literal_plan_t* out, double* P_star, void* ws, cudaStream_t st);
 cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st);
 // wait_before_pack: an event the stream waits for right before the packing kernel (the length tuning on
 // another stream), or nullptr

@@ -495,11 +495,20 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
         const uint64_t n_rows = (n_units + kRowUnits - 1) / kRowUnits;
         const uint64_t n_words = (n_rows + 31) / 32;          // half words of row flags
         const uint64_t tile0 = seg_first_tile(p0, b + c);
-        for (uint64_t w = warp; w < ((n_words + 1) & ~(uint64_t)1); w += kPlanThreads / 32) {  // whole 64-bit words
-          const uint64_t r = w * 32 + lane;
-          const bool flag = (r < n_rows) && row_max[tile0 * kTileRows + r] >= thresh_key;
-          const unsigned bits = __ballot_sync(kFull, flag);
-          if (lane == 0) row_flags[tile0 * 2 + w] = bits;
+        const uint64_t n_half = (n_words + 1) & ~(uint64_t)1;  // whole 64-bit words
+        for (uint64_t w0 = (uint64_t)warp * 4; w0 < n_half; w0 += 4 * (kPlanThreads / 32)) {  // four loads in flight
+          uint32_t mx[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint64_t r = (w0 + j) * 32 + lane;
+            mx[j] = (r < n_rows) ? row_max[tile0 * kTileRows + r] : 0u;
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint64_t r = (w0 + j) * 32 + lane;
+            const unsigned bits = __ballot_sync(kFull, (r < n_rows) && mx[j] >= thresh_key);
+            if (lane == 0 && w0 + j < n_half) row_flags[tile0 * 2 + w0 + j] = bits;
+          }
         }
       }
     }
@@ -1187,6 +1196,217 @@ cudaError_t launch_plan_from_hist(const ClientDesc* clients, uint32_t n, const S
                                   const unsigned long long* hist, void* ws, cudaStream_t st) {
   if (n <= (uint32_t)kSmallBatch) return launch_plan_from_hist_t<kSmallBatch>(clients, n, shape, hist, ws, st);
   return launch_plan_from_hist_t<kLargeBatch>(clients, n, shape, hist, ws, st);
+}
+
+// ===================================================================================
+// Problem P2 with real-valued packet sizes (Section IV-C; Algorithm 1 steps 2-14 with the equidistant
+// search over k of Section IV-D): a plan only, for comparing its error bound with the integer-length rule
+// ===================================================================================
+// One warp per value of k.  For that k the packets start equal and are re-split two consecutive ones at a time,
+// r = 2 .. R in order (each re-split sees the previous one: the sweep is sequential by definition); a re-split
+// minimises Eq. (7), strongly convex in the split (Lemma 2), by bracketing: the 32 lanes evaluate 32 equidistant
+// splits of the bracket, the bracket shrinks to the neighbours of the best one, eight times.  All arithmetic is
+// binary64 with separately rounded operations in a fixed order, so the result does not depend on the machine.
+
+struct LiteralArgs {
+  double bH, s, B, P_min, P_max, tol, alpha_q;
+  unsigned long long k_lo, k_hi, d;
+  uint32_t R, n_k, max_sweeps, quantizer;
+};
+
+// the bracket of Eq. (5) for a packet of P records at the length the packet constraint leaves: y = (b - H) / P - s
+__device__ __forceinline__ double literal_cost(double P, const LiteralArgs& a) {
+  const double y = __dsub_rn(__ddiv_rn(a.bH, P), a.s);
+  double Q;
+  if (a.quantizer == CVLC_QUANT_QSGD) {
+    const double sq = __dsub_rn(series_exp2(__dsub_rn(y, 1.0)), 1.0);
+    const double Q1 = __ddiv_rn(P, __dmul_rn(sq, sq));
+    const double Q2 = __ddiv_rn(__dsqrt_rn(P), sq);
+    Q = (Q1 < Q2) ? Q1 : Q2;
+  } else {
+    const double L = __dsub_rn(series_exp2(y), 1.0);
+    Q = __ddiv_rn(P, __dmul_rn(L, L));
+  }
+  const double one_m = __dsub_rn(1.0, __ddiv_rn(1.0, a.B));
+  return __dadd_rn(__ddiv_rn(Q, __dmul_rn(a.B, a.B)), __dmul_rn(one_m, one_m));
+}
+
+__device__ __forceinline__ double literal_energy(double Z, double beta, double D) {
+  return __ddiv_rn(__dsub_rn(series_powr(__dadd_rn(Z, 1.0), beta), 1.0), D);
+}
+
+// Eq. (7) as a function of p = P_r: X = P_{r-1} + P_r, Z0 = Z_{r-2}, Z2 = Z_r
+__device__ __forceinline__ double literal_pair_f(double p, double X, double Z0, double Z2, const LiteralArgs& a, double beta, double D) {
+  const double Em = literal_energy(__dadd_rn(Z0, __dsub_rn(X, p)), beta, D);
+  const double hi_part = __dmul_rn(literal_cost(p, a), __dsub_rn(literal_energy(Z2, beta, D), Em));
+  const double lo_part = __dmul_rn(literal_cost(__dsub_rn(X, p), a), __dsub_rn(Em, literal_energy(Z0, beta, D)));
+  return __dadd_rn(hi_part, lo_part);
+}
+
+__global__ void __launch_bounds__(32)
+k_plan_literal(const __grid_constant__ LiteralArgs a, unsigned long long* __restrict__ k_grid, double* __restrict__ gamma_of_k,
+               uint32_t* __restrict__ sweeps_of_k, double* __restrict__ P_all) {
+  extern __shared__ double lit_smem[];  // P[R], Z[R + 1]
+  double* P = lit_smem;
+  double* Z = lit_smem + a.R;
+  const int lane = threadIdx.x;
+  const uint32_t ik = blockIdx.x, R = a.R;
+  const double beta = __dadd_rn(__dmul_rn(2.0, a.alpha_q), 1.0);
+  const double D = __dsub_rn(series_powr((double)a.d, beta), 1.0);
+  // equidistant values of k; the product stays below 2^64 (n_k <= 4096, k <= 2^31 * 2^31 is never reached: k <= d)
+  const unsigned long long k = (a.n_k == 1) ? a.k_lo : a.k_lo + ((unsigned long long)ik * (a.k_hi - a.k_lo)) / (a.n_k - 1);
+  const double P0 = __ddiv_rn((double)k, (double)R);
+  for (uint32_t r = lane; r < R; r += 32) P[r] = P0;
+  __syncwarp();
+  uint32_t sweep = 0;
+  for (; sweep < a.max_sweeps; ++sweep) {
+    if (lane == 0) {
+      double z = 0.0;
+      Z[0] = 0.0;
+      for (uint32_t r = 0; r < R; ++r) {
+        z = __dadd_rn(z, P[r]);
+        Z[r + 1] = z;
+      }
+    }
+    __syncwarp();
+    double moved = 0.0;
+    for (uint32_t r = 1; r < R; ++r) {
+      const double Pr = P[r];
+      const double X = __dadd_rn(P[r - 1], Pr), Z0 = Z[r - 1], Z2 = Z[r + 1];
+      double lo = __ddiv_rn(X, 2.0), hi = __dsub_rn(X, a.P_min);
+      if (lo < a.P_min) lo = a.P_min;
+      const double lo2 = __dsub_rn(X, a.P_max);
+      if (lo < lo2) lo = lo2;
+      if (hi > a.P_max) hi = a.P_max;
+      if (!(lo < hi)) continue;
+      double best_x = lo;
+      for (int round = 0; round < 8; ++round) {
+        const double step = __ddiv_rn(__dsub_rn(hi, lo), 31.0);
+        const double xj = (lane == 31) ? hi : __dadd_rn(lo, __dmul_rn((double)lane, step));
+        double f = literal_pair_f(xj, X, Z0, Z2, a, beta, D);
+        int j = lane;
+        // the first of the smallest values
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          const double fo = __shfl_xor_sync(kFull, f, off);
+          const int jo = __shfl_xor_sync(kFull, j, off);
+          if (fo < f || (fo == f && jo < j)) {
+            f = fo;
+            j = jo;
+          }
+        }
+        const double nlo = (j == 0) ? lo : __dadd_rn(lo, __dmul_rn((double)(j - 1), step));
+        const double nhi = (j >= 30) ? hi : __dadd_rn(lo, __dmul_rn((double)(j + 1), step));
+        best_x = (j == 31) ? hi : __dadd_rn(lo, __dmul_rn((double)j, step));
+        lo = nlo;
+        hi = nhi;
+      }
+      // lanes 0 and 1 evaluate the new and the current split
+      const double fe = literal_pair_f(lane == 0 ? best_x : Pr, X, Z0, Z2, a, beta, D);
+      const double f_new = __shfl_sync(kFull, fe, 0), f_old = __shfl_sync(kFull, fe, 1);
+      if (f_new < f_old) {
+        const double delta = fabs(__dsub_rn(best_x, Pr));
+        if (delta > moved) moved = delta;
+        if (lane == 0) {
+          const double Pm = __dsub_rn(X, best_x);
+          P[r - 1] = Pm;
+          P[r] = best_x;
+          Z[r] = __dadd_rn(Z0, Pm);
+        }
+      }
+      __syncwarp();
+    }
+    if (!(moved > a.tol)) {
+      ++sweep;
+      break;
+    }
+  }
+  // Eq. (5) at these packet sizes: the terms side by side, their sum in packet order
+  if (lane == 0) {
+    double z = 0.0;
+    Z[0] = 0.0;
+    for (uint32_t r = 0; r < R; ++r) {
+      z = __dadd_rn(z, P[r]);
+      Z[r + 1] = z;
+    }
+  }
+  __syncwarp();
+  double* P_out = P_all + (size_t)ik * R;
+  double* term = P_out;  // the terms borrow the output slots; the packet sizes follow once the sum is taken
+  for (uint32_t r = lane; r < R; r += 32) {
+    const double Eprev = (r == 0) ? 0.0 : literal_energy(Z[r], beta, D);
+    const double Ecur = literal_energy(Z[r + 1], beta, D);
+    term[r] = __dmul_rn(literal_cost(P[r], a), __dsub_rn(Ecur, Eprev));
+  }
+  __syncwarp();
+  if (lane == 0) {
+    double gamma = __dsub_rn(1.0, literal_energy(Z[R], beta, D));
+    for (uint32_t r = 0; r < R; ++r) gamma = __dadd_rn(gamma, term[r]);
+    gamma_of_k[ik] = gamma;
+    k_grid[ik] = k;
+    sweeps_of_k[ik] = sweep;
+  }
+  __syncwarp();
+  for (uint32_t r = lane; r < R; r += 32) P_out[r] = P[r];
+}
+
+// the value of k with the smallest error bound (the first one on ties) and its packet sizes
+__global__ void __launch_bounds__(256)
+k_plan_literal_pick(const __grid_constant__ LiteralArgs a, const unsigned long long* __restrict__ k_grid,
+                    const double* __restrict__ gamma_of_k, const uint32_t* __restrict__ sweeps_of_k,
+                    const double* __restrict__ P_all, cvlc_literal_plan_t* __restrict__ out, double* __restrict__ P_star) {
+  __shared__ uint32_t s_best;
+  if (threadIdx.x == 0) {
+    uint32_t best = 0;
+    for (uint32_t i = 1; i < a.n_k; ++i)
+      if (gamma_of_k[i] < gamma_of_k[best]) best = i;
+    s_best = best;
+    out->status = CVLC_OK;
+    out->R = a.R;
+    out->n_k = a.n_k;
+    out->sweeps = sweeps_of_k[best];
+    out->k_star = k_grid[best];
+    out->gamma_star = gamma_of_k[best];
+    out->alpha_q = a.alpha_q;
+    out->beta = __dadd_rn(__dmul_rn(2.0, a.alpha_q), 1.0);
+  }
+  __syncthreads();
+  if (P_star)
+    for (uint32_t r = threadIdx.x; r < a.R; r += 256) P_star[r] = P_all[(size_t)s_best * a.R + r];
+}
+
+cudaError_t launch_plan_literal(const cvlc_params& p, double alpha_q, uint32_t s, uint32_t R, uint32_t n_k, uint32_t max_sweeps,
+                                unsigned long long k_lo, unsigned long long k_hi, double P_min, double P_max, double tol,
+                                cvlc_literal_plan_t* out, double* P_star, void* ws, cudaStream_t st) {
+  LiteralArgs a;
+  a.bH = (double)(p.packet_bits - p.header_bits);
+  a.s = (double)s;
+  a.B = p.scale_B;
+  a.P_min = P_min;
+  a.P_max = P_max;
+  a.tol = tol;
+  a.alpha_q = alpha_q;
+  a.k_lo = k_lo;
+  a.k_hi = k_hi;
+  a.d = p.d;
+  a.R = R;
+  a.n_k = n_k;
+  a.max_sweeps = max_sweeps;
+  a.quantizer = p.quantizer;
+  unsigned char* w = static_cast<unsigned char*>(ws);
+  unsigned long long* k_grid = reinterpret_cast<unsigned long long*>(w + literal_off_k(n_k));
+  double* gamma_of_k = reinterpret_cast<double*>(w + literal_off_gamma(n_k));
+  uint32_t* sweeps_of_k = reinterpret_cast<uint32_t*>(w + literal_off_sweeps(n_k));
+  double* P_all = reinterpret_cast<double*>(w + literal_off_P(n_k));
+  {
+    LaunchScope ls(kKPlanLiteral, st);
+    k_plan_literal<<<n_k, 32, (2 * (size_t)R + 1) * 8, st>>>(a, k_grid, gamma_of_k, sweeps_of_k, P_all);
+  }
+  {
+    LaunchScope ls(kKPlanLiteral, st);
+    k_plan_literal_pick<<<1, 256, 0, st>>>(a, k_grid, gamma_of_k, sweeps_of_k, P_all, out, P_star);
+  }
+  return cudaGetLastError();
 }
 
 // ---- diagnostics ---------------------------------------------------------------------

@@ -258,6 +258,159 @@ def test_brute_force_cases_not_all_skipped():
     assert ran >= 30
 
 
+# ---- the same against an enumeration that knows nothing of the oracle's candidate list: every length
+# 1 .. max_code_bits may be used, and every plan is scored by Eq. (5) written packet by packet with libm
+
+ALL_LENGTH_CASES = []
+_rng2 = np.random.default_rng(77)
+while len(ALL_LENGTH_CASES) < 48:
+    c = dict(d=int(_rng2.choice([4_000, 50_000, 2_000_000, 60_000_000])), R=int(_rng2.integers(1, 5)),
+             packet_bits=int(_rng2.choice([384, 1024, 4096, 12000])), max_code_bits=int(_rng2.integers(4, 10)),
+             alpha_q=float(_rng2.integers(-700, -8)) / 256.0, B=float(_rng2.choice([1.0, 1.002, 1.03, 1.4, 2.5])))
+    if c["alpha_q"] != -0.5:
+        ALL_LENGTH_CASES.append(c)
+# scales right above (Q + 1) / 2 of some length: its coefficient is positive but tiny, and it still belongs to the plan
+for _d, _pb, _y0, _eps, _aq in [(50_000, 1024, 3, 0.01, -0.3), (50_000, 1024, 3, 0.002, -0.7), (2_000_000, 4096, 3, 0.005, -0.25),
+                                (60_000_000, 12000, 4, 0.01, -0.2), (4_000, 384, 2, 0.004, -0.4), (50_000, 1024, 3, 0.02, -1.2)]:
+    _s = max(1, math.ceil(math.log2(_d)))
+    _Q = ((_pb - 80) // (_s + _y0)) / float((2 ** _y0 - 1) ** 2)
+    ALL_LENGTH_CASES.append(dict(d=_d, R=3, packet_bits=_pb, max_code_bits=9, alpha_q=_aq, B=max(1.0, (_Q + 1.0) / 2.0) * (1.0 + _eps),
+                                 tiny_g=_y0))
+
+
+@pytest.mark.parametrize("case", ALL_LENGTH_CASES)
+def test_length_tuning_is_optimal_over_all_lengths(case):
+    """Dropping the lengths with a non-positive coefficient and the lengths that fit no more records than the next
+    longer one must not lose the optimum: the plan's gamma equals the minimum of Eq. (5) over every non-increasing
+    sequence of lengths 1 .. max_code_bits (Theorem 1), and no sequence outside the plan's support does better."""
+    p = O.make_params(case["d"], case["R"] * case["packet_bits"], packet_bits=case["packet_bits"],
+                      max_code_bits=case["max_code_bits"], scale_B=case["B"])
+    rc, s, R, cap = O.derive(p)
+    if rc != O.ORC_OK:
+        pytest.skip("packet too small")
+    beta = 2.0 * case["alpha_q"] + 1.0
+    try:
+        pl = O.plan_from_alpha(p, case["alpha_q"])
+    except O.OracleError as e:
+        # no usable length at this scale, or even the longest code overshoots d: the enumeration agrees
+        if e.code == O.ORC_ERR_BUDGET_TOO_LARGE:
+            assert R * cap[case["max_code_bits"]] > case["d"]
+        else:
+            assert e.code == O.ORC_ERR_SCALE_TOO_SMALL
+            assert all(O.coeff_g(p, y) <= 0 for y in range(1, case["max_code_bits"] + 1))
+        return
+    best = math.inf
+    for combo in itertools.combinations_with_replacement(range(case["max_code_bits"], 0, -1), R):  # y_1 >= ... >= y_R
+        if sum(cap[y] for y in combo) > case["d"]:
+            continue
+        g, _ = gamma_eq5(case["d"], beta, case["B"], cap, combo)
+        best = min(best, g)
+    assert pl.gamma == pytest.approx(best, rel=1e-9, abs=1e-12)
+    if "tiny_g" in case:
+        # B sits right above (Q + 1) / 2 of this length (Proposition 1's condition): it is the shortest usable one
+        assert 0.0 < O.coeff_g(p, case["tiny_g"]) < 0.05 and pl.y_min == case["tiny_g"]
+
+
+def test_all_length_cases_cover_pruned_lengths():
+    """the enumeration above must meet instances where the pruning is active (some length below y_min, some
+    length dominated); all of them leave the constraint k <= d slack (with it active the exchange rule is a
+    heuristic: the candidate-list brute force above skips those instances for the same reason)"""
+    below, dominated = 0, 0
+    for case in ALL_LENGTH_CASES:
+        p = O.make_params(case["d"], case["R"] * case["packet_bits"], packet_bits=case["packet_bits"],
+                          max_code_bits=case["max_code_bits"], scale_B=case["B"])
+        rc, s, R, cap = O.derive(p)
+        if rc != O.ORC_OK:
+            continue
+        Y = O.candidates(p)
+        if not Y:
+            continue
+        below += Y[0] > 1
+        dominated += any(y not in Y for y in range(Y[0], case["max_code_bits"]))
+        assert R * cap[1] <= case["d"]
+    assert below >= 10 and dominated >= 5
+
+
+# ---- which histogram bins enter the fit of the decay exponent (Definition 1): the non-empty normal bins
+# 16 .. 4079 whose survival count N_j lies in 1 .. floor(d / 2)
+
+def _fit_reference(h, d):
+    """least squares of log2(bin edge) on log2(survival count) with numpy, over the window stated above"""
+    h = np.asarray(h, dtype=np.int64)
+    N = np.cumsum(h[::-1])[::-1]
+    j = np.arange(4096)
+    sel = (j >= 16) & (j <= 4079) & (h > 0) & (N >= 1) & (N <= d // 2)
+    if sel.sum() < 2:
+        return -1.0
+    X = np.log2(N[sel].astype(np.float64))
+    Y = ((j[sel] >> 4) - 127) + np.log2(1.0 + (j[sel] & 15) / 16.0)
+    return float(np.polyfit(X, Y, 1)[0])
+
+
+def _two_slope_histogram(d, seed):
+    """ranks 1 .. d/2 follow |x| ~ l^-0.4, the lower half of the ranks falls off much faster (l^-3): a fit that lets
+    points of the lower half in sees a different slope"""
+    rng = np.random.default_rng(seed)
+    l = np.arange(1, d + 1, dtype=np.float64)
+    mag = np.where(l <= d // 2, l ** -0.4, (d // 2) ** -0.4 * (l / (d // 2)) ** -3.0) * 0.8
+    x = (mag * rng.choice([-1.0, 1.0], d)).astype(np.float32)
+    return x
+
+
+def test_fit_window_upper_half_of_the_ranks():
+    d = 300_000
+    x = _two_slope_histogram(d, 3)
+    rc, h = O.histogram(x)
+    a, aq = O.alpha_fit(h, d)
+    ref = _fit_reference(h, d)
+    assert a == pytest.approx(ref, abs=1e-9)
+    assert abs(a + 0.4) < 0.02
+    # the same least squares over all non-empty bins gives a clearly different slope: the window matters here
+    hh = np.asarray(h, dtype=np.int64)
+    N = np.cumsum(hh[::-1])[::-1]
+    j = np.arange(4096)
+    sel = (j >= 16) & (j <= 4079) & (hh > 0)
+    wide = np.polyfit(np.log2(N[sel].astype(np.float64)), ((j[sel] >> 4) - 127) + np.log2(1.0 + (j[sel] & 15) / 16.0), 1)[0]
+    assert abs(wide - a) > 0.05
+
+
+@pytest.mark.parametrize("which", ["bin15", "bin4080", "half_plus_one", "half_exact"])
+def test_fit_window_edges(which):
+    """one extra point right outside each edge of the window would change the slope; it must not be used, and the
+    point right inside (N_j = floor(d/2)) must"""
+    d = 1 << 16
+    h = np.zeros(4096, dtype=np.uint64)
+    # three points on an exact power law |x| = 2^-2 * l^-1/2 ... ranks 4^m at magnitude 2^-m: slope -1/2
+    prev = 0
+    for m in range(2, 6):
+        h[(127 - m) << 4] = 4 ** m - prev
+        prev = 4 ** m
+    rest = d - prev
+    if which == "bin15":            # the top subnormal bin, far off the line, N = prev + 7 <= d/2
+        h[15] = 7
+        rest -= 7
+    elif which == "bin4080":        # a bin of exponent 255 (the histogram may carry it; the fit must not use it)
+        h[4080] = 5
+        rest -= 5
+    elif which == "half_plus_one":  # a normal bin whose survival count is floor(d/2) + 1: outside
+        h[(127 - 40) << 4] = d // 2 + 1 - prev
+        rest -= d // 2 + 1 - prev
+    else:                           # ... and with floor(d/2) exactly: inside, and it bends the fit
+        h[(127 - 40) << 4] = d // 2 - prev
+        rest -= d // 2 - prev
+    h[0] += rest
+    assert int(h.sum()) == d
+    a, aq = O.alpha_fit(h, d)
+    assert a == pytest.approx(_fit_reference(h, d), abs=1e-9)
+    if which == "half_exact":
+        assert abs(a + 0.5) > 0.5
+    elif which == "bin4080":
+        # the counts of the exponent-255 bin still add to every survival count below it: ranks are 5 higher
+        assert abs(a + 0.5) < 0.1
+    else:
+        assert abs(a + 0.5) < 1e-9
+
+
 # ---------------------------------------------------------------- plan invariants
 
 PLAN_CASES = [

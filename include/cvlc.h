@@ -268,6 +268,24 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
                       void* cuda_stream);
 
 /*
+ * Error compensation (Section II: Top_k sparsification is used "with an error compensation mechanism"; the paper
+ * gives no rule of its own, so this is the cited one): the client keeps a memory of what compression lost.
+ * A round with it: cvlc_ec_accumulate_batch (memory <- memory + update, fp32), cvlc_plan_batch on the memory,
+ * cvlc_encode_batch_ec on the memory.  cvlc_encode_batch_ec is cvlc_encode_batch, except that its input buffers
+ * are also its output: when it returns, every transmitted coordinate of memory_dev[i] has given up what the
+ * parameter server rebuilds for it, fp32(centroid value / B), in one fp32 subtraction, and every other coordinate
+ * is unchanged: the memory for the next round.  (The selection reads the buffers before the packing kernel writes
+ * them; cvlc_plan's workspace stays valid for this one encode call.)
+ *  memory_dev / update_dev   HOST arrays of n device pointers (d fp32 each, 16-byte aligned, distinct)
+ * Errors as cvlc_encode_batch; cvlc_ec_accumulate_batch: INVALID_ARG.
+ */
+int cvlc_ec_accumulate_batch(float* const* memory_dev, const float* const* update_dev, uint32_t n, uint64_t d,
+                             void* cuda_stream);
+int cvlc_encode_batch_ec(float* const* memory_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                         const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                         uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+
+/*
  * cvlc_plan_batch followed by cvlc_encode_batch (with the plan's workspace) in one call: Algorithm 1 from the
  * update to the packets.  Selection and ranking need the histogram but not the tuned lengths (they work on
  * the candidates down to an upper bound of k, see cvlc_plan_t::thresh_bin), so with a second stream the
@@ -373,7 +391,7 @@ int cvlc_selftest_wait(uint64_t* word_dev, int32_t* status_dev, uint32_t max_pol
  * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist").  Kernel names: k_zero_words,
  * k_hist, k_plan_fit, k_plan_tune, k_plan_finish, k_encode_init, k_select, k_select_lookback, k_sort_hist,
  * k_sort_scan, k_sort_pass, k_pack, k_decode_prepare, k_fill_zero, k_prefetch_l2, k_decode,
- * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply, k_plan_literal. */
+ * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply, k_plan_literal, k_ec_accumulate. */
 unsigned long long cvlc_launch_count(const char* kernel_name);
 /* Optional kernel timing: after cvlc_profile_select(name, n) the next n launches of that kernel
  * ("*" = of every kernel) are bracketed by a CUDA event pair on their own stream;

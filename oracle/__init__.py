@@ -102,6 +102,10 @@ def lib() -> C.CDLL:
         L.cvlc_plan_literal_oracle.restype = C.c_int
         L.cvlc_plan_literal_oracle.argtypes = [P(OrcParams), f64, u32, u32, C.c_void_p, C.c_void_p, C.c_void_p,
                                                P(u64), P(f64), C.c_void_p]
+        L.cvlc_ec_accumulate_oracle.restype = None
+        L.cvlc_ec_accumulate_oracle.argtypes = [C.c_void_p, C.c_void_p, u64]
+        L.cvlc_ec_residual_oracle.restype = C.c_int
+        L.cvlc_ec_residual_oracle.argtypes = [C.c_void_p, C.c_void_p, u64, u64, C.c_void_p]
         L.cvlc_plan_fixed_oracle.restype = C.c_int
         L.cvlc_plan_fixed_oracle.argtypes = [P(OrcParams), u32, P(OrcPlan)]
         L.cvlc_rank_oracle.restype = C.c_int
@@ -337,6 +341,26 @@ def decode_aggregate(streams: Sequence[np.ndarray], weights: np.ndarray, d: int,
                                             out.ctypes.data, 1 if accumulate else 0)
     if rc != ORC_OK:
         raise OracleError(rc, "decode_aggregate")
+    return out
+
+
+def ec_accumulate(memory: np.ndarray, update: np.ndarray) -> np.ndarray:
+    """memory <- memory + update in fp32, in place; returns memory (the compensated update to compress)"""
+    assert memory.dtype == np.float32 and memory.flags.c_contiguous
+    u = _f32(update)
+    assert u.size == memory.size
+    lib().cvlc_ec_accumulate_oracle(memory.ctypes.data, u.ctypes.data, memory.size)
+    return memory
+
+
+def ec_residual(compensated: np.ndarray, stream: np.ndarray) -> np.ndarray:
+    """the new memory: compensated minus what the parameter server rebuilds from the stream"""
+    a = _f32(compensated)
+    st = np.ascontiguousarray(stream, dtype=np.uint8)
+    out = np.empty_like(a)
+    rc = lib().cvlc_ec_residual_oracle(a.ctypes.data, st.ctypes.data, st.size, a.size, out.ctypes.data)
+    if rc != ORC_OK:
+        raise OracleError(rc, "ec_residual")
     return out
 
 

@@ -934,6 +934,41 @@ int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* 
   return rc;
 }
 
+/* Error compensation (Section II: Top_k "with an error compensation mechanism", Stich et al.): the client keeps
+ * what compression lost and adds it to its next update.  compensated = memory + update is what gets compressed
+ * this round; the new memory is compensated - U_hat, U_hat being the update the parameter server rebuilds from the
+ * stream: the dequantized value divided by B on the transmitted coordinates, zero elsewhere. */
+void cvlc_ec_accumulate_oracle(float* memory, const float* update, uint64_t d) {
+  for (uint64_t i = 0; i < d; ++i) memory[i] = memory[i] + update[i];
+}
+
+int cvlc_ec_residual_oracle(const float* compensated, const uint8_t* stream, uint64_t stream_bytes, uint64_t d,
+                            float* memory_out) {
+  stream_head h;
+  int rc = parse_head(stream, stream_bytes, d, &h);
+  if (rc != ORC_OK) return rc;
+  for (uint64_t i = 0; i < d; ++i) memory_out[i] = compensated[i];
+  for (uint32_t r = 0; r < h.R; ++r) {
+    const uint8_t* pkt = stream + 64 + (size_t)r * (h.packet_bits / 8);
+    uint32_t y = (uint32_t)get_bits(pkt, 8, 8);
+    if (y < 1 || y > ORC_MAX_Y) return ORC_ERR_BAD_STREAM;
+    float lo = bits_float((uint32_t)get_bits(pkt, 16, 32));
+    float hi = bits_float((uint32_t)get_bits(pkt, 48, 32));
+    uint32_t P = (h.packet_bits - h.header_bits) / (h.s + y);
+    for (uint32_t j = 0; j < P; ++j) {
+      uint64_t bitpos = (uint64_t)h.header_bits + (uint64_t)j * (h.s + y);
+      uint64_t pid = get_bits(pkt, bitpos, h.s);
+      uint32_t code = (uint32_t)get_bits(pkt, bitpos + h.s, y);
+      if (pid >= d) return ORC_ERR_BAD_STREAM;
+      float v = (h.quantizer == ORC_QUANT_QSGD) ? cvlc_qsgd_dequantize_oracle(code, lo, y)
+                                                : cvlc_pq_dequantize_oracle(code, lo, hi, y);
+      float u_hat = (float)((double)v / h.B);
+      memory_out[pid] = canon(compensated[pid]) - u_hat;
+    }
+  }
+  return ORC_OK;
+}
+
 /* Section III, step 3: w_{t+1} = w_t - (weighted mean of the decoded updates), in fp32 */
 int cvlc_decode_apply_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
                              const float* weights, uint32_t n_clients, double weight_total,

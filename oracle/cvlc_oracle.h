@@ -124,6 +124,11 @@ int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan
 int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
                                  const float* weights, uint32_t n_clients, double weight_total,
                                  uint64_t d, float* out, int accumulate);
+/* error compensation: memory <- memory + update before compression; memory_out = compensated - (what the server
+ * rebuilds from the stream) after it */
+void cvlc_ec_accumulate_oracle(float* memory, const float* update, uint64_t d);
+int cvlc_ec_residual_oracle(const float* compensated, const uint8_t* stream, uint64_t stream_bytes, uint64_t d,
+                            float* memory_out);
 /* model <- model - aggregate (Section III, step 3) */
 int cvlc_decode_apply_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
                              const float* weights, uint32_t n_clients, double weight_total,

@@ -47,7 +47,7 @@ EXPORTS = [
     "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math", "cvlc_histogram_batch", "cvlc_plan_from_histogram_batch", "cvlc_decode_apply",
     "cvlc_decode_aggregate_noalloc", "cvlc_compress_batch", "cvlc_selftest_wait", "cvlc_plan_literal",
-    "cvlc_plan_literal_workspace_bytes", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
+    "cvlc_plan_literal_workspace_bytes", "cvlc_ec_accumulate_batch", "cvlc_encode_batch_ec", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -132,6 +132,10 @@ def lib() -> C.CDLL:
     L.cvlc_plan_literal_workspace_bytes.argtypes = [PP, u32]
     L.cvlc_plan_literal.restype = C.c_int
     L.cvlc_plan_literal.argtypes = [PP, f64, u32, u32, vp, vp, vp, sz, vp]
+    L.cvlc_ec_accumulate_batch.restype = C.c_int
+    L.cvlc_ec_accumulate_batch.argtypes = [vp, vp, u32, u64, vp]
+    L.cvlc_encode_batch_ec.restype = C.c_int
+    L.cvlc_encode_batch_ec.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
     L.cvlc_selftest_wait.restype = C.c_int
     L.cvlc_selftest_wait.argtypes = [vp, vp, u32, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
@@ -300,6 +304,28 @@ def cvlc_compress_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams]
            "cvlc_compress_batch")
 
 
+def cvlc_ec_accumulate_batch(memories: Sequence[torch.Tensor], updates: Sequence[torch.Tensor],
+                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """memory <- memory + update for every client (error compensation, first step of a round)"""
+    n = len(memories)
+    assert len(updates) == n and all(m.dtype == torch.float32 and u.dtype == torch.float32 and m.numel() == u.numel()
+                                     for m, u in zip(memories, updates))
+    _check(lib().cvlc_ec_accumulate_batch(_ptr_array(memories), _ptr_array(updates), n, memories[0].numel(),
+                                          _stream_handle(stream)), "cvlc_ec_accumulate_batch")
+
+
+def cvlc_encode_batch_ec(memories: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor,
+                         outs: Sequence[torch.Tensor], ws: torch.Tensor, max_candidates: int = 0,
+                         stream: Optional[torch.cuda.Stream] = None, plan_ws: Optional[torch.Tensor] = None) -> None:
+    """cvlc_encode_batch on the compensated updates; on return they hold the new error-compensation memories"""
+    n = len(memories)
+    assert len(params) == n and len(outs) == n
+    cap = min(o.numel() for o in outs)
+    _check(lib().cvlc_encode_batch_ec(_ptr_array(memories), _params_array(params), n, _ptr(plans), _ptr(plan_ws),
+                                      _ptr_array(outs), cap, int(max_candidates), _ptr(ws), ws.numel() * ws.element_size(),
+                                      _stream_handle(stream)), "cvlc_encode_batch_ec")
+
+
 class CvlcLiteralPlan(C.Structure):
     _fields_ = [("status", C.c_int32), ("R", C.c_uint32), ("n_k", C.c_uint32), ("sweeps", C.c_uint32),
                 ("k_star", C.c_uint64), ("gamma_star", C.c_double), ("alpha_q", C.c_double), ("beta", C.c_double),
@@ -433,7 +459,7 @@ def cvlc_profile_reset() -> None:
 
 KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan_fit", "k_plan_tune", "k_plan_finish", "k_encode_init", "k_select",
                 "k_select_lookback", "k_sort_hist", "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero",
-                "k_prefetch_l2", "k_decode", "k_noalloc_publish_status", "k_selftest", "k_hist_check", "k_apply"]
+                "k_prefetch_l2", "k_decode", "k_noalloc_publish_status", "k_selftest", "k_hist_check", "k_apply", "k_plan_literal", "k_ec_accumulate"]
 
 
 def cvlc_profile_read(kernel_name: str = "*"):

@@ -292,9 +292,9 @@ int cvlc_plan_fixed(const float* x_dev, const cvlc_params* p, uint32_t y, cvlc_p
   return cvlc_plan_batch(&x_dev, p, 1, y, plan_dev, ws_dev, ws_bytes, cuda_stream);
 }
 
-int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
-                      const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
-                      uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+static int encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                        const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                        uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream, int write_residual) {
   if (!x_dev || !params || !streams_dev || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
   Shape S;
   ClientDesc desc[CVLC_MAX_BATCH];
@@ -330,9 +330,33 @@ int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint
   if (ws_bytes < enc_layout(S.d, n, cap).total) return CVLC_ERR_WORKSPACE_TOO_SMALL;
   if (!pack_fits(S)) return CVLC_ERR_INVALID_ARG;
   if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
-  return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream), nullptr) == cudaSuccess
+  return launch_encode(desc, n, S, cap, plan_ws_dev, ws_dev, static_cast<cudaStream_t>(cuda_stream), nullptr, write_residual) ==
+                 cudaSuccess
              ? CVLC_OK
              : CVLC_ERR_CUDA;
+}
+
+int cvlc_encode_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                      const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                      uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  return encode_batch(x_dev, params, n, plans_dev, plan_ws_dev, streams_dev, stream_capacity, max_candidates, ws_dev,
+                      ws_bytes, cuda_stream, 0);
+}
+
+int cvlc_encode_batch_ec(float* const* memory_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                         const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                         uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  return encode_batch(const_cast<const float* const*>(memory_dev), params, n, plans_dev, plan_ws_dev, streams_dev,
+                      stream_capacity, max_candidates, ws_dev, ws_bytes, cuda_stream, 1);
+}
+
+int cvlc_ec_accumulate_batch(float* const* memory_dev, const float* const* update_dev, uint32_t n, uint64_t d,
+                             void* cuda_stream) {
+  if (!memory_dev || !update_dev || n == 0 || n > CVLC_MAX_BATCH || d < 2 || d > (1ull << 31)) return CVLC_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n; ++i)
+    if (!aligned(memory_dev[i], 16) || !aligned(update_dev[i], 16) || memory_dev[i] == update_dev[i]) return CVLC_ERR_INVALID_ARG;
+  return launch_ec_accumulate(memory_dev, update_dev, n, d, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CVLC_OK
+                                                                                                                  : CVLC_ERR_CUDA;
 }
 
 // Two events per device order the two streams of cvlc_compress_batch (created on first use, kept until exit).
@@ -390,7 +414,7 @@ int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, ui
   if (launch_plan_front(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
   if (!two) {
     if (launch_plan_back(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
-    return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, nullptr) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+    return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, nullptr, 0) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
   }
   // the length tuning reads the histograms' fit only; selection and ranking do not need its result
   cudaEvent_t fork, join;
@@ -398,7 +422,7 @@ int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, ui
   if (cudaEventRecord(fork, main_st) != cudaSuccess || cudaStreamWaitEvent(side_st, fork, 0) != cudaSuccess) return CVLC_ERR_CUDA;
   if (launch_plan_back(desc, n, S, plan_ws_dev, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
   if (cudaEventRecord(join, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
-  return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, join) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+  return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, join, 0) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, const void* plan_ws_dev,

@@ -207,7 +207,7 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 enum KernelId {
   kKZeroWords = 0, kKHist, kKPlanFit, kKPlanTune, kKPlanFinish, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan,
   kKSortPass, kKPack, kKDecodePrepare, kKFillZero, kKPrefetchL2, kKDecode, kKNoallocStatus, kKSelftest, kKHistCheck, kKApply,
-  kKPlanLiteral, kNumKernelIds
+  kKPlanLiteral, kKEcAccumulate, kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -248,8 +248,11 @@ cudaError_t launch_plan_literal(const cvlc_params& p, double alpha_q, uint32_t s
 cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st);
 // wait_before_pack: an event the stream waits for right before the packing kernel (the length tuning on
 // another stream), or nullptr
+// write_residual: the packing kernel also turns the encoder's input into the error-compensation memory (the input
+// buffers are written: every sent coordinate loses what the parameter server rebuilds for it)
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack);
+                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack, int write_residual);
+cudaError_t launch_ec_accumulate(float* const* memory, const float* const* update, uint32_t n, uint64_t d, cudaStream_t st);
 cudaError_t launch_selftest_wait(unsigned long long* word, int32_t* status, uint32_t max_polls, cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,

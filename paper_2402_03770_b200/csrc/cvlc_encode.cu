@@ -924,7 +924,7 @@ constexpr int kPackGroup = 1;  // packets per warp (more of them amortise the le
 template <int CAP, bool QSGD>
 __global__ void __launch_bounds__(kPackThreads)
 k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Shape shape, unsigned char* ws,
-       const __grid_constant__ EncLayout L, uint32_t warp_bytes) {
+       const __grid_constant__ EncLayout L, uint32_t warp_bytes, int write_residual) {
   extern __shared__ __align__(16) unsigned char s_pack[];  // per warp: packet words; QSGD: then cap(1) squares
   EncHeader* hdr = reinterpret_cast<EncHeader*>(ws);
   if (block_sees_error(&hdr->status)) return;
@@ -938,6 +938,9 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   unsigned char* s_mine = s_pack + (size_t)warp * warp_bytes;
   uint32_t* words = reinterpret_cast<uint32_t*>(s_mine);
   uint32_t* stream_words = reinterpret_cast<uint32_t*>(cd.stream);
+  // error compensation: the encoder's input is memory + update and becomes the new memory, i.e. every sent
+  // coordinate gives up what the parameter server will rebuild for it (its centroid value divided by B)
+  float* __restrict__ residual = write_residual ? const_cast<float*>(cd.x) : nullptr;
 
   const uint32_t mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask)[c];
   const int flips = __popc(~mask & ((1u << kSortPasses) - 1u));
@@ -1058,6 +1061,12 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         }
         const uint32_t code = (sign << (y - 1)) | level;
         put(j, (unsigned long long)pid | ((unsigned long long)code << s));
+        if (residual) {
+          const float mag = (float)__dmul_rn((double)level, __ddiv_rn(dn, sqd));
+          const float v = sign ? -mag : mag;
+          const float xv = __uint_as_float(key ? (key | ((uint32_t)pair & 0x80000000u)) : 0u);
+          residual[pid] = __fsub_rn(xv, (float)__ddiv_rn((double)v, cd.scale_B));
+        }
       }
     } else {
       // ---- PQ: minimum / maximum of the packet's signed values (its centroid distribution) ----
@@ -1083,6 +1092,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
       const double dlo = (double)lo;
       const double den = __dsub_rn((double)hi, dlo);
       const double scale = (hi != lo) ? __ddiv_rn(Lc, den) : 0.0;
+      const double cstep = (hi != lo) ? __ddiv_rn(den, Lc) : 0.0;  // distance of two centroids
       for (uint32_t j = lane; j < P; j += 32) {
         const unsigned long long pair = seg[j];
         const uint32_t key = (uint32_t)(pair >> 32);
@@ -1110,6 +1120,10 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
           }
         }
         put(j, (unsigned long long)pid | ((unsigned long long)code << s));
+        if (residual) {
+          const float v = (hi != lo) ? (float)__dadd_rn(dlo, __dmul_rn((double)code, cstep)) : lo;
+          residual[pid] = __fsub_rn(__uint_as_float(b), (float)__ddiv_rn((double)v, cd.scale_B));
+        }
       }
     }  // PQ
 
@@ -1159,7 +1173,8 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
 
 template <int CAP>
 static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                                   const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack) {
+                                   const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack,
+                                   int write_residual) {
   static bool attr_done[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -1225,17 +1240,66 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
   {
     LaunchScope ls(kKPack, st);
     if (qsgd)
-      k_pack<CAP, true><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp);
+      k_pack<CAP, true><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp, write_residual);
     else
-      k_pack<CAP, false><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp);
+      k_pack<CAP, false><<<dim3(pack_grid, n), kPackThreads, pack_smem, st>>>(batch, shape, w, L, (uint32_t)pack_warp, write_residual);
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
-                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack) {
-  if (n <= (uint32_t)kSmallBatch) return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack);
-  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack);
+                          const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack, int write_residual) {
+  if (n <= (uint32_t)kSmallBatch)
+    return launch_encode_t<kSmallBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack, write_residual);
+  return launch_encode_t<kLargeBatch>(clients, n, shape, capacity, plan_ws, ws, st, wait_before_pack, write_residual);
+}
+
+// memory <- memory + update in fp32, for every client of a batch (the first step of a round with error compensation)
+struct EcPair {
+  float* memory;
+  const float* update;
+};
+struct EcBatch {
+  uint32_t n, pad;
+  EcPair c[CVLC_MAX_BATCH];
+};
+
+__global__ void __launch_bounds__(256)
+k_ec_accumulate(const __grid_constant__ EcBatch batch, uint64_t d) {
+  const uint64_t nvec = d >> 2;
+  const uint64_t per_client = nvec + 1;  // float4 units and one unit for the ragged tail
+  const uint64_t total = per_client * batch.n;
+  for (uint64_t g = (uint64_t)blockIdx.x * 256 + threadIdx.x; g < total; g += (uint64_t)gridDim.x * 256) {
+    const uint32_t c = (uint32_t)(g / per_client);
+    const uint64_t v = g - (uint64_t)c * per_client;
+    float* m = batch.c[c].memory;
+    const float* u = batch.c[c].update;
+    if (v < nvec) {
+      float4 a = reinterpret_cast<float4*>(m)[v];
+      const float4 b = __ldg(reinterpret_cast<const float4*>(u) + v);
+      a.x = __fadd_rn(a.x, b.x);
+      a.y = __fadd_rn(a.y, b.y);
+      a.z = __fadd_rn(a.z, b.z);
+      a.w = __fadd_rn(a.w, b.w);
+      reinterpret_cast<float4*>(m)[v] = a;
+    } else {
+      for (uint64_t i = nvec << 2; i < d; ++i) m[i] = __fadd_rn(m[i], u[i]);
+    }
+  }
+}
+
+cudaError_t launch_ec_accumulate(float* const* memory, const float* const* update, uint32_t n, uint64_t d, cudaStream_t st) {
+  EcBatch batch;
+  batch.n = n;
+  batch.pad = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    batch.c[i].memory = memory[i];
+    batch.c[i].update = update[i];
+  }
+  const uint64_t want = (((d >> 2) + 1) * n + 255) / 256;
+  const unsigned grid = (unsigned)(want < (uint64_t)(8 * kNumSM) ? want : 8 * kNumSM);
+  { LaunchScope ls(kKEcAccumulate, st); k_ec_accumulate<<<grid, 256, 0, st>>>(batch, d); }
+  return cudaGetLastError();
 }
 
 // The bounded wait of the look-back scans, run on a word nobody publishes: after max_polls polls it gives up,

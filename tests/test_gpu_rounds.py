@@ -151,3 +151,55 @@ def test_model_step(env, d):
     agg.apply(n, md2, scratch)
     assert agg.status() == B.CVLC_ERR_BAD_STREAM
     assert (md2.cpu().numpy() == model).all()
+
+
+@pytest.mark.parametrize("quantizer,use_plan_ws", [(0, True), (0, False), (1, True)])
+def test_error_compensation_over_rounds(env, quantizer, use_plan_ws):
+    """three rounds with the error-compensation memory, three clients per batch: the memories (every coordinate)
+    and the streams equal the oracle's bit for bit, round after round"""
+    torch, B = env
+    dev = torch.device("cuda:0")
+    d, n, T = 70_003, 3, 3
+    rng = np.random.default_rng(17)
+    mem_ref = [np.zeros(d, np.float32) for _ in range(n)]
+    mem_gpu = [torch.zeros(d, dtype=torch.float32, device=dev) for _ in range(n)]
+    scale = [None] * n
+    for t in range(T):
+        updates = [(rng.laplace(0, 1e-2, d) * (1.0 + c)).astype(np.float32) for c in range(n)]
+        if t == 1:
+            updates[1][::3] = -0.0
+        pds = [params_dict(d, 9 * 4096, packet_bits=4096, seed=40 + c, client_id=c, round=t, quantizer=quantizer,
+                           scale_B=scale[c]) for c in range(n)]
+        # oracle: accumulate, plan, encode, residual
+        ref_streams, ref_plans = [], []
+        for c in range(n):
+            a = O.ec_accumulate(mem_ref[c], updates[c])
+            po = oracle_params(pds[c])
+            pl = O.plan(a, po)
+            st = O.encode(a, po, pl)
+            mem_ref[c] = O.ec_residual(a, st)
+            ref_streams.append(st)
+            ref_plans.append(pl)
+        # CUDA path
+        params = [gpu_params(pd) for pd in pds]
+        B.cvlc_ec_accumulate_batch(mem_gpu, [torch.from_numpy(u).to(dev) for u in updates])
+        enc = B.BatchEncoder(params, dev)
+        enc.plan(mem_gpu)
+        B.cvlc_encode_batch_ec(mem_gpu, params, enc.plans, enc.outs, enc.enc_ws, plan_ws=enc.plan_ws if use_plan_ws else None)
+        assert enc.status() == B.CVLC_OK
+        for c in range(n):
+            assert_plan_equal(enc.read_plan(c), plan_fields(ref_plans[c]))
+            assert (enc.outs[c].cpu().numpy() == ref_streams[c]).all(), (t, c)
+            got = mem_gpu[c].cpu().numpy()
+            assert (got.view(np.uint32) == mem_ref[c].view(np.uint32)).all(), (t, c)
+            scale[c] = ref_plans[c].B_next
+    assert all(np.abs(m).max() > 0 for m in mem_ref)
+
+
+def test_ec_accumulate_rejects_bad_arguments(env):
+    torch, B = env
+    dev = torch.device("cuda:0")
+    m = torch.zeros(1000, dtype=torch.float32, device=dev)
+    with pytest.raises(B.CvlcError) as e:
+        B.cvlc_ec_accumulate_batch([m], [m])                      # memory and update must be distinct buffers
+    assert e.value.code == B.CVLC_ERR_INVALID_ARG

@@ -34,16 +34,13 @@ METRIC = "encode+decode_aggregate throughput (4*d*clients / step time)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per client and launch from the committed ncu captures
-# (profiles/: resnet18 shape, 2 bits per coordinate, PQ; 32 clients, k_hist 8 clients) of the kernels whose
-# traffic grows in proportion to the client count once their working set is beyond the L2; scaled to the
-# clients of a launch, None for any other configuration or fewer than 32 clients per launch.  k_sort_pass:
-# mean over the four launches of a step (three move data, one is skipped on the device).
+# dram__bytes_read.sum + dram__bytes_write.sum per client and launch, from one ncu capture of the kernels as they
+# stand (resnet18 shape, 2 bits per coordinate, PQ, 32 clients per launch: working sets beyond the L2, traffic in
+# proportion to the clients); scaled to the clients of a launch, None for any other configuration, for fewer than
+# 32 clients per launch, and for a kernel that has changed since its capture.
 NCU_TRAFFIC_BYTES_PER_CLIENT = {
-    "k_select": (1435.81e6 + 169.36e6) / 32,
-    "k_sort_pass": (189.95e6 + 154.89e6 + 189.80e6 + 154.62e6 + 187.02e6 + 154.29e6 + 0.08e6) / 32 / 4,
-    "k_hist": (358.52e6 + 5.24e6) / 8,
 }
+NOMINAL_HBM_GBS = 8000.0
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -67,6 +64,8 @@ def parse_args():
     ap.add_argument("--e2e-batch", type=int, default=10, help="clients per call of the end-to-end leg: host-to-device copies of one sub-batch overlap the kernels of the previous ones")
     ap.add_argument("--e2e-streams", type=int, default=3)
     ap.add_argument("--cpu-sample-clients", type=int, default=3)
+    ap.add_argument("--sustain-seconds", type=float, default=3.0,
+                    help="after the timed steps, repeat the step back to back for this long and report the sustained rate (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -84,7 +83,7 @@ def measured_hbm_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index: int):
         self.index = index
@@ -113,7 +112,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
@@ -127,8 +126,14 @@ class ClockSampler:
             for name, val in zip(names, parts[2:6]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
+            if len(parts) > 6:
+                try:
+                    power.append(float(parts[6]))
+                except ValueError:
+                    pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_median": float(np.median(power)) if power else None,
+                "power_w_max": max(power) if power else None}
 
 
 # --------------------------------------------------------------------------------------------
@@ -136,6 +141,20 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 
 QUANTIZERS = {"pq": 0, "qsgd": 1}
+
+
+def host_info():
+    """cores and CPU model of the host the oracle is timed on"""
+    model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"host_cores": os.cpu_count(), "host_cpu": model}
 
 
 def oracle_step(w, d, bpc, clients, quantizer=0):
@@ -172,7 +191,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64 plan / f32 data", "data": "synthetic",
         "config": {"workload": f"{w.name} d={d} bits_per_coord={args.bits_per_coord} quantizer={args.quantizer}", "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": dict({"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}, **host_info()),
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "params_per_s": d * n / t,
     }))
@@ -315,6 +334,36 @@ def run_ours(args):
 
     ms_per_step = total_ms / args.steps
     units = d * n_clients * world
+
+    # ---- the same step back to back for a few seconds: what the rate settles at under power and temperature
+    sustained = None
+    if args.sustain_seconds > 0:
+        n_sus = max(args.steps, int(np.ceil(args.sustain_seconds * 1e3 / ms_per_step)))
+        sampler2 = ClockSampler(local_rank)
+        if rank == 0:
+            sampler2.start()
+            time.sleep(0.2)
+        sus_ms, _ = timed(n_sus, False)
+        clocks2 = sampler2.stop() if rank == 0 else None
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "value": 4.0 * units / (sus_ms / n_sus * 1e-3) / 1e9, "unit": UNIT, "clocks": clocks2}
+
+    # ---- what this GPU moves right now: a read-only pass and a copy over 4 GiB (library kernels, as a yardstick beside
+    # the recorded peak: a read-only kernel of the path may exceed a peak that was measured with a copy)
+    probe = None
+    if rank == 0:
+        n_probe = 1 << 30
+        a = torch.empty(n_probe, dtype=torch.float32, device=dev).fill_(1.0)
+        b = torch.empty_like(a)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best_copy = best_read = 0.0
+        for _ in range(5):
+            ev0.record(main); b.copy_(a); ev1.record(main); torch.cuda.synchronize(dev)
+            best_copy = max(best_copy, 8.0 * n_probe / (ev0.elapsed_time(ev1) * 1e-3) / 1e9)
+            ev0.record(main); a.sum(); ev1.record(main); torch.cuda.synchronize(dev)
+            best_read = max(best_read, 4.0 * n_probe / (ev0.elapsed_time(ev1) * 1e-3) / 1e9)
+        probe = {"copy_GBps": best_copy, "read_only_GBps": best_read, "how": "torch copy_ / sum over 2^30 fp32, best of 5, CUDA events"}
+        del a, b
     value = 4.0 * units / (ms_per_step * 1e-3) / 1e9
 
     e2e = None
@@ -341,12 +390,17 @@ def run_ours(args):
     n_groups = len(groups)
     sum_cand = float(sum(p.n_candidates for p in plans))
     sum_k = float(sum(p.k for p in plans))
-    sort_passes_per_step = kernel_times.get("k_sort_pass", (0, 0))[0] / max(1, args.steps)
+    # digit passes that move a client's candidates: its sort key keytop - key has 19 bits below the histogram bins plus
+    # the bits of the bin range between the threshold and the top bin; 9 bits per pass
+    def moving_passes(p):
+        bits = 19 + int(np.ceil(np.log2(max(1, p.top_bin + 1 - p.thresh_bin))))
+        return min(4, (bits + 8) // 9)
+    sort_bytes = float(sum(16.0 * p.n_candidates * moving_passes(p) for p in plans))
     alg_bytes_per_step = {   # algorithmic bytes all launches of one step move
         "k_hist": 4.0 * d * n_clients,
         "k_select": 4.0 * d * n_clients + 8.0 * sum_cand,
         "k_sort_hist": 8.0 * sum_cand,
-        "k_sort_pass": 16.0 * sum_cand * 3.0,           # three digit passes move data (the fourth digit is constant)
+        "k_sort_pass": sort_bytes,
         "k_pack": 8.0 * sum_k + float(n_clients) * stream_bytes,
         "k_decode": float(n_clients) * stream_bytes + 4.0 * d,
         "k_fill_zero": 4.0 * d,
@@ -360,6 +414,7 @@ def run_ours(args):
         if name in alg_bytes_per_step:
             entry["achieved_GBps"] = alg_bytes_per_step[name] / (kms / args.steps * 1e-3) / 1e9
             entry["frac_of_hbm_peak"] = entry["achieved_GBps"] / peak
+            entry["frac_of_nominal_8TBps"] = entry["achieved_GBps"] / NOMINAL_HBM_GBS
         kernels[name] = entry
     dominant = args.profile_kernel or (max(kernel_times.items(), key=lambda kv: kv[1][1])[0] if kernel_times else "")
     roofline = None
@@ -373,6 +428,7 @@ def run_ours(args):
             achieved = per_launch / (kms / kn * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak,
                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                        "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
                         "traffic": ncu_traffic, "launches_timed": kn,
                         "mean_launch_us": kms / kn * 1e3, "algorithmic_bytes_per_launch": per_launch}
         else:
@@ -389,13 +445,15 @@ def run_ours(args):
     # ranking passes, pack, decode): what this multi-pass design has to move
     pass_bytes = sum(alg_bytes_per_step[k] for k in ("k_hist", "k_select", "k_sort_pass", "k_pack", "k_decode"))
     pass_frac = pass_bytes / (ms_per_step * 1e-3) / 1e9 / peak
+    pass_frac_nominal = pass_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         n_s = max(1, min(args.cpu_sample_clients, n_clients))
         t = oracle_step(w, d, bpc, list(range(n_s)), QUANTIZERS[args.quantizer])
-        cpu_baseline = {"value": 4.0 * d * n_s / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                        "sample": f"{n_s} of {n_clients} clients: plan+encode each, decode-aggregate of those {n_s}; {t:.1f} s"}
+        cpu_baseline = dict({"value": 4.0 * d * n_s / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"{n_s} of {n_clients} clients: plan+encode each, decode-aggregate of those {n_s}; {t:.1f} s"},
+                            **host_info())
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -407,6 +465,9 @@ def run_ours(args):
         "params_per_s": units / (ms_per_step * 1e-3),
         "step_min_bytes_frac_of_hbm_peak": step_frac,
         "step_pass_bytes_frac_of_hbm_peak": pass_frac,
+        "step_pass_bytes_frac_of_nominal_8TBps": pass_frac_nominal,
+        "step_pass_bytes": pass_bytes, "target_frac_of_hbm_peak": 0.5, "target_met": bool(pass_frac >= 0.5),
+        "sustained": sustained, "hbm_probe": probe,
         "per_step_ms": per,
         "plan_of_client_0": {"k": int(plans[0].k), "R": int(plans[0].R), "n_candidates": int(plans[0].n_candidates), "alpha_q": plans[0].alpha_q,
                  "lengths": {str(y): int(plans[0].n_y[y]) for y in range(33) if plans[0].n_y[y]}},

@@ -106,6 +106,14 @@ def lib() -> C.CDLL:
         L.cvlc_ec_accumulate_oracle.argtypes = [C.c_void_p, C.c_void_p, u64]
         L.cvlc_ec_residual_oracle.restype = C.c_int
         L.cvlc_ec_residual_oracle.argtypes = [C.c_void_p, C.c_void_p, u64, u64, C.c_void_p]
+        L.cvlc_unframed_header_bytes_oracle.restype = C.c_size_t
+        L.cvlc_unframed_header_bytes_oracle.argtypes = [u32]
+        L.cvlc_unframed_capacity_oracle.restype = C.c_size_t
+        L.cvlc_unframed_capacity_oracle.argtypes = [P(OrcParams)]
+        L.cvlc_encode_unframed_oracle.restype = C.c_int
+        L.cvlc_encode_unframed_oracle.argtypes = [C.c_void_p, P(OrcParams), P(OrcPlan), C.c_void_p, C.c_size_t, P(C.c_size_t)]
+        L.cvlc_decode_aggregate_unframed_oracle.restype = C.c_int
+        L.cvlc_decode_aggregate_unframed_oracle.argtypes = [P(C.c_void_p), P(u64), C.c_void_p, u32, f64, u64, C.c_void_p, C.c_int]
         L.cvlc_plan_fixed_oracle.restype = C.c_int
         L.cvlc_plan_fixed_oracle.argtypes = [P(OrcParams), u32, P(OrcPlan)]
         L.cvlc_rank_oracle.restype = C.c_int
@@ -341,6 +349,38 @@ def decode_aggregate(streams: Sequence[np.ndarray], weights: np.ndarray, d: int,
                                             out.ctypes.data, 1 if accumulate else 0)
     if rc != ORC_OK:
         raise OracleError(rc, "decode_aggregate")
+    return out
+
+
+def encode_unframed(x: np.ndarray, p: OrcParams, plan: OrcPlan) -> np.ndarray:
+    """the unframed (version 2) stream of the same records: returns its bytes"""
+    x = _f32(x)
+    capacity = int(lib().cvlc_unframed_capacity_oracle(C.byref(p)))
+    buf = np.zeros(capacity, dtype=np.uint8)
+    n = C.c_size_t()
+    rc = lib().cvlc_encode_unframed_oracle(x.ctypes.data, C.byref(p), C.byref(plan), buf.ctypes.data, capacity, C.byref(n))
+    if rc != ORC_OK:
+        raise OracleError(rc, "encode_unframed")
+    return buf[:n.value].copy()
+
+
+def unframed_capacity(p: OrcParams) -> int:
+    return int(lib().cvlc_unframed_capacity_oracle(C.byref(p)))
+
+
+def decode_aggregate_unframed(streams: Sequence[np.ndarray], weights: np.ndarray, d: int, *, weight_total: float = 0.0,
+                              out: Optional[np.ndarray] = None, accumulate: bool = False) -> np.ndarray:
+    n = len(streams)
+    streams = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    ptrs = (C.c_void_p * n)(*[s.ctypes.data for s in streams])
+    sizes = (C.c_uint64 * n)(*[s.size for s in streams])
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    if out is None:
+        out = np.zeros(d, dtype=np.float32)
+    rc = lib().cvlc_decode_aggregate_unframed_oracle(ptrs, sizes, w.ctypes.data, n, float(weight_total), d,
+                                                     out.ctypes.data, 1 if accumulate else 0)
+    if rc != ORC_OK:
+        raise OracleError(rc, "decode_aggregate_unframed")
     return out
 
 

@@ -840,6 +840,152 @@ int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan
 }
 
 /* ======================================================================== */
+/* Unframed stream (version 2): the same records without the packet frame.    */
+/* Section IV-C fixes one length per packet and a fixed packet size only       */
+/* because of the header a real network needs; Proposition 1 itself groups the */
+/* top-k by code length.  Here the groups are kept (the records of packet r,   */
+/* longest codes first, with the packet's own centroid distribution, so the    */
+/* plan and its error bound are unchanged), but a block is as long as its      */
+/* records need: no s / y_r fields (a table of n_y and cap(y) in the stream    */
+/* header says which block has which length), no padding, and the position IDs */
+/* of a block are sorted and sent as differences in a Golomb-Rice code.        */
+/* ======================================================================== */
+
+/* Rice parameter of a block of P records out of d coordinates: the gaps between sorted positions are about
+ * d / P, so the low m = floor(log2(d / P)) bits go out verbatim and the rest in unary. */
+static uint32_t rice_param(uint64_t d, uint32_t P) {
+  uint64_t g = d / (uint64_t)P;
+  uint32_t m = 0;
+  while (g >= 2) { g >>= 1; ++m; }
+  return m;
+}
+
+static int cmp_u64_asc(const void* a, const void* b) {
+  uint64_t x = *(const uint64_t*)a, y = *(const uint64_t*)b;
+  return (x > y) - (x < y);
+}
+
+size_t cvlc_unframed_header_bytes_oracle(uint32_t R) { return 64 + 33 * 4 * 2 + 8 + (size_t)R * 8; }
+
+/* upper bound of the stream size: per block 64 header bits and per record 1 + m + y bits, plus fewer than 2P unary
+ * one-bits per block (the differences of a block add up to less than d, and 2^m > d / (2P)) */
+size_t cvlc_unframed_capacity_oracle(const orc_params* p) {
+  uint32_t s, R, cap[ORC_MAX_Y + 1];
+  if (cvlc_derive_oracle(p, &s, &R, cap) != ORC_OK) return 0;
+  uint64_t worst = 0;
+  for (uint32_t y = 1; y <= p->max_code_bits; ++y) {
+    uint64_t bits = 64 + (uint64_t)cap[y] * (1 + rice_param(p->d, cap[y]) + y) + 2 * (uint64_t)cap[y];
+    if (bits > worst) worst = bits;
+  }
+  return cvlc_unframed_header_bytes_oracle(R) + (size_t)((worst * R + 63) / 64) * 8;
+}
+
+int cvlc_encode_unframed_oracle(const float* x, const orc_params* p, const orc_plan* plan, uint8_t* stream,
+                                size_t capacity, size_t* bytes_out) {
+  if (!params_ok(p) || !plan) return ORC_ERR_INVALID_ARG;
+  uint32_t s, R, cap[ORC_MAX_Y + 1];
+  int rc = cvlc_derive_oracle(p, &s, &R, cap);
+  if (rc != ORC_OK) return rc;
+  if (plan->R != R || plan->s != s) return ORC_ERR_INVALID_ARG;
+  uint64_t k = 0, nsum = 0;
+  for (uint32_t y = 1; y <= ORC_MAX_Y; ++y) {
+    if (plan->n_y[y] && cap[y] == 0) return ORC_ERR_INVALID_ARG;
+    k += (uint64_t)plan->n_y[y] * cap[y];
+    nsum += plan->n_y[y];
+  }
+  if (nsum != R || k != plan->k || k > p->d) return ORC_ERR_INVALID_ARG;
+  if (capacity < cvlc_unframed_capacity_oracle(p)) return ORC_ERR_OUTPUT_TOO_SMALL;
+  for (uint64_t i = 0; i < p->d; ++i)
+    if (key_of(x[i]) >= 0x7F800000u) return ORC_ERR_NONFINITE_INPUT;
+
+  uint32_t* rank = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)(k ? k : 1));
+  if (!rank) return ORC_ERR_INVALID_ARG;
+  rc = cvlc_rank_oracle(x, p->d, k, rank);
+  if (rc != ORC_OK) { free(rank); return rc; }
+
+  const size_t head = cvlc_unframed_header_bytes_oracle(R);
+  memset(stream, 0, capacity);
+  put_le(stream + 0, 0x434C5643u, 4);
+  put_le(stream + 4, 2, 2); /* version 2: unframed */
+  put_le(stream + 6, p->quantizer, 1);
+  put_le(stream + 7, s, 1);
+  put_le(stream + 8, p->d, 8);
+  put_le(stream + 16, R, 4);
+  put_le(stream + 20, p->packet_bits, 4);
+  put_le(stream + 24, p->header_bits, 4);
+  put_le(stream + 28, p->client_id, 4);
+  put_le(stream + 32, p->seed, 8);
+  put_le(stream + 40, p->round, 4);
+  put_le(stream + 44, 0, 4);
+  put_le(stream + 48, double_to_bits(p->scale_B), 8);
+  put_le(stream + 56, k, 8);
+  for (uint32_t y = 0; y <= ORC_MAX_Y; ++y) {
+    put_le(stream + 64 + 4 * y, plan->n_y[y], 4);
+    put_le(stream + 64 + 132 + 4 * y, cap[y], 4);
+  }
+  uint8_t* dir = stream + 64 + 264 + 8; /* bit offset of every block inside the body */
+  uint8_t* body = stream + head;
+  uint64_t bit = 0, Z = 0;
+  uint32_t r = 0;
+  uint64_t* recs = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)(cap[1] ? cap[1] : 1));
+  float* seg = (float*)malloc(sizeof(float) * (size_t)(cap[1] ? cap[1] : 1));
+  if (!recs || !seg) { free(rank); free(recs); free(seg); return ORC_ERR_INVALID_ARG; }
+  for (int y = ORC_MAX_Y; y >= 1; --y) {
+    for (uint32_t q = 0; q < plan->n_y[y]; ++q, ++r) {
+      uint32_t P = cap[y];
+      uint32_t m = rice_param(p->d, P);
+      put_le(dir + 8 * (size_t)r, bit, 8);
+      /* the block's centroid distribution is that of the packet it replaces: over its records in rank order */
+      float lo = 0.0f, hi = 0.0f, norm = 0.0f;
+      if (p->quantizer == ORC_QUANT_QSGD) {
+        if (y < 2) { free(rank); free(recs); free(seg); return ORC_ERR_INVALID_ARG; }
+        for (uint32_t j = 0; j < P; ++j) seg[j] = canon(x[rank[Z + j]]);
+        norm = cvlc_qsgd_norm_oracle(seg, P);
+        lo = norm;
+      } else {
+        lo = canon(x[rank[Z]]);
+        hi = lo;
+        for (uint32_t j = 1; j < P; ++j) {
+          float v = canon(x[rank[Z + j]]);
+          if (v < lo) lo = v;
+          if (v > hi) hi = v;
+        }
+      }
+      put_bits(body, bit, float_bits(lo), 32);
+      put_bits(body, bit + 32, float_bits(hi), 32);
+      bit += 64;
+      /* records in ascending position */
+      for (uint32_t j = 0; j < P; ++j) recs[j] = rank[Z + j];
+      qsort(recs, P, sizeof(uint64_t), cmp_u64_asc);
+      uint64_t prev = 0; /* one past the previous position */
+      for (uint32_t j = 0; j < P; ++j) {
+        uint32_t pid = (uint32_t)recs[j];
+        uint32_t rnd = cvlc_philox_coord_oracle(p->seed, p->client_id, p->round, pid);
+        uint32_t code = (p->quantizer == ORC_QUANT_QSGD)
+                            ? cvlc_qsgd_quantize_oracle(canon(x[pid]), norm, (uint32_t)y, rnd)
+                            : cvlc_pq_quantize_oracle(canon(x[pid]), lo, hi, (uint32_t)y, rnd);
+        uint64_t delta = (uint64_t)pid - prev; /* positions skipped since the previous record */
+        uint64_t quo = delta >> m;
+        for (uint64_t u = 0; u < quo; ++u) put_bits(body, bit + u, 1, 1);
+        bit += quo + 1; /* quo ones, then a zero */
+        put_bits(body, bit, delta & (((uint64_t)1 << m) - 1), m);
+        bit += m;
+        put_bits(body, bit, code, (uint32_t)y);
+        bit += (uint32_t)y;
+        prev = (uint64_t)pid + 1;
+      }
+      Z += P;
+    }
+  }
+  put_le(stream + 64 + 264, bit, 8);
+  *bytes_out = head + (size_t)((bit + 63) / 64) * 8;
+  free(rank);
+  free(recs);
+  free(seg);
+  return ORC_OK;
+}
+
+/* ======================================================================== */
 /* Parameter-server side: w_{t+1} = w_t - (1/|S_t|) sum_i U_i (Section III,   */
 /* step 3), with U_i rebuilt from the packets and divided by B_i               */
 /* ======================================================================== */
@@ -850,10 +996,14 @@ typedef struct {
   double B;
 } stream_head;
 
-static int parse_head(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_head* h) {
+static int parse_head_any(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_head* h, uint32_t version);
+
+static int parse_head(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_head* h) { return parse_head_any(st, nbytes, d, h, 1); }
+
+static int parse_head_any(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_head* h, uint32_t version) {
   if (nbytes < 64) return ORC_ERR_BAD_STREAM;
   if (get_le(st, 4) != 0x434C5643u) return ORC_ERR_BAD_STREAM;
-  if (get_le(st + 4, 2) != 1) return ORC_ERR_BAD_STREAM;
+  if (get_le(st + 4, 2) != version) return ORC_ERR_BAD_STREAM;
   h->quantizer = (uint32_t)get_le(st + 6, 1);
   if (h->quantizer != ORC_QUANT_PQ && h->quantizer != ORC_QUANT_QSGD) return ORC_ERR_BAD_STREAM;
   h->s = (uint32_t)get_le(st + 7, 1);
@@ -868,9 +1018,90 @@ static int parse_head(const uint8_t* st, uint64_t nbytes, uint64_t d, stream_hea
   if (h->s != s) return ORC_ERR_BAD_STREAM;
   if (h->packet_bits == 0 || h->packet_bits % 32) return ORC_ERR_BAD_STREAM;
   if (h->header_bits < 80 || h->header_bits >= h->packet_bits) return ORC_ERR_BAD_STREAM;
-  if (64 + (uint64_t)h->R * (h->packet_bits / 8) != nbytes) return ORC_ERR_BAD_STREAM;
+  if (version == 1 && 64 + (uint64_t)h->R * (h->packet_bits / 8) != nbytes) return ORC_ERR_BAD_STREAM;
   if (!(h->B >= 1.0) || !(h->B < 1e300)) return ORC_ERR_BAD_STREAM;
   return ORC_OK;
+}
+
+/* Decode + aggregate of unframed (version 2) streams: the same arithmetic as for packets */
+int cvlc_decode_aggregate_unframed_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
+                                          const float* weights, uint32_t n_clients, double weight_total,
+                                          uint64_t d, float* out, int accumulate) {
+  if (d < 2 || d > ((uint64_t)1 << 31) || n_clients == 0) return ORC_ERR_INVALID_ARG;
+  double W = weight_total;
+  if (W == 0.0) {
+    for (uint32_t i = 0; i < n_clients; ++i) W = W + (double)weights[i];
+  }
+  if (!(W > 0.0)) return ORC_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n_clients; ++i)
+    if (!(weights[i] > 0.0f) || !isfinite(weights[i])) return ORC_ERR_INVALID_ARG;
+  double* acc = (double*)calloc((size_t)d, sizeof(double));
+  if (!acc) return ORC_ERR_INVALID_ARG;
+  int rc = ORC_OK;
+  for (uint32_t i = 0; i < n_clients && rc == ORC_OK; ++i) {
+    stream_head h;
+    const uint8_t* st = streams[i];
+    rc = parse_head_any(st, stream_bytes[i], d, &h, 2);
+    if (rc != ORC_OK) break;
+    const size_t head = cvlc_unframed_header_bytes_oracle(h.R);
+    if (stream_bytes[i] < head) { rc = ORC_ERR_BAD_STREAM; break; }
+    uint32_t n_y[ORC_MAX_Y + 1], cap[ORC_MAX_Y + 1];
+    uint64_t blocks = 0;
+    for (uint32_t y = 0; y <= ORC_MAX_Y; ++y) {
+      n_y[y] = (uint32_t)get_le(st + 64 + 4 * y, 4);
+      cap[y] = (uint32_t)get_le(st + 64 + 132 + 4 * y, 4);
+      blocks += n_y[y];
+      if (n_y[y] && (y == 0 || cap[y] == 0)) rc = ORC_ERR_BAD_STREAM;
+    }
+    uint64_t total_bits = get_le(st + 64 + 264, 8);
+    if (rc != ORC_OK || blocks != h.R || head + ((total_bits + 63) / 64) * 8 != stream_bytes[i]) { rc = ORC_ERR_BAD_STREAM; break; }
+    const uint8_t* dir = st + 64 + 264 + 8;
+    const uint8_t* body = st + head;
+    float coef = (float)((double)weights[i] / (W * h.B));
+    uint32_t r = 0;
+    for (int y = ORC_MAX_Y; y >= 1 && rc == ORC_OK; --y) {
+      for (uint32_t q = 0; q < n_y[y] && rc == ORC_OK; ++q, ++r) {
+        uint32_t P = cap[y];
+        uint32_t m = rice_param(d, P);
+        uint64_t bit = get_le(dir + 8 * (size_t)r, 8);
+        if (bit + 64 > total_bits) { rc = ORC_ERR_BAD_STREAM; break; }
+        float lo = bits_float((uint32_t)get_bits(body, bit, 32));
+        float hi = bits_float((uint32_t)get_bits(body, bit + 32, 32));
+        bit += 64;
+        if (h.quantizer == ORC_QUANT_QSGD) {
+          uint32_t nb = float_bits(lo);
+          if (y < 2 || nb >= 0x7F800000u) { rc = ORC_ERR_BAD_STREAM; break; }
+        } else if (!isfinite(lo) || !isfinite(hi) || lo > hi) { rc = ORC_ERR_BAD_STREAM; break; }
+        uint64_t prev = 0;
+        for (uint32_t j = 0; j < P; ++j) {
+          uint64_t quo = 0;
+          while (bit < total_bits && get_bits(body, bit, 1)) { ++quo; ++bit; }
+          if (bit + 1 + m + (uint32_t)y > total_bits) { rc = ORC_ERR_BAD_STREAM; break; }
+          bit += 1;
+          uint64_t delta = (quo << m) | get_bits(body, bit, m);
+          bit += m;
+          uint32_t code = (uint32_t)get_bits(body, bit, (uint32_t)y);
+          bit += (uint32_t)y;
+          uint64_t pid = prev + delta;
+          if (pid >= d) { rc = ORC_ERR_BAD_STREAM; break; }
+          prev = pid + 1;
+          float v = (h.quantizer == ORC_QUANT_QSGD) ? cvlc_qsgd_dequantize_oracle(code, lo, (uint32_t)y)
+                                                    : cvlc_pq_dequantize_oracle(code, lo, hi, (uint32_t)y);
+          acc[pid] = acc[pid] + (double)coef * (double)v;
+        }
+      }
+    }
+  }
+  if (rc == ORC_OK) {
+    for (uint64_t i = 0; i < d; ++i) {
+      if (accumulate)
+        out[i] = (float)((double)out[i] + acc[i]);
+      else
+        out[i] = (float)acc[i];
+    }
+  }
+  free(acc);
+  return rc;
 }
 
 int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,

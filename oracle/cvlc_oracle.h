@@ -120,6 +120,17 @@ float cvlc_qsgd_dequantize_oracle(uint32_t code, float norm, uint32_t y);
 int cvlc_encode_oracle(const float* x, const orc_params* p, const orc_plan* plan, uint8_t* stream,
                        size_t capacity, uint32_t* ranked_idx_out /* k entries or NULL */);
 
+/* --- unframed stream (version 2): the packets' records without the frame; blocks in the packets' order, each with
+ * its centroid distribution (64 bits) and its records sorted by position, positions as Golomb-Rice coded
+ * differences, lengths and capacities in a table of the stream header, a directory of block offsets ------------- */
+size_t cvlc_unframed_header_bytes_oracle(uint32_t R);
+size_t cvlc_unframed_capacity_oracle(const orc_params* p);
+int cvlc_encode_unframed_oracle(const float* x, const orc_params* p, const orc_plan* plan, uint8_t* stream,
+                                size_t capacity, size_t* bytes_out);
+int cvlc_decode_aggregate_unframed_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
+                                          const float* weights, uint32_t n_clients, double weight_total,
+                                          uint64_t d, float* out, int accumulate);
+
 /* --- decoding ------------------------------------------------------------ */
 int cvlc_decode_aggregate_oracle(const uint8_t* const* streams, const uint64_t* stream_bytes,
                                  const float* weights, uint32_t n_clients, double weight_total,

@@ -99,3 +99,61 @@ def dequantize_qsgd(pk: Packet) -> np.ndarray:
     negative = ((pk.cid >> np.uint64(pk.y - 1)) & np.uint64(1)).astype(bool)
     mag = (level * (np.float64(pk.lo) / np.float64(sq))).astype(np.float32)
     return np.where(negative, -mag, mag).astype(np.float32)
+
+
+# ---- unframed stream (version 2) ---------------------------------------------------------------------------------
+# header (64 bytes, as version 1 with version = 2) | n_y[33] u32 | cap[33] u32 | total body bits u64 |
+# directory: R x u64 bit offsets | body: blocks in descending code length, each {lo 32, hi 32, records in ascending
+# position: Golomb-Rice(position - previous position - 1, previous = -1 at the start of a block) then CID (y bits)};
+# Rice parameter m = floor(log2(d // P)); a value v is sent as v >> m one-bits, a zero bit, then the low m bits.
+
+@dataclass
+class UnframedStream:
+    head: Stream                 # packets: one Packet per block (s = 0: the blocks carry no s field)
+    total_bits: int
+    directory: np.ndarray
+    n_y: List[int]
+    cap: List[int]
+    tail_zero: bool
+
+
+def parse_unframed(stream: np.ndarray) -> UnframedStream:
+    raw = np.ascontiguousarray(stream, dtype=np.uint8).tobytes()
+    (magic, version, quantizer, s, d, R, packet_bits, header_bits, client_id, seed, rnd, zero, scale_B,
+     k) = struct.unpack_from("<IHBBQIIIIQIIdQ", raw, 0)
+    assert version == 2 and zero == 0
+    n_y = list(struct.unpack_from("<33I", raw, 64))
+    cap = list(struct.unpack_from("<33I", raw, 64 + 132))
+    total_bits = struct.unpack_from("<Q", raw, 64 + 264)[0]
+    directory = np.frombuffer(raw, dtype="<u8", count=R, offset=64 + 264 + 8).copy()
+    head_bytes = 64 + 264 + 8 + 8 * R
+    assert len(raw) == head_bytes + ((total_bits + 63) // 64) * 8
+    bits = np.unpackbits(np.frombuffer(raw, dtype=np.uint8, offset=head_bytes), bitorder="little")
+    out = Stream(magic, version, quantizer, s, d, R, packet_bits, header_bits, client_id, seed, rnd, scale_B, k, [])
+    pos, r = 0, 0
+    for y in range(32, 0, -1):
+        for _ in range(n_y[y]):
+            assert directory[r] == pos
+            P = cap[y]
+            m = max(0, (d // P).bit_length() - 1)
+            lo = struct.unpack("<f", struct.pack("<I", _field(bits, pos, 32)))[0]
+            hi = struct.unpack("<f", struct.pack("<I", _field(bits, pos + 32, 32)))[0]
+            pos += 64
+            pids, cids = [], []
+            prev = 0
+            for _j in range(P):
+                q = 0
+                while bits[pos]:
+                    q += 1
+                    pos += 1
+                pos += 1
+                delta = (q << m) | _field(bits, pos, m)
+                pos += m
+                cids.append(_field(bits, pos, y))
+                pos += y
+                pids.append(prev + delta)
+                prev = prev + delta + 1
+            out.packets.append(Packet(0, y, lo, hi, np.array(pids, dtype=np.uint64), np.array(cids, dtype=np.uint64), True))
+            r += 1
+    assert pos == total_bits and r == R
+    return UnframedStream(out, total_bits, directory, n_y, cap, not bits[pos:].any())

@@ -286,6 +286,34 @@ int cvlc_encode_batch_ec(float* const* memory_dev, const cvlc_params* params, ui
                          uint64_t max_candidates, void* ws_dev, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Unframed stream (version 2).  Section IV-C gives every packet one code length and a fixed size because a packet
+ * on a real network needs a header; Proposition 1 / Eq. (1) itself only groups the top-k coordinates by code
+ * length.  This format keeps the plan's groups (block r = the records of packet r, longest codes first, with that
+ * packet's centroid distribution, so k, the lengths and the error bound are those of cvlc_plan) and drops the
+ * frame: no s / y_r fields (a table of n_y and cap(y) in the stream header), no padding, and the position IDs of
+ * a block are sorted and sent as Golomb-Rice coded differences (parameter floor(log2(d / P)) for a block of P
+ * records).  Records then differ in length: their bit offsets are an exclusive prefix sum of the per-record code
+ * lengths (warp scans inside a block, a decoupled look-back across the blocks of a client).  The layout is in the
+ * header of csrc/cvlc_unframed.cu.  A stream decodes to exactly the aggregate of the framed stream of the same plan.
+ *  stream_capacity      bytes of every output buffer, at least cvlc_unframed_stream_capacity(p) (0: the shape is not
+ *                       supported: a block may hold at most 2048 records, i.e. (b - H) / (s + 1) <= 2048)
+ *  stream_bytes_dev     DEVICE array of n uint64 that receives the streams' lengths (they depend on the data), or NULL;
+ *                       the length is also 336 + 8 R + 8 * ceil(total bits / 64) with the total at byte 328 of the stream
+ *  uf_ws_dev            cvlc_unframed_workspace_bytes(p, n) bytes
+ * Other arguments and errors as cvlc_encode_batch / cvlc_decode_aggregate (which takes framed streams only; the two
+ * decoders refuse each other's streams with BAD_STREAM).
+ */
+size_t cvlc_unframed_stream_capacity(const cvlc_params* p);
+size_t cvlc_unframed_workspace_bytes(const cvlc_params* p, uint32_t n);
+int cvlc_encode_unframed_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                               const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                               uint64_t* stream_bytes_dev, uint64_t max_candidates, void* enc_ws_dev, size_t enc_ws_bytes,
+                               void* uf_ws_dev, size_t uf_ws_bytes, void* cuda_stream);
+int cvlc_decode_aggregate_unframed(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev,
+                                   const float* weights_dev, uint32_t n_clients, double weight_total, uint64_t d,
+                                   float* out_dev, int accumulate, void* ws_dev, size_t ws_bytes, void* cuda_stream);
+
+/*
  * cvlc_plan_batch followed by cvlc_encode_batch (with the plan's workspace) in one call: Algorithm 1 from the
  * update to the packets.  Selection and ranking need the histogram but not the tuned lengths (they work on
  * the candidates down to an upper bound of k, see cvlc_plan_t::thresh_bin), so with a second stream the
@@ -391,7 +419,7 @@ int cvlc_selftest_wait(uint64_t* word_dev, int32_t* status_dev, uint32_t max_pol
  * (all kernels when kernel_name is NULL or "", else the named one, e.g. "k_hist").  Kernel names: k_zero_words,
  * k_hist, k_plan_fit, k_plan_tune, k_plan_finish, k_encode_init, k_select, k_select_lookback, k_sort_hist,
  * k_sort_scan, k_sort_pass, k_pack, k_decode_prepare, k_fill_zero, k_prefetch_l2, k_decode,
- * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply, k_plan_literal, k_ec_accumulate. */
+ * k_noalloc_publish_status, k_selftest, k_hist_check, k_apply, k_plan_literal, k_ec_accumulate, k_pack_unframed, k_decode_unframed. */
 unsigned long long cvlc_launch_count(const char* kernel_name);
 /* Optional kernel timing: after cvlc_profile_select(name, n) the next n launches of that kernel
  * ("*" = of every kernel) are bracketed by a CUDA event pair on their own stream;

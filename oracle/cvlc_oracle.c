@@ -1089,6 +1089,9 @@ int cvlc_decode_aggregate_unframed_oracle(const uint8_t* const* streams, const u
                                                     : cvlc_pq_dequantize_oracle(code, lo, hi, (uint32_t)y);
           acc[pid] = acc[pid] + (double)coef * (double)v;
         }
+        /* blocks follow one another without gaps: a block ends where the directory says the next one starts */
+        uint64_t next = (r + 1 < h.R) ? get_le(dir + 8 * ((size_t)r + 1), 8) : total_bits;
+        if (rc == ORC_OK && bit != next) rc = ORC_ERR_BAD_STREAM;
       }
     }
   }

@@ -47,7 +47,8 @@ EXPORTS = [
     "cvlc_encode_batch_workspace_bytes", "cvlc_plan_batch", "cvlc_encode_batch", "cvlc_decode_aggregate", "cvlc_read_status",
     "cvlc_selftest_philox", "cvlc_selftest_math", "cvlc_histogram_batch", "cvlc_plan_from_histogram_batch", "cvlc_decode_apply",
     "cvlc_decode_aggregate_noalloc", "cvlc_compress_batch", "cvlc_selftest_wait", "cvlc_plan_literal",
-    "cvlc_plan_literal_workspace_bytes", "cvlc_ec_accumulate_batch", "cvlc_encode_batch_ec", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
+    "cvlc_plan_literal_workspace_bytes", "cvlc_ec_accumulate_batch", "cvlc_encode_batch_ec",
+    "cvlc_unframed_stream_capacity", "cvlc_unframed_workspace_bytes", "cvlc_encode_unframed_batch", "cvlc_decode_aggregate_unframed", "cvlc_launch_count", "cvlc_profile_select", "cvlc_profile_reset", "cvlc_profile_read",
 ]
 
 
@@ -136,6 +137,14 @@ def lib() -> C.CDLL:
     L.cvlc_ec_accumulate_batch.argtypes = [vp, vp, u32, u64, vp]
     L.cvlc_encode_batch_ec.restype = C.c_int
     L.cvlc_encode_batch_ec.argtypes = [vp, PP, u32, vp, vp, vp, sz, u64, vp, sz, vp]
+    L.cvlc_unframed_stream_capacity.restype = sz
+    L.cvlc_unframed_stream_capacity.argtypes = [PP]
+    L.cvlc_unframed_workspace_bytes.restype = sz
+    L.cvlc_unframed_workspace_bytes.argtypes = [PP, u32]
+    L.cvlc_encode_unframed_batch.restype = C.c_int
+    L.cvlc_encode_unframed_batch.argtypes = [vp, PP, u32, vp, vp, vp, sz, vp, u64, vp, sz, vp, sz, vp]
+    L.cvlc_decode_aggregate_unframed.restype = C.c_int
+    L.cvlc_decode_aggregate_unframed.argtypes = [vp, vp, vp, u32, f64, u64, vp, C.c_int, vp, sz, vp]
     L.cvlc_selftest_wait.restype = C.c_int
     L.cvlc_selftest_wait.argtypes = [vp, vp, u32, vp]
     L.cvlc_decode_aggregate.restype = C.c_int
@@ -326,6 +335,39 @@ def cvlc_encode_batch_ec(memories: Sequence[torch.Tensor], params: Sequence[Cvlc
                                       _stream_handle(stream)), "cvlc_encode_batch_ec")
 
 
+def cvlc_unframed_stream_capacity(p: CvlcParams) -> int:
+    return int(lib().cvlc_unframed_stream_capacity(C.byref(p)))
+
+
+def cvlc_unframed_workspace_bytes(p: CvlcParams, n: int) -> int:
+    return int(lib().cvlc_unframed_workspace_bytes(C.byref(p), int(n)))
+
+
+def cvlc_encode_unframed_batch(xs: Sequence[torch.Tensor], params: Sequence[CvlcParams], plans: torch.Tensor,
+                               outs: Sequence[torch.Tensor], sizes: Optional[torch.Tensor], enc_ws: torch.Tensor,
+                               uf_ws: torch.Tensor, max_candidates: int = 0, stream: Optional[torch.cuda.Stream] = None,
+                               plan_ws: Optional[torch.Tensor] = None) -> None:
+    """the unframed (version 2) streams of n planned clients; sizes: device int64[n] that receives their lengths"""
+    n = len(xs)
+    assert len(params) == n and len(outs) == n
+    cap = min(o.numel() for o in outs)
+    _check(lib().cvlc_encode_unframed_batch(_ptr_array(xs), _params_array(params), n, _ptr(plans), _ptr(plan_ws),
+                                            _ptr_array(outs), cap, _ptr(sizes), int(max_candidates), _ptr(enc_ws),
+                                            enc_ws.numel() * enc_ws.element_size(), _ptr(uf_ws),
+                                            uf_ws.numel() * uf_ws.element_size(), _stream_handle(stream)),
+           "cvlc_encode_unframed_batch")
+
+
+def cvlc_decode_aggregate_unframed(stream_ptrs: torch.Tensor, stream_bytes: torch.Tensor, weights: torch.Tensor,
+                                   n_clients: int, weight_total: float, d: int, out: torch.Tensor, accumulate: bool,
+                                   ws: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    assert weights.dtype == torch.float32 and out.dtype == torch.float32 and out.numel() == d
+    _check(lib().cvlc_decode_aggregate_unframed(_ptr(stream_ptrs), _ptr(stream_bytes), _ptr(weights), int(n_clients),
+                                                float(weight_total), int(d), _ptr(out), 1 if accumulate else 0, _ptr(ws),
+                                                ws.numel() * ws.element_size(), _stream_handle(stream)),
+           "cvlc_decode_aggregate_unframed")
+
+
 class CvlcLiteralPlan(C.Structure):
     _fields_ = [("status", C.c_int32), ("R", C.c_uint32), ("n_k", C.c_uint32), ("sweeps", C.c_uint32),
                 ("k_star", C.c_uint64), ("gamma_star", C.c_double), ("alpha_q", C.c_double), ("beta", C.c_double),
@@ -459,7 +501,7 @@ def cvlc_profile_reset() -> None:
 
 KERNEL_NAMES = ["k_zero_words", "k_hist", "k_plan_fit", "k_plan_tune", "k_plan_finish", "k_encode_init", "k_select",
                 "k_select_lookback", "k_sort_hist", "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero",
-                "k_prefetch_l2", "k_decode", "k_noalloc_publish_status", "k_selftest", "k_hist_check", "k_apply", "k_plan_literal", "k_ec_accumulate"]
+                "k_prefetch_l2", "k_decode", "k_noalloc_publish_status", "k_selftest", "k_hist_check", "k_apply", "k_plan_literal", "k_ec_accumulate", "k_pack_unframed", "k_decode_unframed"]
 
 
 def cvlc_profile_read(kernel_name: str = "*"):

@@ -13,8 +13,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OUT = os.path.join(HERE, "libcvlc.so")
-SOURCES = ["cvlc_api.cu", "cvlc_plan.cu", "cvlc_encode.cu", "cvlc_decode.cu", "cvlc_profile.cu"]
-HEADERS = [os.path.join(CSRC, "cvlc_common.cuh"), os.path.join(INCLUDE, "cvlc.h")]
+SOURCES = ["cvlc_api.cu", "cvlc_plan.cu", "cvlc_encode.cu", "cvlc_decode.cu", "cvlc_unframed.cu", "cvlc_profile.cu"]
+HEADERS = [os.path.join(CSRC, h) for h in ("cvlc_common.cuh", "cvlc_lookback.cuh", "cvlc_quant.cuh")] + [os.path.join(INCLUDE, "cvlc.h")]
 
 
 def _nvcc() -> str:

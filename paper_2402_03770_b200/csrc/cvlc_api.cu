@@ -350,6 +350,98 @@ int cvlc_encode_batch_ec(float* const* memory_dev, const cvlc_params* params, ui
                       stream_capacity, max_candidates, ws_dev, ws_bytes, cuda_stream, 1);
 }
 
+// ---- unframed stream (version 2) ------------------------------------------------------
+
+static bool unframed_fits(const Derived& D, const cvlc_params* p, size_t* capacity_out) {
+  const uint32_t y_lo = (p->quantizer == CVLC_QUANT_QSGD) ? 2u : 1u;
+  if (p->max_code_bits < y_lo || D.cap[y_lo] > kUfMaxRecords) return false;
+  uint64_t worst = 0;
+  for (uint32_t y = 1; y <= p->max_code_bits; ++y) {
+    const uint64_t bits = 64 + (uint64_t)D.cap[y] * (1 + uf_rice_param(p->d, D.cap[y]) + y) + 2 * (uint64_t)D.cap[y];
+    if (bits > worst) worst = bits;
+  }
+  if (capacity_out) *capacity_out = (uf_head_bytes(D.R) + (size_t)((worst * D.R + 63) / 64) * 8 + 15) & ~(size_t)15;
+  return true;
+}
+
+size_t cvlc_unframed_stream_capacity(const cvlc_params* p) {
+  Derived D;
+  size_t cap = 0;
+  if (derive(p, &D) != CVLC_OK || !unframed_fits(D, p, &cap)) return 0;
+  return cap;
+}
+
+size_t cvlc_unframed_workspace_bytes(const cvlc_params* p, uint32_t n) {
+  Derived D;
+  if (derive(p, &D) != CVLC_OK || n == 0 || n > CVLC_MAX_BATCH) return 0;
+  return uf_ws_bytes(n, D.R);
+}
+
+int cvlc_encode_unframed_batch(const float* const* x_dev, const cvlc_params* params, uint32_t n, const cvlc_plan_t* plans_dev,
+                               const void* plan_ws_dev, uint8_t* const* streams_dev, size_t stream_capacity,
+                               uint64_t* stream_bytes_dev, uint64_t max_candidates, void* enc_ws_dev, size_t enc_ws_bytes,
+                               void* uf_ws_dev, size_t uf_ws_bytes_given, void* cuda_stream) {
+  if (!x_dev || !params || !streams_dev || n == 0 || n > CVLC_MAX_BATCH) return CVLC_ERR_INVALID_ARG;
+  Shape S;
+  ClientDesc desc[CVLC_MAX_BATCH];
+  size_t need_capacity = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    Derived D;
+    const int rc = derive(&params[i], &D);
+    if (rc != CVLC_OK) return rc;
+    if (i && !same_shape(params[0], params[i])) return CVLC_ERR_INVALID_ARG;
+    if (!aligned(x_dev[i], 16) || !aligned(streams_dev[i], 16)) return CVLC_ERR_INVALID_ARG;
+    if (i == 0) {
+      if (!unframed_fits(D, &params[0], &need_capacity)) return CVLC_ERR_INVALID_ARG;  // blocks of more than 2048 records
+      memset(&S, 0, sizeof S);
+      S.d = params[0].d;
+      S.s = D.s;
+      S.R = D.R;
+      S.packet_bits = params[0].packet_bits;
+      S.header_bits = params[0].header_bits;
+      S.quantizer = params[0].quantizer;
+      S.max_code_bits = params[0].max_code_bits;
+      for (uint32_t y = 0; y <= CVLC_MAX_CODE_BITS; ++y) S.cap[y] = D.cap[y];
+    }
+    desc[i].x = x_dev[i];
+    desc[i].plan = const_cast<cvlc_plan_t*>(plans_dev) + i;
+    desc[i].stream = streams_dev[i];
+    desc[i].seed = params[i].seed;
+    desc[i].scale_B = params[i].scale_B;
+    desc[i].client_id = params[i].client_id;
+    desc[i].round = params[i].round;
+  }
+  if (!aligned(plans_dev, 8) || !aligned(enc_ws_dev, 256) || !aligned(uf_ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (plan_ws_dev && !aligned(plan_ws_dev, 256)) return CVLC_ERR_INVALID_ARG;
+  if (stream_bytes_dev && !aligned(stream_bytes_dev, 8)) return CVLC_ERR_INVALID_ARG;
+  if (stream_capacity < need_capacity) return CVLC_ERR_OUTPUT_TOO_SMALL;
+  const uint64_t cap = (max_candidates == 0 || max_candidates > S.d) ? S.d : max_candidates;
+  if (enc_ws_bytes < enc_layout(S.d, n, cap).total || uf_ws_bytes_given < uf_ws_bytes(n, S.R)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  if (S.R > 0x7FFFFFFFu || n > 65535) return CVLC_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (launch_encode(desc, n, S, cap, plan_ws_dev, enc_ws_dev, st, nullptr, kPackNone) != cudaSuccess) return CVLC_ERR_CUDA;
+  return launch_pack_unframed(desc, n, S, cap, stream_capacity, enc_ws_dev, uf_ws_dev,
+                              reinterpret_cast<unsigned long long*>(stream_bytes_dev), st) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
+}
+
+int cvlc_decode_aggregate_unframed(const uint8_t* const* streams_dev, const uint64_t* stream_bytes_dev, const float* weights_dev,
+                                   uint32_t n_clients, double weight_total, uint64_t d, float* out_dev, int accumulate,
+                                   void* ws_dev, size_t ws_bytes, void* cuda_stream) {
+  if (n_clients == 0 || n_clients > CVLC_MAX_CLIENTS_PER_CALL) return CVLC_ERR_INVALID_ARG;
+  if (d < 2 || d > (1ull << 31)) return CVLC_ERR_INVALID_ARG;
+  if (!(weight_total >= 0.0) || !(weight_total < 1e300)) return CVLC_ERR_INVALID_ARG;
+  if (!aligned(streams_dev, 8) || !aligned(stream_bytes_dev, 8) || !aligned(weights_dev, 4) || !aligned(out_dev, 16) ||
+      !aligned(ws_dev, 256))
+    return CVLC_ERR_INVALID_ARG;
+  if (ws_bytes < dec_ws_bytes(n_clients)) return CVLC_ERR_WORKSPACE_TOO_SMALL;
+  return launch_decode_unframed(streams_dev, stream_bytes_dev, weights_dev, n_clients, weight_total, d, position_bits(d), out_dev,
+                                accumulate ? 1 : 0, ws_dev, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? CVLC_OK
+             : CVLC_ERR_CUDA;
+}
+
 int cvlc_ec_accumulate_batch(float* const* memory_dev, const float* const* update_dev, uint32_t n, uint64_t d,
                              void* cuda_stream) {
   if (!memory_dev || !update_dev || n == 0 || n > CVLC_MAX_BATCH || d < 2 || d > (1ull << 31)) return CVLC_ERR_INVALID_ARG;
@@ -414,7 +506,7 @@ int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, ui
   if (launch_plan_front(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
   if (!two) {
     if (launch_plan_back(desc, n, S, plan_ws_dev, main_st) != cudaSuccess) return CVLC_ERR_CUDA;
-    return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, nullptr, 0) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+    return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, nullptr, kPackFramed) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
   }
   // the length tuning reads the histograms' fit only; selection and ranking do not need its result
   cudaEvent_t fork, join;
@@ -422,7 +514,7 @@ int cvlc_compress_batch(const float* const* x_dev, const cvlc_params* params, ui
   if (cudaEventRecord(fork, main_st) != cudaSuccess || cudaStreamWaitEvent(side_st, fork, 0) != cudaSuccess) return CVLC_ERR_CUDA;
   if (launch_plan_back(desc, n, S, plan_ws_dev, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
   if (cudaEventRecord(join, side_st) != cudaSuccess) return CVLC_ERR_CUDA;
-  return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, join, 0) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
+  return launch_encode(desc, n, Senc, cap, plan_ws_dev, enc_ws_dev, main_st, join, kPackFramed) == cudaSuccess ? CVLC_OK : CVLC_ERR_CUDA;
 }
 
 int cvlc_encode(const float* x_dev, const cvlc_params* p, const cvlc_plan_t* plan_dev, const void* plan_ws_dev,

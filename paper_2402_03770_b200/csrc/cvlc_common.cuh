@@ -207,7 +207,7 @@ CVLC_HD constexpr size_t dec_ws_bytes(uint32_t n) { return align256(dec_off_meta
 enum KernelId {
   kKZeroWords = 0, kKHist, kKPlanFit, kKPlanTune, kKPlanFinish, kKEncodeInit, kKSelect, kKSelectLookback, kKSortHist, kKSortScan,
   kKSortPass, kKPack, kKDecodePrepare, kKFillZero, kKPrefetchL2, kKDecode, kKNoallocStatus, kKSelftest, kKHistCheck, kKApply,
-  kKPlanLiteral, kKEcAccumulate, kNumKernelIds
+  kKPlanLiteral, kKEcAccumulate, kKPackUnframed, kKDecodeUnframed, kNumKernelIds
 };
 
 // Called around every kernel launch.  Counts launches; when a kernel has been selected with
@@ -248,11 +248,35 @@ cudaError_t launch_plan_literal(const cvlc_params& p, double alpha_q, uint32_t s
 cudaError_t launch_apply(float* model, const float* agg, uint64_t d, const void* dec_ws, cudaStream_t st);
 // wait_before_pack: an event the stream waits for right before the packing kernel (the length tuning on
 // another stream), or nullptr
-// write_residual: the packing kernel also turns the encoder's input into the error-compensation memory (the input
-// buffers are written: every sent coordinate loses what the parameter server rebuilds for it)
+// write_residual: kPackFramed = packets only; kPackResidual = the packing kernel also turns the encoder's input into
+// the error-compensation memory (the input buffers are written: every sent coordinate loses what the parameter
+// server rebuilds for it); kPackNone = selection and ranking only (the unframed writer follows)
+constexpr int kPackFramed = 0, kPackResidual = 1, kPackNone = 2;
 cudaError_t launch_encode(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
                           const void* plan_ws, void* ws, cudaStream_t st, cudaEvent_t wait_before_pack, int write_residual);
 cudaError_t launch_ec_accumulate(float* const* memory, const float* const* update, uint32_t n, uint64_t d, cudaStream_t st);
+// unframed stream (version 2)
+constexpr uint32_t kUfMaxRecords = 2048;  // records of a block (it is sorted and assembled in one warp's shared memory)
+constexpr size_t kUfTables = 64, kUfTotalBits = 64 + 264, kUfDirectory = 64 + 264 + 8;
+CVLC_HD constexpr size_t uf_head_bytes(uint32_t R) { return kUfDirectory + (size_t)R * 8; }
+CVLC_HD constexpr size_t uf_off_ticket() { return 256; }
+CVLC_HD constexpr size_t uf_off_state(uint32_t n) { return align256(uf_off_ticket() + (size_t)n * 4); }
+CVLC_HD constexpr size_t uf_ws_bytes(uint32_t n, uint32_t R) { return align256(uf_off_state(n) + (size_t)n * R * 8); }
+CVLC_HD inline uint32_t uf_rice_param(uint64_t d, uint32_t P) {  // floor(log2(d / P)), 0 when d < 2 P
+  uint64_t g = d / (uint64_t)P;
+  uint32_t m = 0;
+  while (g >= 2) {
+    g >>= 1;
+    ++m;
+  }
+  return m;
+}
+cudaError_t launch_pack_unframed(const ClientDesc* clients, uint32_t n, const Shape& shape, uint64_t capacity,
+                                 size_t stream_capacity, void* enc_ws, void* uf_ws, unsigned long long* sizes_out, cudaStream_t st);
+cudaError_t launch_decode_unframed(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
+                                   uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,
+                                   void* ws, cudaStream_t st);
+cudaError_t launch_fill_zero(float* out, uint64_t d, cudaStream_t st);
 cudaError_t launch_selftest_wait(unsigned long long* word, int32_t* status, uint32_t max_polls, cudaStream_t st);
 cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_bytes, const float* weights,
                           uint32_t n, double weight_total, uint64_t d, uint32_t s, float* out, int accumulate,

@@ -269,6 +269,14 @@ cudaError_t launch_decode(const uint8_t* const* streams, const uint64_t* stream_
   return cudaGetLastError();
 }
 
+cudaError_t launch_fill_zero(float* out, uint64_t d, cudaStream_t st) {
+  const uint64_t want = (d / 4 + 255) / 256;
+  const int grid = (int)(want < (uint64_t)(8 * kNumSM) ? (want ? want : 1) : 8 * kNumSM);
+  LaunchScope ls(kKFillZero, st);
+  k_fill_zero<<<grid, 256, 0, st>>>(out, d);
+  return cudaGetLastError();
+}
+
 // K8  model <- model - aggregate (Section III, step 3); nothing is touched after a decode error
 __global__ void __launch_bounds__(256)
 k_apply(float* __restrict__ model, const float* __restrict__ agg, uint64_t d, const unsigned char* dec_ws) {

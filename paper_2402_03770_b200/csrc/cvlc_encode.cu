@@ -4,40 +4,12 @@
 // stochastic quantization with Philox4x32-10 (PQ or QSGD) and bit packing of
 // (position ID, centroid ID) pairs into fixed-size packets (Fig. 2).
 #include "cvlc_common.cuh"
+#include "cvlc_lookback.cuh"
+#include "cvlc_quant.cuh"
 
 namespace cvlc {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr unsigned long long kFlagAgg = 1ull << 62;     // tile aggregate published
-constexpr unsigned long long kFlagPrefix = 2ull << 62;  // inclusive prefix published
-constexpr unsigned long long kFlagMask = 3ull << 62;
-constexpr unsigned long long kValMask = ~kFlagMask;
-constexpr int kMaxPolls = 1 << 20;  // bounded wait of the look-back; then DEVICE_TIMEOUT
-
-__device__ __forceinline__ unsigned long long ld_relaxed(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-
-// Waits (bounded) until a look-back state word carries a flag.  Returns 0 after a timeout.
-__device__ __forceinline__ unsigned long long wait_state(const unsigned long long* p, int32_t* status, int max_polls = kMaxPolls) {
-  unsigned long long v = ld_relaxed(p);
-  int polls = 0;
-  while ((v & kFlagMask) == 0) {
-    if (++polls > max_polls) {
-      set_status(status, CVLC_ERR_DEVICE_TIMEOUT);
-      return 0;
-    }
-    if (polls > 64) __nanosleep(64);
-    v = ld_relaxed(p);
-  }
-  return v;
-}
-
 // Whether an earlier kernel of the call has reported an error.  Other blocks may set the word while this kernel
 // runs, so one thread reads it and the whole block takes the same branch.
 __device__ __forceinline__ bool block_sees_error(const int32_t* status) {
@@ -1012,20 +984,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
       __syncwarp();
       // the norm is defined with the squares added in rank order in double: one lane walks the chain
       float norm = 0.0f;
-      if (lane == 0) {
-        double sum = 0.0;
-        uint32_t j = 0;
-        for (; j + 8 <= P; j += 8) {
-          double v[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) v[u] = sqv[j + u];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) sum = __dadd_rn(sum, v[u]);
-        }
-        for (; j < P; ++j) sum = __dadd_rn(sum, sqv[j]);
-        const double rt = __dsqrt_rn(sum);
-        norm = (rt > 3.4028234663852886e38) ? 3.4028234663852886e38f : __double2float_rn(rt);
-      }
+      if (lane == 0) norm = qsgd_norm_of_squares(sqv, P);
       norm = __shfl_sync(kFull, norm, 0);
       lo = norm;
       hi = 0.0f;
@@ -1042,22 +1001,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         if (norm > 0.0f) {
           const double a = (double)__uint_as_float(key);
           const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
-          // t = (a / norm) * s_q decides floor(t) and [u < frac(t)]; a * (s_q / norm) is within a few ulp of it
-          // and decides the same unless its fraction sits that close to 0, 1 or u
-          const double tf = __dmul_rn(a, scale);
-          const double jf = floor(tf);
-          const double ff = __dsub_rn(tf, jf);
-          const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
-          if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < sqd) {
-            level = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
-          } else {
-            const double t = __dmul_rn(__ddiv_rn(a, dn), sqd);
-            double j0 = floor(t);
-            if (j0 > sqd) j0 = sqd;
-            const double frac = __dsub_rn(t, j0);
-            level = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
-            if (level > sq) level = sq;
-          }
+          level = qsgd_quantize_level(a, dn, sqd, sq, scale, u);
         }
         const uint32_t code = (sign << (y - 1)) | level;
         put(j, (unsigned long long)pid | ((unsigned long long)code << s));
@@ -1102,22 +1046,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         if (hi != lo) {
           const double num = __dsub_rn((double)__uint_as_float(b), dlo);
           const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
-          // t = (num / den) * L decides floor(t) and [u < frac(t)].  num * (L / den) is within a few ulp of it;
-          // unless its fraction sits that close to 0, 1 or u, both decisions are the same and the division
-          // is not needed.
-          const double tf = __dmul_rn(num, scale);
-          const double jf = floor(tf);
-          const double ff = __dsub_rn(tf, jf);
-          const double eps = __dmul_rn(tf, 0x1p-48) + 0x1p-1000;
-          if (ff > eps && ff < 1.0 - eps && fabs(ff - u) > eps && jf < Lc) {
-            code = __double2uint_rz(jf) + ((u < ff) ? 1u : 0u);
-          } else {
-            const double t = __dmul_rn(__ddiv_rn(num, den), Lc);
-            double j0 = floor(t);
-            if (j0 > Lc) j0 = Lc;
-            const double frac = __dsub_rn(t, j0);
-            code = __double2uint_rz(j0) + ((u < frac) ? 1u : 0u);
-          }
+          code = pq_quantize(num, den, Lc, scale, u);
         }
         put(j, (unsigned long long)pid | ((unsigned long long)code << s));
         if (residual) {
@@ -1237,6 +1166,7 @@ static cudaError_t launch_encode_t(const ClientDesc* clients, uint32_t n, const 
     const cudaError_t ew = cudaStreamWaitEvent(st, wait_before_pack, 0);
     if (ew != cudaSuccess) return ew;
   }
+  if (write_residual == kPackNone) return cudaGetLastError();  // the caller writes the ranked records in a format of its own
   {
     LaunchScope ls(kKPack, st);
     if (qsgd)

@@ -10,7 +10,7 @@ namespace {
 const char* const kKernelNames[kNumKernelIds] = {
     "k_zero_words", "k_hist", "k_plan_fit", "k_plan_tune", "k_plan_finish", "k_encode_init", "k_select", "k_select_lookback", "k_sort_hist",
     "k_sort_scan", "k_sort_pass", "k_pack", "k_decode_prepare", "k_fill_zero", "k_prefetch_l2", "k_decode", "k_noalloc_publish_status",
-    "k_selftest", "k_hist_check", "k_apply", "k_plan_literal", "k_ec_accumulate"};
+    "k_selftest", "k_hist_check", "k_apply", "k_plan_literal", "k_ec_accumulate", "k_pack_unframed", "k_decode_unframed"};
 
 unsigned long long g_launches[kNumKernelIds] = {};
 int g_prof_kernel = -1;          // kernel id being timed; kNumKernelIds = every kernel; -1 = off

@@ -99,7 +99,7 @@ def test_malformed_unframed_streams_are_rejected():
     for bad in (u[:-8], np.concatenate([u, np.zeros(8, np.uint8)])):
         with pytest.raises(O.OracleError):
             O.decode_aggregate_unframed([bad], w, 20000)
-    for off, val in ((0, 0), (4, 1), (64 + 4 * 8, 99), (64 + 264 + 8 + 8, 0xFF)):     # magic, version, n_y, directory
+    for off, val in ((0, 0), (4, 1), (64 + 4 * 8, 99), (64 + 264 + 8 + 8, 0xFF), (64 + 264 + 8 + 8, 1)):     # magic, version, n_y, directory
         b = u.copy()
         b[off] = val
         with pytest.raises(O.OracleError):

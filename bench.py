@@ -39,14 +39,18 @@ FALLBACK_HBM_GBS = 6650.0
 # proportion to the clients); scaled to the clients of a launch, None for any other configuration, for fewer than
 # 32 clients per launch, and for a kernel that has changed since its capture.
 NCU_TRAFFIC_BYTES_PER_CLIENT = {
+    "k_hist": (1434.11e6 + 48.13e6) / 32,          # the update once, plus row maxima and per-segment histograms
+    "k_select": (512.26e6 + 166.99e6) / 32,        # the rows that hold candidates (36 % of the update), plus the candidates
+    "k_sort_pass": (208.92e6 + 174.73e6 + 208.06e6 + 174.69e6 + 206.50e6 + 174.18e6 + 0.08e6) / 32 / 4,  # mean of a step's four launches
+    "k_pack": (177.98e6 + 54.09e6) / 32,
 }
 NOMINAL_HBM_GBS = 8000.0
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18")
     ap.add_argument("--bits-per-coord", type=float, default=2.0)
@@ -308,6 +312,11 @@ def run_ours(args):
         total_ms = R.max_over_ranks(total_ms, dev)
         return total_ms, per
 
+    # the clock sampler runs from before the warm-up to the end of the timed region, with no idle gap in between
+    # (an idle GPU drops its clocks, and the first steps after a pause are slow)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step(False)
     barrier()
@@ -315,13 +324,13 @@ def run_ours(args):
         assert enc.status() == B.CVLC_OK, "encode reported a device-side error"
     assert agg.status() == B.CVLC_OK, "decode-aggregate reported a device-side error"
 
-    launches_before = B.cvlc_launch_count()
     per_step_launch_cap = 16 * len(groups) + 8 + 3 * (d // (24 << 20) + 1)  # decode: one fill + one launch per window
     B.cvlc_profile_select("*", per_step_launch_cap * args.steps)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
+    for _ in range(2):        # the GPU idled while the profiling events were created: two more untimed steps
+        step(False)
+    barrier()
+    B.cvlc_profile_reset()    # the per-kernel times cover the timed steps only
+    launches_before = B.cvlc_launch_count()
     total_ms, per = timed(args.steps, False)
     clocks = sampler.stop() if rank == 0 else None
     gpu_launches = B.cvlc_launch_count() - launches_before
@@ -342,7 +351,6 @@ def run_ours(args):
         sampler2 = ClockSampler(local_rank)
         if rank == 0:
             sampler2.start()
-            time.sleep(0.2)
         sus_ms, _ = timed(n_sus, False)
         clocks2 = sampler2.stop() if rank == 0 else None
         sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,

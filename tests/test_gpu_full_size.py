@@ -11,7 +11,9 @@ from gpu_util import assert_aggregate_close, assert_plan_equal, gpu_params, orac
 pytestmark = pytest.mark.gpu
 
 
-def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, quantizer=0):
+def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, quantizer=0, one_call=True):
+    """one_call: cvlc_compress_batch with the length tuning on a side stream (what the benchmark times); otherwise
+    cvlc_plan_batch followed by cvlc_encode_batch"""
     w = W.WORKLOADS[workload]
     dev = torch.device("cuda:0")
     params, xs = [], []
@@ -22,7 +24,7 @@ def gpu_batch_encode(workload, clients, d, bpc, max_candidates, torch, B, quanti
                                              quantizer=quantizer)))
         xs.append(torch.from_numpy(x).to(dev))
     enc = B.BatchEncoder(params, dev, max_candidates=max_candidates)
-    outs = enc.run(xs)
+    outs = enc.compress(xs, side_stream=torch.cuda.Stream(device=dev)) if one_call else enc.run(xs)
     assert enc.status() == B.CVLC_OK
     del xs
     return enc, outs
@@ -72,8 +74,9 @@ def test_small_cnn_all_20_clients(env):
     w = W.WORKLOADS["small_cnn"]
     clients = list(range(w.n_clients))
     ref = oracle_encode_clients("small_cnn", clients, None, 2.0)
-    enc, outs = gpu_batch_encode("small_cnn", clients, None, 2.0, 0, torch, B)
-    check_against_oracle(enc, outs, ref)
+    for one_call in (True, False):
+        enc, outs = gpu_batch_encode("small_cnn", clients, None, 2.0, 0, torch, B, one_call=one_call)
+        check_against_oracle(enc, outs, ref)
     decode_both(outs, [r[2] for r in ref], W.client_weights(w), w.d, torch, B)
 
 
@@ -89,8 +92,9 @@ def test_resnet18_budget_sweep_two_clients(env, bpc):
 
 
 def test_resnet18_all_100_clients_as_benchmarked(env):
-    """the benchmark's step: one batched plan + encode of 100 clients at 2 bits per coordinate with the
-    benchmark's reduced candidate workspace, then one decode-aggregate with sample-count weights"""
+    """the benchmark's step: plan + encode of 100 clients at 2 bits per coordinate in one call, the length tuning on
+    a side stream, with the benchmark's reduced candidate workspace, then one decode-aggregate with sample-count
+    weights"""
     torch, B = env
     w = W.WORKLOADS["resnet18"]
     clients = list(range(w.n_clients))

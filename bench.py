@@ -89,8 +89,9 @@ class ClockSampler:
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_ms: int = 100):
         self.index = index
+        self.period_ms = period_ms
         self.proc = None
         self.lines = []
 
@@ -98,7 +99,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", str(self.period_ms)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -107,6 +108,12 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
+
+    def wait_first_sample(self, timeout_s: float = 3.0):
+        """nvidia-smi takes a moment to start: wait until it has answered once"""
+        t0 = time.time()
+        while self.proc is not None and not self.lines and time.time() - t0 < timeout_s:
+            time.sleep(0.01)
 
     def stop(self):
         if self.proc is None:
@@ -314,9 +321,10 @@ def run_ours(args):
 
     # the clock sampler runs from before the warm-up to the end of the timed region, with no idle gap in between
     # (an idle GPU drops its clocks, and the first steps after a pause are slow)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, period_ms=25)   # the timed region is short: sample often
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample()
     for _ in range(max(args.warmup, 3)):
         step(False)
     barrier()

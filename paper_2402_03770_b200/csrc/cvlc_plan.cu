@@ -303,7 +303,7 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
   double* ptY = ptX + 4096;
   __shared__ PlanShared S;
   __shared__ PlanTab T;
-  __shared__ uint32_t s_thresh_bin;
+  __shared__ uint32_t s_thresh_bin, s_top_bin;
   int32_t* ws_status = reinterpret_cast<int32_t*>(ws);
 
   // blockIdx.x = client
@@ -431,7 +431,10 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
       plan->n_candidates = N;
       s_thresh_bin = (uint32_t)j;
     }
-    if (N > 0 && Nn == 0) plan->top_bin = (uint32_t)j;
+    if (N > 0 && Nn == 0) {
+      plan->top_bin = (uint32_t)j;
+      s_top_bin = (uint32_t)j;
+    }
   }
   if (tid == 0) {
     const double aq = S.alpha_q;
@@ -471,11 +474,11 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
     const uint32_t* seg_hist = reinterpret_cast<const uint32_t*>(ws + plan_off_seg_hist(batch.n, S, row_tiles));
     const uint64_t first = (uint64_t)c * part.units, last = first + part.units - 1;
     const uint32_t b0 = (uint32_t)(first / part.chunk), b1 = (uint32_t)(last / part.chunk);
-    const uint32_t jt = s_thresh_bin;
+    const uint32_t jt = s_thresh_bin, jtop = s_top_bin;  // nothing above the client's highest non-empty bin
     for (uint32_t b = b0 + warp; b <= b1; b += kPlanThreads / 32) {
       const uint32_t* hsrc = seg_hist + ((size_t)b + c) * CVLC_HIST_BINS;
       uint32_t sum = 0;
-      for (uint32_t j = jt + lane; j < CVLC_HIST_BINS; j += 32) sum += hsrc[j];
+      for (uint32_t j = jt + lane; j <= jtop; j += 32) sum += hsrc[j];
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
       if (lane == 0) seg_count[b + c] = sum;

@@ -153,3 +153,47 @@ def test_decode_windows_with_a_ragged_last_window(env):
     enc, outs = gpu_batch_encode("stress", clients, d, 0.25, 0, torch, B)
     check_against_oracle(enc, outs, ref)
     decode_both(outs, [r[2] for r in ref], np.array([1.0, 3.0], dtype=np.float32), d, torch, B, batches=2)
+
+
+def test_resnet18_unframed_and_error_compensation_two_clients(env):
+    """the unframed writer and the error-compensation residual at the benchmark's size and budget"""
+    torch, B = env
+    dev = torch.device("cuda:0")
+    w = W.WORKLOADS["resnet18"]
+    clients = [3, 77]
+    xs = [W.client_update(w, c) for c in clients]
+    pds = [params_dict(w.d, 2 * w.d, seed=W.philox_ids(w, c)[0], client_id=W.philox_ids(w, c)[1]) for c in clients]
+    params = [gpu_params(pd) for pd in pds]
+    from gpu_util import oracle_params
+    plans = [O.plan(x, oracle_params(pd)) for x, pd in zip(xs, pds)]
+    # unframed streams, byte for byte, and the aggregate they decode to
+    enc = B.BatchEncoder(params, dev)
+    dxs = [torch.from_numpy(x).to(dev) for x in xs]
+    enc.plan(dxs)
+    cap = B.cvlc_unframed_stream_capacity(params[0])
+    outs = [torch.zeros(cap, dtype=torch.uint8, device=dev) for _ in clients]
+    sizes = torch.zeros(len(clients), dtype=torch.int64, device=dev)
+    uf_ws = B.alloc_bytes(B.cvlc_unframed_workspace_bytes(params[0], len(clients)), dev)
+    B.cvlc_encode_unframed_batch(dxs, params, enc.plans, outs, sizes, enc.enc_ws, uf_ws, plan_ws=enc.plan_ws)
+    assert enc.status() == B.CVLC_OK
+    refs = [O.encode_unframed(x, oracle_params(pd), pl) for x, pd, pl in zip(xs, pds, plans)]
+    for i, ref in enumerate(refs):
+        n = int(sizes[i].item())
+        assert n == ref.size and (outs[i][:n].cpu().numpy() == ref).all(), i
+    ptrs = torch.tensor([o.data_ptr() for o in outs], dtype=torch.int64, device=dev)
+    wts = torch.tensor([1.0, 3.0], dtype=torch.float32, device=dev)
+    dws = B.alloc_bytes(B.cvlc_decode_workspace_bytes(2), dev)
+    agg = torch.empty(w.d, dtype=torch.float32, device=dev)
+    B.cvlc_decode_aggregate_unframed(ptrs, sizes, wts, 2, 0.0, w.d, agg, False, dws)
+    assert B.cvlc_read_status(dws) == B.CVLC_OK
+    assert_aggregate_close(agg.cpu().numpy(), O.decode_aggregate_unframed(refs, np.array([1.0, 3.0], np.float32), w.d))
+    # error compensation: the framed streams are unchanged, the inputs become the memories
+    mems = [torch.from_numpy(x).to(dev) for x in xs]
+    enc.plan(mems)
+    B.cvlc_encode_batch_ec(mems, params, enc.plans, enc.outs, enc.enc_ws, plan_ws=enc.plan_ws)
+    assert enc.status() == B.CVLC_OK
+    for i, (x, pd, pl) in enumerate(zip(xs, pds, plans)):
+        st = O.encode(x, oracle_params(pd), pl)
+        assert (enc.outs[i].cpu().numpy() == st).all(), i
+        want = O.ec_residual(x, st)
+        assert (mems[i].cpu().numpy().view(np.uint32) == want.view(np.uint32)).all(), i

@@ -41,6 +41,40 @@ def draw_case(rng):
     return x.astype(np.float32), pd, kind
 
 
+def check_unframed(torch, B, x, pd, framed):
+    """where the shape allows it, the unframed stream equals the oracle's byte for byte and decodes to the aggregate of
+    the framed one; where it does not (blocks of more than 2048 records), the capacity query says so"""
+    from gpu_util import gpu_params
+    dev = torch.device("cuda:0")
+    p = gpu_params(pd)
+    cap = B.cvlc_unframed_stream_capacity(p)
+    po = oracle_params(pd)
+    s_bits = max(1, int(np.ceil(np.log2(pd["d"]))))
+    y_lo = 2 if pd["quantizer"] else 1
+    if (pd["packet_bits"] - pd["header_bits"]) // (s_bits + y_lo) > 2048 or pd["max_code_bits"] < y_lo:
+        assert cap == 0
+        return
+    assert cap >= O.unframed_capacity(po)
+    ref = O.encode_unframed(x, po, O.plan(x, po))
+    enc = B.BatchEncoder([p], dev)
+    xd = [torch.from_numpy(x).to(dev)]
+    enc.plan(xd)
+    out = torch.full((cap,), 0x5A, dtype=torch.uint8, device=dev)
+    size = torch.zeros(1, dtype=torch.int64, device=dev)
+    uf_ws = B.alloc_bytes(B.cvlc_unframed_workspace_bytes(p, 1), dev)
+    B.cvlc_encode_unframed_batch(xd, [p], enc.plans, [out], size, enc.enc_ws, uf_ws, plan_ws=enc.plan_ws)
+    assert enc.status() == 0
+    n = int(size.item())
+    assert n == ref.size and (out[:n].cpu().numpy() == ref).all(), pd
+    ptr = torch.tensor([out.data_ptr()], dtype=torch.int64, device=dev)
+    w = torch.ones(1, dtype=torch.float32, device=dev)
+    ws = B.alloc_bytes(B.cvlc_decode_workspace_bytes(1), dev)
+    agg = torch.empty(pd["d"], dtype=torch.float32, device=dev)
+    B.cvlc_decode_aggregate_unframed(ptr, size, w, 1, 0.0, pd["d"], agg, False, ws)
+    assert B.cvlc_read_status(ws) == 0
+    assert_aggregate_close(agg.cpu().numpy(), O.decode_aggregate([framed], np.ones(1, np.float32), pd["d"]))
+
+
 @pytest.mark.parametrize("seed", range(20))
 def test_random_shapes(seed):
     import torch
@@ -60,11 +94,12 @@ def test_random_shapes(seed):
             assert e.value.code == oe.code, (pd, kind)
             refused += 1
             continue
-        for use_plan_ws in (True, False):
-            status, gp, gst = gpu_plan_encode(x, pd, use_plan_ws=use_plan_ws)
+        for use_plan_ws, compress in ((True, 0), (False, 0), (True, 2 if done % 2 else 1)):
+            status, gp, gst = gpu_plan_encode(x, pd, use_plan_ws=use_plan_ws, compress=compress)
             assert status == 0, (status, pd, kind)
             assert_plan_equal(gp, of)
-            assert gst.size == ost.size and (gst == ost).all(), (pd, kind, use_plan_ws)
+            assert gst.size == ost.size and (gst == ost).all(), (pd, kind, use_plan_ws, compress)
+        check_unframed(torch, B, x, pd, ost)
         weights = np.array([1.0, 0.5, 3.0], dtype=np.float32)
         ref = O.decode_aggregate([ost, ost, ost], weights, pd["d"])
         status, out = gpu_decode_aggregate([ost, ost, ost], weights, pd["d"])

@@ -50,3 +50,20 @@ def test_binding_raises_when_library_is_missing(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError):
         B.lib()
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/cvlc.h is a C header: it compiles as C11 with no CUDA or C++ in sight, and the two structs that cross
+    the boundary have the sizes the binding assumes"""
+    import subprocess
+    src = tmp_path / "t.c"
+    src.write_text('#include "cvlc.h"\n'
+                   '_Static_assert(sizeof(cvlc_plan_t) == 512, "plan");\n'
+                   '_Static_assert(sizeof(cvlc_literal_plan_t) == 64, "literal plan");\n'
+                   '_Static_assert(sizeof(cvlc_params) == 56, "params");\n'
+                   'int main(void) { return CVLC_OK; }\n')
+    r = subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-fsyntax-only", "-I", os.path.join(ROOT, "include"), str(src)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    from paper_2402_03770_b200 import binding as B
+    assert ctypes.sizeof(B.CvlcParams) == 56 and ctypes.sizeof(B.CvlcLiteralPlan) == 64

@@ -137,6 +137,37 @@ k_prefetch_l2(const float* __restrict__ p, uint64_t n) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(base + l * 128));
 }
 
+// The records of one staged packet whose width s + y is at most 32 bits: record j starts at bit H + j (s + y), so it
+// lies in the words wi, wi + 1 of the packet and one funnel shift cuts it out.  WHOLE: the accumulator is one window.
+template <bool QSGD, bool WHOLE>
+__device__ __forceinline__ void decode_narrow(const uint32_t* __restrict__ sp, uint32_t P, uint32_t H, uint32_t wd, uint32_t s,
+                                              uint32_t y, uint64_t d, uint64_t win_lo, uint64_t win_hi, double dlo, double step,
+                                              float cf, float* __restrict__ out, int32_t* status, int lane) {
+  const uint32_t rmask = (wd == 32) ? 0xFFFFFFFFu : ((1u << wd) - 1u);
+  const uint32_t pmask = (1u << s) - 1u;  // s + y <= 32 and y >= 1: s <= 31
+  const uint32_t level_mask = QSGD ? ((1u << (y - 1)) - 1u) : 0u;
+  const uint32_t d32 = (d > 0xFFFFFFFFull) ? 0xFFFFFFFFu : (uint32_t)d;  // d <= 2^31
+  for (uint32_t j = lane; j < P; j += 32) {
+    const uint32_t bit = H + j * wd;
+    const uint32_t wi = bit >> 5;
+    const uint32_t rec = __funnelshift_r(sp[wi], sp[wi + 1], bit & 31u) & rmask;
+    const uint32_t pid = rec & pmask, code = rec >> s;
+    if (pid >= d32) {
+      set_status(status, CVLC_ERR_BAD_STREAM);
+      continue;
+    }
+    if (!WHOLE && (pid < win_lo || pid >= win_hi)) continue;
+    float v;
+    if (QSGD) {
+      const float mag = (float)__dmul_rn((double)(code & level_mask), step);
+      v = ((code >> (y - 1)) & 1u) ? -mag : mag;
+    } else {
+      v = (float)__dadd_rn(dlo, __dmul_rn((double)code, step));
+    }
+    atomicAdd(out + pid, cf * v);
+  }
+}
+
 // K6  decode + dequantize + weighted scatter-accumulate, one warp per packet.  Only the records whose
 // position lies in [win_lo, win_hi) are accumulated: an accumulator larger than the L2 is filled window by
 // window (one launch each), so that the reductions stay in the L2 instead of becoming DRAM read-modify-writes.
@@ -146,7 +177,7 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
   extern __shared__ uint32_t s_prefix[];  // [n + 1]
   // a packet of up to kDecStageWords words is first copied to the warp's own shared-memory buffer with
   // coalesced, independent loads; the records are then cut out of shared memory (larger packets: out of global)
-  __shared__ uint32_t s_pkt[kDecodeThreads / 32][kDecStageWords];
+  __shared__ uint32_t s_pkt[kDecodeThreads / 32][kDecStageWords + 1];  // one word of slack: the narrow path reads word wi + 1
   uint32_t* sp = s_pkt[threadIdx.x >> 5];
   int32_t* status = reinterpret_cast<int32_t*>(ws + kDecWsStatus);
   const float* coef = reinterpret_cast<const float*>(ws + kDecWsCoef);
@@ -212,6 +243,17 @@ k_decode(const uint8_t* const* __restrict__ streams, uint32_t n, uint64_t d, uin
                              : ((hi == lo) ? 0.0 : __ddiv_rn(__dsub_rn((double)hi, dlo), (double)((1ull << y) - 1ull)));
     const float cf = coef[c];
     const unsigned long long code_mask = (1ull << y) - 1ull;
+    if (staged && wd <= 32) {
+      // the usual case: a record fits one 32-bit funnel shift of two staged words
+      const bool whole = (win_lo == 0 && win_hi >= d);
+      if (qsgd)
+        whole ? decode_narrow<true, true>(sp, P, H, wd, s, y, d, win_lo, win_hi, dlo, step, cf, out, status, lane)
+              : decode_narrow<true, false>(sp, P, H, wd, s, y, d, win_lo, win_hi, dlo, step, cf, out, status, lane);
+      else
+        whole ? decode_narrow<false, true>(sp, P, H, wd, s, y, d, win_lo, win_hi, dlo, step, cf, out, status, lane)
+              : decode_narrow<false, false>(sp, P, H, wd, s, y, d, win_lo, win_hi, dlo, step, cf, out, status, lane);
+      continue;
+    }
     for (uint32_t j = lane; j < P; j += 32) {
       const uint32_t bit = H + j * wd;
       const uint32_t wi = bit >> 5, sh = bit & 31;

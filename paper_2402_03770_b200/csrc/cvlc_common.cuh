@@ -312,6 +312,32 @@ __device__ __forceinline__ uint32_t philox_coord(uint64_t seed, uint32_t client_
   return r.x;
 }
 
+// The same word with the ten round keys worked out once per client instead of once per coordinate.
+struct PhiloxRoundKeys {
+  uint32_t x[10], y[10];
+};
+__device__ __forceinline__ PhiloxRoundKeys philox_round_keys(uint64_t seed) {
+  PhiloxRoundKeys rk;
+  uint32_t kx = (uint32_t)seed, ky = (uint32_t)(seed >> 32);
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    rk.x[i] = kx;
+    rk.y[i] = ky;
+    kx += 0x9E3779B9u;
+    ky += 0xBB67AE85u;
+  }
+  return rk;
+}
+__device__ __forceinline__ uint32_t philox_coord(const PhiloxRoundKeys& rk, uint32_t client_id, uint32_t round, uint32_t coord) {
+  uint4 c = make_uint4(coord, 0u, client_id, round);  // coordinates are below 2^32: counter word 1 is zero
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const unsigned long long p0 = (unsigned long long)0xD2511F53u * c.x, p1 = (unsigned long long)0xCD9E8D57u * c.z;
+    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ rk.x[i], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ rk.y[i], (uint32_t)p0);
+  }
+  return c.x;
+}
+
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
   // first error wins
   atomicCAS(status, 0, code);

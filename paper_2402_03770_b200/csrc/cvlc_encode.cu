@@ -913,6 +913,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
   // error compensation: the encoder's input is memory + update and becomes the new memory, i.e. every sent
   // coordinate gives up what the parameter server will rebuild for it (its centroid value divided by B)
   float* __restrict__ residual = write_residual ? const_cast<float*>(cd.x) : nullptr;
+  const PhiloxRoundKeys rk = philox_round_keys(cd.seed);
 
   const uint32_t mask = reinterpret_cast<const uint32_t*>(ws + L.off_pass_mask)[c];
   const int flips = __popc(~mask & ((1u << kSortPasses) - 1u));
@@ -963,9 +964,17 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
     const unsigned long long* __restrict__ seg = sorted + Z;
     float lo, hi;  // the header's two centroid fields
     // a record's bits, low bit first from packet bit H + j * wd
+    const bool narrow = wd <= 32;  // a record then touches at most two words
     auto put = [&](uint32_t j, unsigned long long rec) {
       const uint32_t bitpos = H + j * wd;
       const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+      if (narrow) {
+        const uint32_t r32 = (uint32_t)rec;
+        const uint32_t p0 = r32 << sh, p1 = __funnelshift_l(r32, 0u, sh);  // the bits that leave the first word
+        if (p0) atomicOr(words + w, p0);
+        if (p1) atomicOr(words + w + 1, p1);
+        return;
+      }
       const unsigned long long lo64 = rec << sh;
       const uint32_t p0 = (uint32_t)lo64, p1 = (uint32_t)(lo64 >> 32);
       const uint32_t p2 = sh ? (uint32_t)(rec >> (64 - sh)) : 0u;
@@ -1000,7 +1009,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         uint32_t level = 0;
         if (norm > 0.0f) {
           const double a = (double)__uint_as_float(key);
-          const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+          const double u = __dmul_rn((double)philox_coord(rk, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
           level = qsgd_quantize_level(a, dn, sqd, sq, scale, u);
         }
         const uint32_t code = (sign << (y - 1)) | level;
@@ -1045,7 +1054,7 @@ k_pack(const __grid_constant__ BatchDesc<CAP> batch, const __grid_constant__ Sha
         uint32_t code = 0;
         if (hi != lo) {
           const double num = __dsub_rn((double)__uint_as_float(b), dlo);
-          const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+          const double u = __dmul_rn((double)philox_coord(rk, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
           code = pq_quantize(num, den, Lc, scale, u);
         }
         put(j, (unsigned long long)pid | ((unsigned long long)code << s));

@@ -132,6 +132,7 @@ k_pack_unframed(const __grid_constant__ BatchDesc<CAP> batch, const __grid_const
   const uint32_t P = __shfl_sync(kFull, capl, src_lane);
   const uint32_t m = uf_rice_param(shape.d, P);
   const unsigned long long* __restrict__ seg = sorted + Z;
+  const PhiloxRoundKeys rk = philox_round_keys(cd.seed);
 
   // ---- the block's records and its centroid distribution (over the records in rank order, as for a packet)
   float vmin = CUDART_INF_F, vmax = -CUDART_INF_F;
@@ -214,7 +215,7 @@ k_pack_unframed(const __grid_constant__ BatchDesc<CAP> batch, const __grid_const
       const uint32_t delta = pid - prev;
       quo = delta >> m;
       uint32_t code = 0;
-      const double u = __dmul_rn((double)philox_coord(cd.seed, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
+      const double u = __dmul_rn((double)philox_coord(rk, cd.client_id, cd.round, pid), 1.0 / 4294967296.0);
       if constexpr (QSGD) {
         const uint32_t key = b & 0x7FFFFFFFu;
         uint32_t level = 0;

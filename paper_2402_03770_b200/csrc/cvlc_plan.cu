@@ -175,7 +175,7 @@ __device__ __forceinline__ double energy_E(uint64_t Z, double beta, double D) {
 }
 
 // ===================================================================================
-// K2  planner: one CTA of 1024 threads
+// K2  planner: per client a fit kernel (one CTA of 1024 threads), a tuning kernel and a small copy kernel
 // ===================================================================================
 
 constexpr int kPlanThreads = 1024;  // the fit kernel: one thread per four histogram bins
@@ -188,7 +188,7 @@ constexpr int kPlanItems = 1024;
 constexpr int kPairSlots = (496 + kTuneThreads - 1) / kTuneThreads;  // pairs of a sweep a thread looks at
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
-// scratch of the length-tuning loop (lives in the dynamic shared memory of the fit points)
+// scratch of the length-tuning loop (the tuning kernel's dynamic shared memory)
 constexpr int kMaxBatchOps = 32;  // atomic operations evaluated together
 struct PlanOp {                   // one atomic operation of a batch
   int i, j;                       // candidate indices, i > j
@@ -206,9 +206,9 @@ struct PlanSolver {
   double Eab[33];                 // energy of the nearest used length at or above l
   unsigned long long Wc[32];      // ranks covered by lengths >= l, current counts
   unsigned used;                  // lengths with a positive count
-  double Ev[1024];                // trial energies, one per item
-  double Fv[1024];                // trial objective values, one per evaluation
-  uint32_t tv[1024];              // trial split of every evaluation (0xFFFFFFFF: not needed)
+  double Ev[kPlanItems];          // trial energies, one per item
+  double Fv[kPlanItems];          // trial objective values, one per evaluation
+  uint32_t tv[kPlanItems];        // trial split of every evaluation (0xFFFFFFFF: not needed)
   PlanOp op[kMaxBatchOps];
   int item_end[kMaxBatchOps];     // exclusive end of every operation's items / evaluations in this round
   int eval_end[kMaxBatchOps];
@@ -216,7 +216,7 @@ struct PlanSolver {
   int next_i, next_j, moved;      // where the sweep resumes after the batch
   uint32_t col_warp[32];          // batch collection: warp totals of the (operations, items) scan
   int col_nops, col_last, col_first_left;  // operations taken; thread of the last one; thread of the first one left over
-  unsigned char ea[1024];         // operation of every evaluation
+  unsigned char ea[kPlanItems];   // operation of every evaluation
 };
 
 struct PlanShared {

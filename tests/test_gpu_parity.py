@@ -381,12 +381,40 @@ def test_host_side_errors_match_oracle(torch_cuda):
         (params_dict(1000, 96, packet_bits=96, scale_B=1.0), B.CVLC_ERR_PACKET_TOO_SMALL),
         (params_dict(100_000, 12000, max_code_bits=3, scale_B=1.0), B.CVLC_ERR_SCALE_TOO_SMALL),
     ]:
-        with pytest.raises(B.CvlcError) as e:
-            gpu_plan_encode(np.ones(pd["d"], np.float32), pd)
-        assert e.value.code == code, pd
+        for compress in (0, 1, 2):
+            with pytest.raises(B.CvlcError) as e:
+                gpu_plan_encode(np.ones(pd["d"], np.float32), pd, compress=compress)
+            assert e.value.code == code, (pd, compress)
         with pytest.raises(O.OracleError) as oe:
             O.plan(np.ones(pd["d"], np.float32), oracle_params(pd))
         assert oe.value.code == code                                             # same numbering on both sides
+
+
+def test_compress_batch_argument_checks(torch_cuda):
+    torch = torch_cuda
+    from paper_2402_03770_b200 import binding as B
+    dev = torch.device("cuda:0")
+    d = 40_000
+    p = B.make_params(d, 8 * 12000)
+    enc = B.BatchEncoder([p, p], dev)
+    xs = [torch.zeros(d, device=dev), torch.zeros(d, device=dev)]
+    small = B.alloc_bytes(1024, dev)
+    for kw, code in ((dict(plan_ws=small), B.CVLC_ERR_WORKSPACE_TOO_SMALL), (dict(enc_ws=small), B.CVLC_ERR_WORKSPACE_TOO_SMALL),
+                     (dict(outs=[small, small]), B.CVLC_ERR_OUTPUT_TOO_SMALL), (dict(fixed_y=33), B.CVLC_ERR_INVALID_ARG)):
+        a = dict(plan_ws=enc.plan_ws, enc_ws=enc.enc_ws, outs=enc.outs, fixed_y=0)
+        a.update(kw)
+        with pytest.raises(B.CvlcError) as e:
+            B.cvlc_compress_batch(xs, enc.params, enc.plans, a["outs"], a["plan_ws"], a["enc_ws"], fixed_y=a["fixed_y"])
+        assert e.value.code == code, kw
+    # the same stream given as side stream: everything runs in order on it
+    s1 = torch.cuda.Stream(device=dev)
+    x = np.random.default_rng(3).laplace(0, 1e-2, d).astype(np.float32)
+    xs = [torch.from_numpy(x).to(dev), torch.from_numpy(-x).to(dev)]
+    enc.compress(xs, stream=s1, side_stream=s1)
+    assert enc.status(s1) == B.CVLC_OK
+    po = oracle_params(params_dict(d, 8 * 12000))
+    ref = O.encode(x, po, O.plan(x, po))
+    assert (enc.outs[0].cpu().numpy() == ref).all()
 
 
 def test_plan_mismatch_is_detected(torch_cuda):

@@ -236,6 +236,39 @@ def test_batched_plan_encode_matches_oracle_per_client(torch_cuda, n):
             assert (outs[c].cpu().numpy() == ost).all(), c
 
 
+def test_clients_that_share_a_tuning_key_get_the_same_lengths(torch_cuda):
+    """clients with the same quantised exponent and scale are tuned once and copy the result: every one of them must
+    still equal its own oracle run (different Philox ids, so different streams)"""
+    torch = torch_cuda
+    from paper_2402_03770_b200 import binding as B
+    from gpu_util import gpu_params
+    dev = torch.device("cuda:0")
+    d = 90_001
+    rng = np.random.default_rng(44)
+    base = [rng.laplace(0, 1e-2, d).astype(np.float32), (rng.standard_t(3, d) * 1e-3).astype(np.float32)]
+    xs, pds = [], []
+    for c in range(7):
+        x = base[c % 2].copy() if c != 6 else np.zeros(d, np.float32)
+        if c == 4:
+            x = -x[::-1].copy()                                   # same magnitudes, other places: same histogram, same key
+        xs.append(x)
+        pds.append(params_dict(d, 15 * 12000, seed=7 + c, client_id=c, round=1, scale_B=1.25 if c == 5 else None))
+    params = [gpu_params(pd) for pd in pds]
+    for side in (False, True):
+        enc = B.BatchEncoder(params, dev)
+        dxs = [torch.from_numpy(x).to(dev) for x in xs]
+        outs = enc.compress(dxs, side_stream=torch.cuda.Stream(device=dev) if side else None)
+        assert enc.status() == 0
+        keys = set()
+        for c in range(7):
+            of, ost = oracle_plan_encode(xs[c], pds[c])
+            gp = enc.read_plan(c)
+            assert_plan_equal(gp, of)
+            assert (outs[c].cpu().numpy() == ost).all(), c
+            keys.add((gp.alpha_q, pds[c]["scale_B"]))
+        assert len(keys) < 7                                       # some clients did share a key
+
+
 def test_batch_rejects_mixed_shapes(torch_cuda):
     torch = torch_cuda
     from paper_2402_03770_b200 import binding as B

@@ -93,12 +93,13 @@ CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
   return P;
 }
 
-// Rows: the float4 units of a segment are also grouped into rows of 32 units (128 coordinates, one warp-wide load)
-// and tiles of 64 rows (the selection kernel's tile).  The histogram kernel leaves the largest magnitude key of every
-// row; once the selection threshold is known the planner turns them into one bit per row ("holds a candidate"), 64
-// rows = one tile per 64-bit word, and the selection kernel skips rows and whole tiles without candidates.  Tile t
-// of the segment that starts at position p0 of the concatenated array has index p0 / 2048 + segment id + t: the
-// index ranges of different segments do not overlap.
+// Rows: the float4 units of a segment are also grouped into rows of 32 units (128 coordinates, one warp-wide load).
+// The histogram kernel leaves the largest magnitude key of every row; once the selection threshold is known the
+// planner lists, per segment and in ascending order, the rows that hold a candidate (a key at or above the threshold).
+// The selection kernel works through that list 64 rows (one tile of its staging buffers) at a time: rows without
+// candidates are neither read nor looked at.  Both tables are indexed by row; row r of the segment that starts at
+// position p0 of the concatenated array sits at 64 * (p0 / 2048 + segment id) + r, so that the index ranges of
+// different segments do not overlap.
 constexpr int kRowUnits = 32;
 constexpr int kTileRows = 64;
 constexpr int kTileUnits = kRowUnits * kTileRows;  // 2048 float4 = 8192 coordinates
@@ -107,8 +108,8 @@ CVLC_HD inline uint64_t seg_first_tile(uint64_t p0, uint32_t seg) { return p0 / 
 
 // plan workspace:
 //   [0] PlanWsHeader | [256] uint64 hist[n][4096] | uint32 nonfinite[n] | uint64 tune_key[n][2] | uint32 leader[n]
-//   | uint32 seg_count[S] | uint64 seg_prefix[S] | uint32 row_max[64 * tiles] | uint64 row_flags[tiles]
-//   | uint32 seg_hist[S][4096]          (S = max_segments, tiles = row_tiles_total)
+//   | uint32 seg_count[S] | uint64 seg_prefix[S] | uint32 seg_rows[S] | uint32 row_max[64 * tiles]
+//   | uint32 row_list[64 * tiles] | uint32 seg_hist[S][4096]          (S = max_segments, tiles = row_tiles_total)
 // tune_key = (bits of alpha_q, bits of scale_B): clients of a batch with equal keys have the same code lengths;
 // leader[c] = the first client of the batch with c's key (it runs the length tuning, the others copy its result).
 struct PlanWsHeader {
@@ -125,12 +126,13 @@ CVLC_HD constexpr size_t plan_off_keys(uint32_t n) { return align256(plan_off_fl
 CVLC_HD constexpr size_t plan_off_leader(uint32_t n) { return align256(plan_off_keys(n) + (size_t)n * 16); }
 CVLC_HD constexpr size_t plan_off_seg_count(uint32_t n) { return align256(plan_off_leader(n) + (size_t)n * 4); }
 CVLC_HD constexpr size_t plan_off_seg_prefix(uint32_t n, uint32_t S) { return align256(plan_off_seg_count(n) + (size_t)S * 4); }
-CVLC_HD constexpr size_t plan_off_row_max(uint32_t n, uint32_t S) { return align256(plan_off_seg_prefix(n, S) + (size_t)S * 8); }
-CVLC_HD constexpr size_t plan_off_row_flags(uint32_t n, uint32_t S, uint64_t tiles) {
+CVLC_HD constexpr size_t plan_off_seg_rows(uint32_t n, uint32_t S) { return align256(plan_off_seg_prefix(n, S) + (size_t)S * 8); }
+CVLC_HD constexpr size_t plan_off_row_max(uint32_t n, uint32_t S) { return align256(plan_off_seg_rows(n, S) + (size_t)S * 4); }
+CVLC_HD constexpr size_t plan_off_row_list(uint32_t n, uint32_t S, uint64_t tiles) {
   return align256(plan_off_row_max(n, S) + (size_t)tiles * kTileRows * 4);
 }
 CVLC_HD constexpr size_t plan_off_seg_hist(uint32_t n, uint32_t S, uint64_t tiles) {
-  return align256(plan_off_row_flags(n, S, tiles) + (size_t)tiles * 8);
+  return align256(plan_off_row_list(n, S, tiles) + (size_t)tiles * kTileRows * 4);
 }
 CVLC_HD constexpr size_t plan_ws_bytes(uint32_t n, uint32_t S, uint64_t tiles) {
   return align256(plan_off_seg_hist(n, S, tiles) + (size_t)S * CVLC_HIST_BINS * 4);

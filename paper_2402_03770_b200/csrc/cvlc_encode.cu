@@ -329,9 +329,9 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
   const uint32_t S = part.max_segments;
   const uint32_t* seg_count = reinterpret_cast<const uint32_t*>(plan_ws + plan_off_seg_count(batch.n));
   const unsigned long long* seg_prefix = reinterpret_cast<const unsigned long long*>(plan_ws + plan_off_seg_prefix(batch.n, S));
-  // one bit per row of 32 units (does it hold a candidate?), one 64-bit word per tile, from the planner
-  const unsigned long long* row_flags =
-      reinterpret_cast<const unsigned long long*>(plan_ws + plan_off_row_flags(batch.n, S, row_tiles_total(part)));
+  // per segment, the rows of 32 units that hold a candidate, in ascending order (from the planner)
+  const uint32_t* row_list = reinterpret_cast<const uint32_t*>(plan_ws + plan_off_row_list(batch.n, S, row_tiles_total(part)));
+  const uint32_t* seg_rows = reinterpret_cast<const uint32_t*>(plan_ws + plan_off_seg_rows(batch.n, S));
   unsigned long long* n_selected = reinterpret_cast<unsigned long long*>(ws + L.off_n_selected);
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;
@@ -371,57 +371,61 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     unsigned long long run = seg_prefix[seg];
     const unsigned long long run0 = run;
     const uint64_t n_vec = (v_end > u0) ? v_end - u0 : 0;        // float4 units of the segment
-    const uint32_t n_tiles = (uint32_t)((n_vec + kTileVec - 1) / kTileVec);
+    // The segment's rows with candidates, 64 at a time: tile v of the staging buffers holds the rows 64 v .. 64 v + 63
+    // of the list, warp w the four rows 64 v + 4 w .. + 3 (ascending rows in ascending lanes: index order is kept).
+    const uint32_t n_listed = seg_rows[seg];
+    const uint32_t n_tiles = (n_listed + kTileRows - 1) / kTileRows;
+    const uint4* __restrict__ quads = reinterpret_cast<const uint4*>(row_list + seg_first_tile(pos, seg) * kTileRows);
 
     // A warp stages exactly the 128 units (512 coordinates) its own lanes will read: four copies of 32
     // consecutive float4s each (coalesced).  Waiting for a tile and reusing a staging slot are then a matter
     // between the lanes of one warp, and the block meets only once per tile, for the scan.
-    // Rows without a candidate are neither copied nor looked at, tiles without one are passed over altogether.
-    const unsigned long long* __restrict__ tile_flags = row_flags + seg_first_tile(pos, seg);
-    auto flags_of = [&](uint32_t t) -> unsigned long long { return t < n_tiles ? __ldg(tile_flags + t) : 0ull; };
+    auto quad_of = [&](uint32_t t) -> uint4 { return t < n_tiles ? __ldg(quads + (size_t)t * 16 + warp) : make_uint4(0u, 0u, 0u, 0u); };
     uint32_t istage = 0;
-    auto issue = [&](uint32_t t, unsigned long long tf) {
-      const uint32_t rows = (uint32_t)(tf >> (4 * warp)) & 0xFu;  // this warp's four rows of the tile
-      if (rows) {  // (a tile past the end has no flags)
+    auto issue = [&](uint32_t t, const uint4 q) {
+      if (t < n_tiles) {
         float4* dst = s_stage + (size_t)istage * kTileVec;
-        const uint64_t base = (uint64_t)t * kTileVec;
+        const uint32_t first_row = t * (uint32_t)kTileRows + 4u * (uint32_t)warp;
+        const uint32_t rowv[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
         for (int v = 0; v < kSelVec; ++v) {
           const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
-          if (((rows >> v) & 1u) && base + g < n_vec) cp_async16(dst + sel_slot(g), xseg + base + g);
+          const uint64_t unit = (uint64_t)rowv[v] * kRowUnits + lane;
+          if (first_row + v < n_listed && unit < n_vec) cp_async16(dst + sel_slot(g), xseg + unit);
         }
       }
       istage = (istage + 1 == kSelStages) ? 0u : istage + 1;
       cp_async_commit();  // one group per tile slot, empty past the end, keeps the group count uniform
     };
 
-    static_assert(kSelStages == 3, "the flag words of three tiles are carried along");
-    unsigned long long f0 = flags_of(0), f1 = flags_of(1), f2 = flags_of(2);
-    issue(0, f0);
-    issue(1, f1);
+    static_assert(kSelStages == 3, "the row lists of three tiles are carried along");
+    uint4 q0 = quad_of(0), q1 = quad_of(1), q2 = quad_of(2);
+    issue(0, q0);
+    issue(1, q1);
     uint32_t stage = 0;
     for (uint32_t t = 0; t < n_tiles; ++t) {
-      const unsigned long long tile_rows = f0;
-      const unsigned long long f3 = flags_of(t + 3);  // asked for one tile before it is needed
+      const uint4 qt = q0;
+      const uint4 q3 = quad_of(t + 3);  // asked for one tile before it is needed
       cp_async_wait<kSelStages - 2>();  // this lane's copies of tile t have landed
       __syncwarp();                     // ... and the other lanes'; and the warp is done with its part of tile t - 1,
-      issue(t + kSelStages - 1, f2);    // whose staging slot the next copies overwrite
-      f0 = f1;
-      f1 = f2;
-      f2 = f3;
+      issue(t + kSelStages - 1, q2);    // whose staging slot the next copies overwrite
+      q0 = q1;
+      q1 = q2;
+      q2 = q3;
       const float4* src = s_stage + (size_t)stage * kTileVec;
       stage = (stage + 1 == kSelStages) ? 0u : stage + 1;
-      if (tile_rows == 0ull) continue;  // the same for the whole block
-      const uint64_t base = (uint64_t)t * kTileVec;
-      // this thread's 16 consecutive coordinates: units 4 tid .. 4 tid + 3 of the tile
+      // this thread's 16 consecutive coordinates: units 4 (lane & 7) .. + 3 of the row its quarter of the warp reads
       uint32_t m = 0;
       const uint32_t g0 = (uint32_t)kSelVec * tid;
       const uint32_t ct = ((uint32_t)tid >> 1) & (uint32_t)(kSelVec - 1);
-      const uint32_t left = (base + g0 < n_vec) ? (uint32_t)((n_vec - base - g0 < kSelVec) ? n_vec - base - g0 : kSelVec) : 0u;
-      const bool row_on = (tile_rows >> (4 * warp + (lane >> 3))) & 1ull;  // the thread's four units lie in one row
+      const uint32_t quarter = (uint32_t)lane >> 3;
+      const uint32_t my_row = quarter == 0 ? qt.x : quarter == 1 ? qt.y : quarter == 2 ? qt.z : qt.w;
+      const bool row_on = t * (uint32_t)kTileRows + 4u * (uint32_t)warp + quarter < n_listed;
+      const uint64_t unit0 = (uint64_t)my_row * kRowUnits + ((uint32_t)lane & 7u) * kSelVec;  // first unit of the thread, in the segment
+      const uint32_t left = (row_on && unit0 < n_vec) ? (uint32_t)((n_vec - unit0 < kSelVec) ? n_vec - unit0 : kSelVec) : 0u;
 #pragma unroll
       for (int j = 0; j < kSelVec; ++j) {
-        if (row_on && (uint32_t)j < left) {
+        if ((uint32_t)j < left) {
           // units 4 tid + j sit in slots 4 tid + (j ^ ct): the swizzle only touches the two low bits
           const float4 f = src[g0 + ((uint32_t)j ^ ct)];
           m = __funnelshift_l(__float_as_uint(__fsub_rn(below_thresh_f, fabsf(f.x))), m, 1);
@@ -458,7 +462,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       uint32_t o = (uint32_t)run + below + incl - cnt;  // positions inside a client's buffer fit 32 bits
       const uint32_t* srcw16 = reinterpret_cast<const uint32_t*>(src) + 16 * tid;  // this thread's 16 staged words
       const uint32_t cx = ct << 2;
-      const uint32_t e32 = (uint32_t)((u0 + base + g0) * 4);  // index of the thread's first coordinate (< 2^31)
+      const uint32_t e32 = (uint32_t)((u0 + unit0) * 4);  // index of the thread's first coordinate (< 2^31)
       while (m) {
         const int hb = 31 - __clz(m);  // highest flag = lowest index first
         m ^= 1u << hb;

@@ -483,36 +483,40 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
       for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
       if (lane == 0) seg_count[b + c] = sum;
     }
-    // one bit per row of 128 coordinates: does the row hold a candidate (a key at or above the threshold)?
-    // Tile t (64 rows) of a segment is one 64-bit word; lanes 2w, 2w+1 ... : a warp turns 32 rows into one half word.
+    // the rows of 128 coordinates that hold a candidate (a key at or above the threshold), listed per segment in
+    // ascending order: one warp per segment walks its rows 32 at a time, four loads in flight
     {
       const uint32_t* row_max = reinterpret_cast<const uint32_t*>(ws + plan_off_row_max(batch.n, S));
-      uint32_t* row_flags = reinterpret_cast<uint32_t*>(ws + plan_off_row_flags(batch.n, S, row_tiles));
+      uint32_t* row_list = reinterpret_cast<uint32_t*>(ws + plan_off_row_list(batch.n, S, row_tiles));
+      uint32_t* seg_rows = reinterpret_cast<uint32_t*>(ws + plan_off_seg_rows(batch.n, S));
       const uint32_t thresh_key = jt << 19;
       const uint64_t nvec = shape.d >> 2;
-      for (uint32_t b = b0; b <= b1; ++b) {
+      const unsigned lt = (1u << lane) - 1u;
+      for (uint32_t b = b0 + warp; b <= b1; b += kPlanThreads / 32) {
         const uint64_t p0 = (first > (uint64_t)b * part.chunk) ? first : (uint64_t)b * part.chunk;
         uint64_t p1 = ((uint64_t)(b + 1) * part.chunk < first + part.units) ? (uint64_t)(b + 1) * part.chunk : first + part.units;
         if (p1 > first + nvec) p1 = first + nvec;  // the client's last unit is its ragged tail, not a float4
         const uint64_t n_units = p1 > p0 ? p1 - p0 : 0;
         const uint64_t n_rows = (n_units + kRowUnits - 1) / kRowUnits;
-        const uint64_t n_words = (n_rows + 31) / 32;          // half words of row flags
-        const uint64_t tile0 = seg_first_tile(p0, b + c);
-        const uint64_t n_half = (n_words + 1) & ~(uint64_t)1;  // whole 64-bit words
-        for (uint64_t w0 = (uint64_t)warp * 4; w0 < n_half; w0 += 4 * (kPlanThreads / 32)) {  // four loads in flight
+        const uint64_t base = seg_first_tile(p0, b + c) * kTileRows;
+        uint32_t listed = 0;
+        for (uint64_t r0 = 0; r0 < n_rows; r0 += 128) {
           uint32_t mx[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint64_t r = (w0 + j) * 32 + lane;
-            mx[j] = (r < n_rows) ? row_max[tile0 * kTileRows + r] : 0u;
+            const uint64_t r = r0 + (uint64_t)j * 32 + lane;
+            mx[j] = (r < n_rows) ? row_max[base + r] : 0u;
           }
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint64_t r = (w0 + j) * 32 + lane;
-            const unsigned bits = __ballot_sync(kFull, (r < n_rows) && mx[j] >= thresh_key);
-            if (lane == 0 && w0 + j < n_half) row_flags[tile0 * 2 + w0 + j] = bits;
+            const uint64_t r = r0 + (uint64_t)j * 32 + lane;
+            const bool on = (r < n_rows) && mx[j] >= thresh_key;
+            const unsigned bits = __ballot_sync(kFull, on);
+            if (on) row_list[base + listed + __popc(bits & lt)] = (uint32_t)r;
+            listed += __popc(bits);
           }
         }
+        if (lane == 0) seg_rows[b + c] = listed;
       }
     }
     __syncthreads();

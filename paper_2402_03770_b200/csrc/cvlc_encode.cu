@@ -373,6 +373,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     const uint64_t n_vec = (v_end > u0) ? v_end - u0 : 0;        // float4 units of the segment
     // The segment's rows with candidates, 64 at a time: tile v of the staging buffers holds the rows 64 v .. 64 v + 63
     // of the list, warp w the four rows 64 v + 4 w .. + 3 (ascending rows in ascending lanes: index order is kept).
+    const uint32_t n_vec32 = (uint32_t)n_vec;  // a segment is at most one chunk: far below 2^32 units
     const uint32_t n_listed = seg_rows[seg];
     const uint32_t n_tiles = (n_listed + kTileRows - 1) / kTileRows;
     const uint4* __restrict__ quads = reinterpret_cast<const uint4*>(row_list + seg_first_tile(pos, seg) * kTileRows);
@@ -390,8 +391,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
 #pragma unroll
         for (int v = 0; v < kSelVec; ++v) {
           const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
-          const uint64_t unit = (uint64_t)rowv[v] * kRowUnits + lane;
-          if (first_row + v < n_listed && unit < n_vec) cp_async16(dst + sel_slot(g), xseg + unit);
+          const uint32_t unit = rowv[v] * (uint32_t)kRowUnits + (uint32_t)lane;
+          if (first_row + v < n_listed && unit < n_vec32) cp_async16(dst + sel_slot(g), xseg + unit);
         }
       }
       istage = (istage + 1 == kSelStages) ? 0u : istage + 1;
@@ -421,8 +422,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       const uint32_t quarter = (uint32_t)lane >> 3;
       const uint32_t my_row = quarter == 0 ? qt.x : quarter == 1 ? qt.y : quarter == 2 ? qt.z : qt.w;
       const bool row_on = t * (uint32_t)kTileRows + 4u * (uint32_t)warp + quarter < n_listed;
-      const uint64_t unit0 = (uint64_t)my_row * kRowUnits + ((uint32_t)lane & 7u) * kSelVec;  // first unit of the thread, in the segment
-      const uint32_t left = (row_on && unit0 < n_vec) ? (uint32_t)((n_vec - unit0 < kSelVec) ? n_vec - unit0 : kSelVec) : 0u;
+      const uint32_t unit0 = my_row * (uint32_t)kRowUnits + ((uint32_t)lane & 7u) * kSelVec;  // first unit of the thread, in the segment
+      const uint32_t left = (row_on && unit0 < n_vec32) ? ((n_vec32 - unit0 < (uint32_t)kSelVec) ? n_vec32 - unit0 : (uint32_t)kSelVec) : 0u;
 #pragma unroll
       for (int j = 0; j < kSelVec; ++j) {
         if ((uint32_t)j < left) {

@@ -476,7 +476,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 data / f64 plan+quantizer / u32 keys", "data": "synthetic",
         "config": {"workload": f"{w.name} d={d} clients={n_clients} bits_per_coord={bpc} quantizer={args.quantizer} packet=1500B",
-                   "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams, "clients_per_call": batch, "max_candidates": int(max_cand),
+                   "l2": "inputs (4*d*clients bytes per step) exceed L2", "streams": n_streams, "side_stream_for_length_tuning": not args.no_side_stream, "clients_per_call": batch, "max_candidates": int(max_cand),
                    "multi_gpu": "replicas only: every rank runs its own clients and aggregator"},
         "params_per_s": units / (ms_per_step * 1e-3),
         "step_min_bytes_frac_of_hbm_peak": step_frac,

@@ -484,7 +484,7 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
       if (lane == 0) seg_count[b + c] = sum;
     }
     // the rows of 128 coordinates that hold a candidate (a key at or above the threshold), listed per segment in
-    // ascending order: one warp per segment walks its rows 32 at a time, four loads in flight
+    // ascending order: one warp per segment walks its rows 32 at a time, eight loads in flight
     {
       const uint32_t* row_max = reinterpret_cast<const uint32_t*>(ws + plan_off_row_max(batch.n, S));
       uint32_t* row_list = reinterpret_cast<uint32_t*>(ws + plan_off_row_list(batch.n, S, row_tiles));
@@ -500,15 +500,15 @@ k_plan_fit(const unsigned long long* __restrict__ hist_all, const uint32_t* __re
         const uint64_t n_rows = (n_units + kRowUnits - 1) / kRowUnits;
         const uint64_t base = seg_first_tile(p0, b + c) * kTileRows;
         uint32_t listed = 0;
-        for (uint64_t r0 = 0; r0 < n_rows; r0 += 128) {
-          uint32_t mx[4];
+        for (uint64_t r0 = 0; r0 < n_rows; r0 += 256) {
+          uint32_t mx[8];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
+          for (int j = 0; j < 8; ++j) {
             const uint64_t r = r0 + (uint64_t)j * 32 + lane;
             mx[j] = (r < n_rows) ? row_max[base + r] : 0u;
           }
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
+          for (int j = 0; j < 8; ++j) {
             const uint64_t r = r0 + (uint64_t)j * 32 + lane;
             const bool on = (r < n_rows) && mx[j] >= thresh_key;
             const unsigned bits = __ballot_sync(kFull, on);

@@ -93,16 +93,16 @@ CVLC_HD inline Partition make_partition(uint64_t d, uint32_t n) {
   return P;
 }
 
-// Rows: the float4 units of a segment are also grouped into rows of 32 units (128 coordinates, one warp-wide load).
-// The histogram kernel leaves the largest magnitude key of every row; once the selection threshold is known the
-// planner lists, per segment and in ascending order, the rows that hold a candidate (a key at or above the threshold).
-// The selection kernel works through that list 64 rows (one tile of its staging buffers) at a time: rows without
-// candidates are neither read nor looked at.  Both tables are indexed by row; row r of the segment that starts at
-// position p0 of the concatenated array sits at 64 * (p0 / 2048 + segment id) + r, so that the index ranges of
-// different segments do not overlap.
-constexpr int kRowUnits = 32;
-constexpr int kTileRows = 64;
-constexpr int kTileUnits = kRowUnits * kTileRows;  // 2048 float4 = 8192 coordinates
+// Rows: the float4 units of a segment are also grouped into rows of 16 units (64 coordinates, half of a warp-wide
+// load).  The histogram kernel leaves the largest magnitude key of every row; once the selection threshold is known
+// the planner lists, per segment and in ascending order, the rows that hold a candidate (a key at or above the
+// threshold).  The selection kernel works through that list 128 rows (one tile of its staging buffers) at a time:
+// rows without candidates are neither read nor looked at.  Both tables are indexed by row; row r of the segment that
+// starts at position p0 of the concatenated array sits at 128 * (p0 / 2048 + segment id) + r, so that the index
+// ranges of different segments do not overlap.
+constexpr int kRowUnits = 16;
+constexpr int kTileUnits = 2048;                    // 2048 float4 = 8192 coordinates: a tile of the selection kernel
+constexpr int kTileRows = kTileUnits / kRowUnits;   // 128
 CVLC_HD inline uint64_t row_tiles_total(const Partition& P) { return P.total / kTileUnits + P.max_segments + 1; }
 CVLC_HD inline uint64_t seg_first_tile(uint64_t p0, uint32_t seg) { return p0 / kTileUnits + seg; }
 

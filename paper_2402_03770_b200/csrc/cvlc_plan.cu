@@ -57,8 +57,10 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     const float* __restrict__ x = batch.c[c].x;
     const float4* xv = reinterpret_cast<const float4*>(x);
     const uint64_t v1 = (u1 < nvec) ? u1 : nvec;  // float4 units of this segment: [u0, v1)
-    // largest key of every row (32 consecutive units from u0 on: what one warp loads at a time)
+    // largest key of every row (16 consecutive units from u0 on: what half a warp loads at a time)
     uint32_t* __restrict__ row_max = row_max_all + seg_first_tile(pos, (uint32_t)(q + c)) * kTileRows;
+    static_assert(kRowUnits == 16, "a row is what one half of a warp loads");
+    const bool upper = (lane & 16) != 0;  // two whole-warp reductions per load, each seeing one half's keys
     uint32_t top = 0;
     uint64_t v = u0 + threadIdx.x;
     // four independent 128-bit loads in flight per thread; the loop condition is the same for the lanes of a warp
@@ -68,16 +70,20 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
       for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * kHistThreads);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, hist_add4(my, a[u]));
+        const uint32_t mk = hist_add4(my, a[u]);
+        const uint32_t m_lo = __reduce_max_sync(0xFFFFFFFFu, upper ? 0u : mk), m_hi = __reduce_max_sync(0xFFFFFFFFu, upper ? mk : 0u);
+        const uint32_t m = upper ? m_hi : m_lo;
         top = m > top ? m : top;
-        if (lane == 0) row_max[(v - u0 + u * kHistThreads) >> 5] = m;
+        if ((lane & 15) == 0) row_max[(v - u0 + u * kHistThreads) >> 4] = m;
       }
     }
     for (; v - lane < v1; v += kHistThreads) {  // rows that may end inside the warp
       const bool on = v < v1;
-      const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, on ? hist_add4(my, __ldg(xv + v)) : 0u);
+      const uint32_t mk = on ? hist_add4(my, __ldg(xv + v)) : 0u;
+      const uint32_t m_lo = __reduce_max_sync(0xFFFFFFFFu, upper ? 0u : mk), m_hi = __reduce_max_sync(0xFFFFFFFFu, upper ? mk : 0u);
+      const uint32_t m = upper ? m_hi : m_lo;
       top = m > top ? m : top;
-      if (lane == 0) row_max[(v - u0) >> 5] = m;
+      if ((lane & 15) == 0 && on) row_max[(v - u0) >> 4] = m;
     }
     // ragged tail of the client (d not a multiple of 4)
     if (u1 == units && threadIdx.x < (d & 3)) {

@@ -39,10 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 # proportion to the clients); scaled to the clients of a launch, None for any other configuration, for fewer than
 # 32 clients per launch, and for a kernel that has changed since its capture.
 NCU_TRAFFIC_BYTES_PER_CLIENT = {
-    "k_hist": (1434.16e6 + 48.11e6) / 32,          # the update once, plus row maxima and per-segment histograms
-    "k_select": (518.13e6 + 165.32e6) / 32,        # the rows that hold candidates (36 % of the update), plus the candidates
-    "k_sort_pass": (208.88e6 + 174.21e6 + 209.78e6 + 174.55e6 + 206.08e6 + 174.17e6 + 0.08e6) / 32 / 4,  # mean of a step's four launches
-    "k_pack": (178.00e6 + 52.35e6) / 32,
+    "k_hist": (1434.27e6 + 58.85e6) / 32,          # the update once, plus row maxima and per-segment histograms
+    "k_select": (477.15e6 + 164.51e6) / 32,        # the rows that hold candidates (a third of the update), plus the candidates
+    "k_sort_pass": (209.78e6 + 174.11e6 + 208.96e6 + 173.35e6 + 206.46e6 + 173.98e6 + 0.08e6) / 32 / 4,  # mean of a step's four launches
+    "k_pack": (177.98e6 + 54.22e6) / 32,
 }
 NOMINAL_HBM_GBS = 8000.0
 

@@ -336,7 +336,8 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
   const uint64_t nvec = d >> 2;
   const uint64_t units = part.units;
   constexpr uint32_t kTileVec = kSelTileVec;
-  static_assert(kSelTileVec == kTileUnits && kRowUnits == 16 && kSelVec == 4, "a warp stages eight rows of a tile, four lanes read a row");
+  static_assert(kSelTileVec == kTileUnits && kSelVec == 4 && kRowUnits % kSelVec == 0 && 32 % kRowUnits == 0,
+                "a warp stages whole rows of a tile, a thread's four units lie in one row");
   int parity = 0;
   __shared__ uint32_t s_chunk;
 
@@ -371,27 +372,28 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     unsigned long long run = seg_prefix[seg];
     const unsigned long long run0 = run;
     const uint64_t n_vec = (v_end > u0) ? v_end - u0 : 0;        // float4 units of the segment
-    // The segment's rows with candidates, 128 at a time: tile t of the staging buffers holds the rows 128 t .. 128 t + 127
-    // of the list, warp w the eight rows 128 t + 8 w .. + 7 (ascending rows in ascending lanes: index order is kept).
-    constexpr uint32_t kRowsPerWarp = 32 * kSelVec / kRowUnits;  // 8
+    // The segment's rows with candidates, a tile (kTileRows of them) at a time: tile t of the staging buffers holds the
+    // rows kTileRows t .. of the list, warp w the next kRowsPerWarp of them (ascending rows in ascending lanes: index
+    // order is kept).
+    constexpr uint32_t kRowsPerWarp = 32 * kSelVec / kRowUnits;
     const uint32_t n_vec32 = (uint32_t)n_vec;  // a segment is at most one chunk: far below 2^32 units
     const uint32_t n_listed = seg_rows[seg];
     const uint32_t n_tiles = (n_listed + kTileRows - 1) / kTileRows;
     const uint32_t* __restrict__ list = row_list + seg_first_tile(pos, seg) * kTileRows;
     constexpr uint32_t kNoRow = 0xFFFFFFFFu;
-    auto row_at = [&](uint32_t t, uint32_t slot) -> uint32_t {  // the row in slot `slot` (0 .. 7) of this warp's part of tile t
+    auto row_at = [&](uint32_t t, uint32_t slot) -> uint32_t {  // the row in slot `slot` of this warp's part of tile t
       const uint32_t idx = t * (uint32_t)kTileRows + (uint32_t)warp * kRowsPerWarp + slot;
       return (idx < n_listed) ? __ldg(list + idx) : kNoRow;
     };
 
     // A warp stages exactly the 128 units (512 coordinates) its own lanes will read: four copies of 32 float4s each,
-    // two rows per copy.  Waiting for a tile and reusing a staging slot are then a matter between the lanes of one
+    // 32 / kRowUnits rows per copy.  Waiting for a tile and reusing a staging slot are then a matter between the lanes of one
     // warp, and the block meets only once per tile, for the scan.
     struct CopyRows { uint32_t r[kSelVec]; };
-    auto copy_rows_of = [&](uint32_t t) -> CopyRows {  // the rows this lane copies from in tile t: copy v covers the slots 2 v, 2 v + 1
+    auto copy_rows_of = [&](uint32_t t) -> CopyRows {  // the rows this lane copies from in tile t, one per copy
       CopyRows cr;
 #pragma unroll
-      for (int v = 0; v < kSelVec; ++v) cr.r[v] = row_at(t, 2u * (uint32_t)v + ((uint32_t)lane >> 4));
+      for (int v = 0; v < kSelVec; ++v) cr.r[v] = row_at(t, ((uint32_t)v * 32u + (uint32_t)lane) / kRowUnits);
       return cr;
     };
     uint32_t istage = 0;
@@ -400,7 +402,7 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
 #pragma unroll
       for (int v = 0; v < kSelVec; ++v) {
         const uint32_t g = (uint32_t)(warp * (32 * kSelVec) + v * 32 + lane);
-        const uint32_t unit = cr.r[v] * (uint32_t)kRowUnits + ((uint32_t)lane & 15u);
+        const uint32_t unit = cr.r[v] * (uint32_t)kRowUnits + (uint32_t)lane % kRowUnits;
         if (cr.r[v] != kNoRow && unit < n_vec32) cp_async16(dst + sel_slot(g), xseg + unit);
       }
       istage = (istage + 1 == kSelStages) ? 0u : istage + 1;
@@ -411,12 +413,13 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
     issue(copy_rows_of(0));
     issue(copy_rows_of(1));
     CopyRows ahead = copy_rows_of(2);                 // for the copies of tile t + 2
-    uint32_t mine = row_at(0, (uint32_t)lane >> 2);   // the row this thread reads in tile t
-    uint32_t mine_next = row_at(1, (uint32_t)lane >> 2);
+    const uint32_t my_slot = (uint32_t)lane * kSelVec / kRowUnits;  // the slot of the row this thread's four units lie in
+    uint32_t mine = row_at(0, my_slot);                              // the row this thread reads in tile t
+    uint32_t mine_next = row_at(1, my_slot);
     uint32_t stage = 0;
     for (uint32_t t = 0; t < n_tiles; ++t) {
       const CopyRows ahead2 = copy_rows_of(t + 3);    // asked for one tile before they are needed
-      const uint32_t mine_next2 = row_at(t + 2, (uint32_t)lane >> 2);
+      const uint32_t mine_next2 = row_at(t + 2, my_slot);
       cp_async_wait<kSelStages - 2>();  // this lane's copies of tile t have landed
       __syncwarp();                     // ... and the other lanes'; and the warp is done with its part of tile t - 1,
       issue(ahead);                     // whose staging slot the next copies overwrite
@@ -426,11 +429,11 @@ k_select(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_
       mine_next = mine_next2;
       const float4* src = s_stage + (size_t)stage * kTileVec;
       stage = (stage + 1 == kSelStages) ? 0u : stage + 1;
-      // this thread's 16 consecutive coordinates: units 4 (lane & 3) .. + 3 of the row its four lanes read
+      // this thread's 16 consecutive coordinates: four units of the row that it reads with its neighbours
       uint32_t m = 0;
       const uint32_t g0 = (uint32_t)kSelVec * tid;
       const uint32_t ct = ((uint32_t)tid >> 1) & (uint32_t)(kSelVec - 1);
-      const uint32_t unit0 = my_row * (uint32_t)kRowUnits + ((uint32_t)lane & 3u) * kSelVec;  // first unit of the thread, in the segment
+      const uint32_t unit0 = my_row * (uint32_t)kRowUnits + ((uint32_t)lane * kSelVec) % kRowUnits;  // first unit of the thread, in the segment
       const uint32_t left = (my_row != kNoRow && unit0 < n_vec32) ? ((n_vec32 - unit0 < (uint32_t)kSelVec) ? n_vec32 - unit0 : (uint32_t)kSelVec) : 0u;
 #pragma unroll
       for (int j = 0; j < kSelVec; ++j) {

@@ -57,10 +57,21 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     const float* __restrict__ x = batch.c[c].x;
     const float4* xv = reinterpret_cast<const float4*>(x);
     const uint64_t v1 = (u1 < nvec) ? u1 : nvec;  // float4 units of this segment: [u0, v1)
-    // largest key of every row (16 consecutive units from u0 on: what half a warp loads at a time)
+    // largest key of every row (kRowUnits consecutive units from u0 on: a warp-wide load covers 32 / kRowUnits rows);
+    // one whole-warp reduction per row of a load, each seeing that row's keys only
     uint32_t* __restrict__ row_max = row_max_all + seg_first_tile(pos, (uint32_t)(q + c)) * kTileRows;
-    static_assert(kRowUnits == 16, "a row is what one half of a warp loads");
-    const bool upper = (lane & 16) != 0;  // two whole-warp reductions per load, each seeing one half's keys
+    static_assert(32 % kRowUnits == 0, "a warp-wide load covers whole rows");
+    constexpr int kRowsPerLoad = 32 / kRowUnits;
+    const int my_group = lane / kRowUnits;
+    auto row_maxima = [&](uint32_t mk) -> uint32_t {  // the largest key among the lanes of this lane's row
+      uint32_t mine = 0;
+#pragma unroll
+      for (int g = 0; g < kRowsPerLoad; ++g) {
+        const uint32_t mg = __reduce_max_sync(0xFFFFFFFFu, my_group == g ? mk : 0u);
+        if (my_group == g) mine = mg;
+      }
+      return mine;
+    };
     uint32_t top = 0;
     uint64_t v = u0 + threadIdx.x;
     // four independent 128-bit loads in flight per thread; the loop condition is the same for the lanes of a warp
@@ -70,20 +81,16 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
       for (int u = 0; u < 4; ++u) a[u] = __ldg(xv + v + u * kHistThreads);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t mk = hist_add4(my, a[u]);
-        const uint32_t m_lo = __reduce_max_sync(0xFFFFFFFFu, upper ? 0u : mk), m_hi = __reduce_max_sync(0xFFFFFFFFu, upper ? mk : 0u);
-        const uint32_t m = upper ? m_hi : m_lo;
+        const uint32_t m = row_maxima(hist_add4(my, a[u]));
         top = m > top ? m : top;
-        if ((lane & 15) == 0) row_max[(v - u0 + u * kHistThreads) >> 4] = m;
+        if (lane % kRowUnits == 0) row_max[(v - u0 + u * kHistThreads) / kRowUnits] = m;
       }
     }
     for (; v - lane < v1; v += kHistThreads) {  // rows that may end inside the warp
       const bool on = v < v1;
-      const uint32_t mk = on ? hist_add4(my, __ldg(xv + v)) : 0u;
-      const uint32_t m_lo = __reduce_max_sync(0xFFFFFFFFu, upper ? 0u : mk), m_hi = __reduce_max_sync(0xFFFFFFFFu, upper ? mk : 0u);
-      const uint32_t m = upper ? m_hi : m_lo;
+      const uint32_t m = row_maxima(on ? hist_add4(my, __ldg(xv + v)) : 0u);
       top = m > top ? m : top;
-      if ((lane & 15) == 0 && on) row_max[(v - u0) >> 4] = m;
+      if (lane % kRowUnits == 0 && on) row_max[(v - u0) / kRowUnits] = m;
     }
     // ragged tail of the client (d not a multiple of 4)
     if (u1 == units && threadIdx.x < (d & 3)) {

@@ -64,13 +64,22 @@ k_hist(const __grid_constant__ BatchDesc<CAP> batch, uint64_t d, const __grid_co
     constexpr int kRowsPerLoad = 32 / kRowUnits;
     const int my_group = lane / kRowUnits;
     auto row_maxima = [&](uint32_t mk) -> uint32_t {  // the largest key among the lanes of this lane's row
-      uint32_t mine = 0;
+      if constexpr (kRowsPerLoad <= 2) {  // few rows per load: one whole-warp reduction per row, each seeing that row's keys only
+        uint32_t mine = 0;
 #pragma unroll
-      for (int g = 0; g < kRowsPerLoad; ++g) {
-        const uint32_t mg = __reduce_max_sync(0xFFFFFFFFu, my_group == g ? mk : 0u);
-        if (my_group == g) mine = mg;
+        for (int g = 0; g < kRowsPerLoad; ++g) {
+          const uint32_t mg = __reduce_max_sync(0xFFFFFFFFu, my_group == g ? mk : 0u);
+          if (my_group == g) mine = mg;
+        }
+        return mine;
+      } else {  // more rows per load: a butterfly inside the row's lanes
+#pragma unroll
+        for (int off = 1; off < kRowUnits; off <<= 1) {
+          const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, mk, off);
+          mk = o > mk ? o : mk;
+        }
+        return mk;
       }
-      return mine;
     };
     uint32_t top = 0;
     uint64_t v = u0 + threadIdx.x;

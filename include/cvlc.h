@@ -229,9 +229,11 @@ int cvlc_plan_literal(const cvlc_params* p, double alpha_q, uint32_t n_k, uint32
  * stream_dev (16-byte aligned) receives cvlc_stream_bytes(p) bytes.
  * plan_dev must come from cvlc_plan / cvlc_plan_fixed on the same x_dev and params.
  * plan_ws_dev: the workspace that call used, untouched since (it holds per-chunk candidate
- * counts that let the selection run without any exchange between thread blocks), or NULL
- * when it is gone or the plan came from elsewhere: the selection then computes its output
- * offsets itself with a decoupled look-back scan across blocks (slower).
+ * counts that let the selection run without any exchange between thread blocks, and the list
+ * of the 64-coordinate rows that hold a candidate, so that the rest of the update is not read
+ * a second time), or NULL when it is gone or the plan came from elsewhere: the selection then
+ * reads the whole update and computes its output offsets itself with a decoupled look-back
+ * scan across blocks (slower).
  * Errors: INVALID_ARG, OUTPUT_TOO_SMALL, WORKSPACE_TOO_SMALL (host); PLAN_MISMATCH,
  * DEVICE_TIMEOUT (device, at byte 0 of ws_dev).
  */
